@@ -1,0 +1,182 @@
+"""Pins for the oracle's bucketed-LRU step (Section 5.3).  CPU only."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import spin_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "lru_worked_example.txt")
+
+
+def _fresh(S):
+    return (np.full(S, -1, dtype=np.int64), np.zeros(S, dtype=np.int64),
+            np.full(S, -1, dtype=np.int64))
+
+
+def test_hand_derived_worked_example():
+    part, pidx, ts = _fresh(4)
+    resident = np.zeros(16, dtype=np.int64)
+    npages = np.ones(16, dtype=np.int64)
+    for line in open(GOLDEN):
+        if line.startswith("#") or not line.strip():
+            continue
+        step, sel, slots = [x.strip() for x in line.split("|")]
+        O.bucketed_lru_step(part, pidx, ts, resident, npages,
+                            [int(x) for x in sel.split()], int(step), 4)
+        got = " ".join("-" if part[s] < 0 else f"{part[s]}:{ts[s]}" for s in range(4))
+        assert got == " ".join(slots.split()), f"step {step}"
+
+
+def closed_form_ts(a, t, n):
+    """Timestamp at step t of a page last touched at step a <= t: it got min(a, n-1); one
+    demotion happens at every later step whose counter exceeds n-1; floor 0."""
+    demotions = sum(1 for u in range(a + 1, t + 1) if u > n - 1)
+    return max(0, min(a, n - 1) - demotions)
+
+
+class BruteLru:
+    """Independent simulator: remembers only WHEN each cached page was last used and
+    derives everything else (timestamps, victims) from that by the closed form."""
+
+    def __init__(self, S, n):
+        self.S, self.n = S, n
+        self.slot = [None] * S            # (partition, page_idx) or None
+        self.last = {}                    # partition -> step of last use
+        self.pageless = set()             # partitions without pages, once "admitted"
+
+    def step(self, selected, npages, t):
+        cached = {p for e in self.slot if e for p in [e[0]]} | self.pageless
+        hits = [p for p in selected if p in cached]
+        misses = [p for p in selected if p not in cached]
+        for p in hits:
+            self.last[p] = t
+        demand = sum(npages[p] for p in misses)
+        evicted = []
+        if demand:
+            def ts(e):
+                return -1 if e is None else closed_form_ts(self.last[e[0]], t, self.n)
+            pool = [s for s in range(self.S) if self.slot[s] is None or self.slot[s][0] not in hits]
+            x = self.n - 1
+            for cand in range(-1, self.n):
+                if sum(1 for s in pool if ts(self.slot[s]) <= cand) >= demand:
+                    x = cand
+                    break
+            for s in pool:
+                if self.slot[s] is not None and ts(self.slot[s]) <= x:
+                    evicted.append((s,) + self.slot[s])
+                    self.slot[s] = None
+        free = [s for s in range(self.S) if self.slot[s] is None]
+        bypass = []
+        for p in misses:
+            if npages[p] <= len(free):
+                for i in range(npages[p]):
+                    self.slot[free.pop(0)] = (p, i)
+                self.last[p] = t
+                if npages[p] == 0:        # nothing to cache: resident from now on
+                    self.pageless.add(p)
+            else:
+                bypass.append(p)
+        return hits, misses, evicted, bypass
+
+    def view(self, t):
+        part = [-1 if e is None else e[0] for e in self.slot]
+        pidx = [0 if e is None else e[1] for e in self.slot]
+        ts = [-1 if e is None else closed_form_ts(self.last[e[0]], t, self.n) for e in self.slot]
+        return part, pidx, ts
+
+
+@pytest.mark.parametrize("S,n,P,k,multi", [(8, 4, 40, 3, False), (16, 8, 30, 5, False),
+                                           (24, 3, 30, 4, True), (12, 1, 20, 3, False),
+                                           (40, 64, 25, 6, True), (6, 5, 50, 5, True)])
+def test_against_last_use_simulator(S, n, P, k, multi):
+    rng = np.random.default_rng(S * 1000 + n)
+    npages = (rng.integers(1, 4, size=P) if multi else np.ones(P, dtype=np.int64)).astype(np.int64)
+    if multi:
+        npages[0] = 0                                           # an empty partition
+    part, pidx, ts = _fresh(S)
+    resident = np.zeros(P, dtype=np.int64)
+    brute = BruteLru(S, n)
+    hot = rng.permutation(P)[: 3 * k]
+    for t in range(4 * n + 40):
+        pool = hot if rng.random() < 0.7 else np.arange(P)      # temporal locality + noise
+        sel = sorted(set(int(x) for x in rng.choice(pool, size=k)))
+        res = O.bucketed_lru_step(part, pidx, ts, resident, npages, sel, t, n)
+        hits, misses, evicted, bypass = brute.step(sel, npages, t)
+        assert (res.hits, res.misses, res.evicted, res.bypass) == (hits, misses, evicted, bypass)
+        bp, bi, bt = brute.view(t)
+        assert (list(part), list(pidx), list(ts)) == (bp, bi, bt), f"t={t}"
+        # invariants
+        occ = part >= 0
+        assert len(set(zip(part[occ], pidx[occ]))) == occ.sum()           # no page twice
+        cached = set(int(p) for p in part[occ])
+        assert cached == {p for p in range(P) if resident[p] and npages[p] > 0}
+        assert set(res.hits) | set(res.misses) == set(sel)
+        for p in sel:
+            assert resident[p] or p in res.bypass
+        for p in set(int(x) for x in part[occ]):                           # whole or not at all
+            assert (part == p).sum() == npages[p]
+        if not res.bypass:                                                  # hits never evicted
+            assert not (set(e[1] for e in res.evicted) & set(sel))
+
+
+def test_exact_lru_while_step_counter_below_n():
+    # with t <= n-1 throughout, buckets are exact last-use steps: victims are always the
+    # least recently used generation(s)
+    S, n, P = 10, 64, 60
+    rng = np.random.default_rng(7)
+    part, pidx, ts = _fresh(S)
+    resident = np.zeros(P, dtype=np.int64)
+    npages = np.ones(P, dtype=np.int64)
+    last = {}
+    for t in range(40):
+        sel = sorted(set(int(x) for x in rng.integers(0, P, size=3)))
+        before = {int(p) for p in part[part >= 0]}
+        res = O.bucketed_lru_step(part, pidx, ts, resident, npages, sel, t, n)
+        for p in sel:
+            last[p] = t
+        gone = {e[1] for e in res.evicted}
+        kept = (before - gone) - set(sel)
+        if gone and kept:
+            assert max(last[p] for p in gone) < min(last[p] for p in kept)
+
+
+def test_big_cache_only_compulsory_misses():
+    S, n, P = 64, 8, 50
+    rng = np.random.default_rng(8)
+    part, pidx, ts = _fresh(S)
+    resident = np.zeros(P, dtype=np.int64)
+    npages = np.ones(P, dtype=np.int64)
+    seen = set()
+    for t in range(60):
+        sel = sorted(set(int(x) for x in rng.integers(0, P, size=6)))
+        res = O.bucketed_lru_step(part, pidx, ts, resident, npages, sel, t, n)
+        assert not res.evicted and not res.bypass
+        assert set(res.misses) == set(sel) - seen
+        seen |= set(sel)
+
+
+def test_single_bucket_evicts_every_non_hit_page():
+    S, P = 6, 30
+    part, pidx, ts = _fresh(S)
+    resident = np.zeros(P, dtype=np.int64)
+    npages = np.ones(P, dtype=np.int64)
+    O.bucketed_lru_step(part, pidx, ts, resident, npages, [0, 1, 2, 3, 4, 5], 0, 1)
+    res = O.bucketed_lru_step(part, pidx, ts, resident, npages, [1, 9], 1, 1)
+    assert res.hits == [1] and res.misses == [9]
+    assert sorted(e[1] for e in res.evicted) == [0, 2, 3, 4, 5]
+    assert sorted(int(p) for p in part[part >= 0]) == [1, 9]
+
+
+def test_overflow_bypasses_whole_partitions_and_keeps_hits():
+    S, n = 4, 4
+    part, pidx, ts = _fresh(S)
+    npages = np.array([2, 3, 1, 2, 1], dtype=np.int64)
+    resident = np.zeros(5, dtype=np.int64)
+    r0 = O.bucketed_lru_step(part, pidx, ts, resident, npages, [0], 0, n)
+    assert r0.misses == [0] and list(part) == [0, 0, -1, -1]
+    # 0 hits (2 pages pinned); 1 (3 pages) cannot fit in the 2 other slots -> bypassed whole;
+    # 2 (1 page) still fits; 3 (2 pages) no longer fits; 4 (1 page) does
+    r1 = O.bucketed_lru_step(part, pidx, ts, resident, npages, [0, 1, 2, 3, 4], 1, n)
+    assert r1.hits == [0] and r1.bypass == [1, 3]
+    assert list(part) == [0, 0, 2, 4] and list(resident) == [1, 0, 1, 0, 1]
