@@ -1,0 +1,260 @@
+// Select (Table 1: score(q, k_sums) -> topk; Section 4.1 "Select").
+//
+// k_score streams the summary segments of every set of the batch once (HBM bound: 512 B per
+// page for min/max summaries, 256 B per token key or centroid) and writes one fp32 score per
+// candidate.  The summation order is fixed so that the CPU oracle reproduces every score bit
+// for bit: a lane owns 8 consecutive channels (one 16-byte load) and adds them left to right;
+// the 16 lanes of a row are then combined by a butterfly (xor 1, 2, 4, 8), which is the
+// balanced tree over adjacent blocks; the group's query heads are added in ascending order.
+// Products of two bf16 values are exact in fp32, so fused or separate multiply-add agree.
+//
+// k_topk keeps, per set, the k best candidates (ties -> lower index) with a 4-pass radix
+// select on order-preserving keys followed by one ordered compaction, and emits them in
+// ascending index order.  For token-granular selection it also folds the chosen tokens into
+// their pages with a 16-bit token mask per page.
+#include "spin_dev.cuh"
+
+namespace spin {
+
+namespace {
+
+__device__ __forceinline__ void unpack8(uint4 raw, float *f) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+template <int G, bool MINMAX>
+__global__ void __launch_bounds__(256)
+k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
+  const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
+  const int set = set_index(c, bt.req[i_req], bt.layer, head);
+  if (blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *c.fetch_count = 0;   // new step, new miss queue
+  const SetState st = c.state[set];
+  const int n_cand = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
+  const int seg_entries = 1 << c.sum_shift;
+  const int e0 = blockIdx.x * seg_entries;
+  if (e0 >= n_cand) return;
+  const int seg = c.dir_sumseg[(size_t)set * c.dir_sum + blockIdx.x];
+  if (seg < 0) { if (threadIdx.x == 0) dev_error(c, 1u); return; }
+  const int lane16 = threadIdx.x & 15, grp = threadIdx.x >> 4;
+  // the two 16-lane rows of a warp may leave the loop at different times: each shuffles
+  // only among its own lanes
+  const uint32_t row_mask = 0xffffu << (threadIdx.x & 16);
+
+  float qf[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const uint4 raw = *reinterpret_cast<const uint4 *>(
+        q + ((size_t)i_req * c.Hq + head * G + g) * kHeadDim + lane16 * 8);
+    unpack8(raw, qf[g]);
+  }
+  const int n_here = min(seg_entries, n_cand - e0);
+  constexpr int kEntry = MINMAX ? 2 * kRowBytes : kRowBytes;
+  const uint8_t *base = c.summaries + ((size_t)seg << c.sum_shift) * kEntry + lane16 * 16;
+  float *out = c.scores + (size_t)b * c.max_cand + e0;
+
+#pragma unroll 4
+  for (int e = grp; e < n_here; e += 16) {
+    float a[8], mx[8];
+    unpack8(*reinterpret_cast<const uint4 *>(base + (size_t)e * kEntry), a);
+    if (MINMAX) unpack8(*reinterpret_cast<const uint4 *>(base + (size_t)e * kEntry + kRowBytes), mx);
+    float tot = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float s;
+      if (MINMAX) {
+        s = fmaxf(qf[g][0] * a[0], qf[g][0] * mx[0]);
+#pragma unroll
+        for (int i = 1; i < 8; ++i) s = s + fmaxf(qf[g][i] * a[i], qf[g][i] * mx[i]);
+      } else {
+        s = qf[g][0] * a[0];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) s = s + qf[g][i] * a[i];
+      }
+      s = s + __shfl_xor_sync(row_mask, s, 1);
+      s = s + __shfl_xor_sync(row_mask, s, 2);
+      s = s + __shfl_xor_sync(row_mask, s, 4);
+      s = s + __shfl_xor_sync(row_mask, s, 8);
+      tot = g == 0 ? s : tot + s;
+    }
+    if (lane16 == 0) out[e] = tot + 0.0f;       // -0.0 -> +0.0
+  }
+}
+
+__device__ __forceinline__ uint32_t order_key(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+constexpr int kTopkThreads = 512;
+
+// Exclusive prefix of v over the block (thread order) and the block total.
+__device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t *wsum, uint32_t *total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    uint32_t x = lane < kTopkThreads / 32 ? wsum[lane] : 0, xi = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t t = __shfl_up_sync(0xffffffffu, xi, o);
+      if (lane >= o) xi += t;
+    }
+    wsum[lane] = xi - x;                         // exclusive warp offsets
+    if (lane == 31) wsum[32] = xi;               // total
+  }
+  __syncthreads();
+  const uint32_t res = wsum[w] + inc - v;
+  *total = wsum[32];
+  __syncthreads();                               // wsum is reused by the next call
+  return res;
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+k_topk(DevCtx c, Batch bt) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t wsum[33];
+  __shared__ uint32_t sh_prefix, sh_remaining;
+  const int b = blockIdx.x, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
+  const int set = set_index(c, bt.req[i_req], bt.layer, head);
+  const SetState st = c.state[set];
+  const int n = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
+  const int k = min(c.topk, n);
+  const float *scores = c.scores + (size_t)b * c.max_cand;
+  int32_t *sel = c.sel_ids + (size_t)b * c.max_sel;
+
+  if (tid == 0) {
+    c.n_sel[b] = k;
+    atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
+  }
+  if (k == n) {
+    for (int i = tid; i < n; i += kTopkThreads) sel[i] = i;
+  } else {
+    // ---- radix select: key of the k-th best candidate --------------------------------
+    uint32_t prefix = 0, mask = 0, remaining = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      for (int i = tid; i < n; i += kTopkThreads) {
+        const uint32_t key = order_key(scores[i]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid < 32) {
+        // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the
+        // top reaches `remaining`
+        uint32_t loc[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { loc[j] = hist[255 - 8 * tid - j]; sum += loc[j]; }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += t;
+        }
+        const uint32_t before = inc - sum;
+        if (before < remaining && inc >= remaining) {
+          uint32_t cum = before;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (cum < remaining && cum + loc[j] >= remaining) {
+              sh_prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
+              sh_remaining = remaining - cum;
+            }
+            cum += loc[j];
+          }
+        }
+      }
+      __syncthreads();
+      prefix = sh_prefix;
+      remaining = sh_remaining;
+      mask |= 255u << shift;
+    }
+    const uint32_t thr = prefix, need_eq = remaining;
+    // ---- ordered compaction: everything above thr, plus the first need_eq equal to it --
+    uint32_t run_gt = 0, run_eq = 0;
+    for (int base = 0; base < n; base += kTopkThreads) {
+      const int i = base + tid;
+      uint32_t gt = 0, eq = 0;
+      if (i < n) {
+        const uint32_t key = order_key(scores[i]);
+        gt = key > thr;
+        eq = key == thr;
+      }
+      uint32_t total;
+      const uint32_t ex = block_scan(gt | (eq << 16), wsum, &total);
+      const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
+      if (gt || (eq && eq_before < need_eq))
+        sel[gt_before + min(eq_before, need_eq)] = i;
+      run_gt += total & 0xffffu;
+      run_eq += total >> 16;
+    }
+  }
+  __syncthreads();
+
+  // ---- candidates -> partitions of the cache manager -------------------------------------
+  int32_t *parts = c.parts + (size_t)b * c.max_parts;
+  if (c.kind != kKindToken) {
+    for (int i = tid; i < k; i += kTopkThreads) parts[i] = sel[i];
+    if (tid == 0) c.n_parts[b] = k;
+    return;
+  }
+  uint32_t *pmask = c.part_mask + (size_t)b * c.max_parts;
+  for (int i = tid; i < k; i += kTopkThreads) pmask[i] = 0;
+  __syncthreads();
+  uint32_t run = 0;
+  for (int base = 0; base < k; base += kTopkThreads) {
+    const int i = base + tid;
+    uint32_t first = 0;
+    int tok = 0;
+    if (i < k) {
+      tok = sel[i];
+      first = (i == 0) || ((sel[i - 1] >> 4) != (tok >> 4));
+    }
+    uint32_t total;
+    const uint32_t ex = block_scan(first, wsum, &total);
+    if (i < k) {
+      const uint32_t rank = run + ex + first - 1;
+      if (first) parts[rank] = tok >> 4;
+      atomicOr(&pmask[rank], 1u << (tok & 15));
+    }
+    run += total;
+  }
+  if (tid == 0) c.n_parts[b] = (int)run;
+}
+
+template <int G>
+void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, dim3 grid, cudaStream_t st) {
+  if (c.kind == kKindPage) k_score<G, true><<<grid, 256, 0, st>>>(c, b, q);
+  else k_score<G, false><<<grid, 256, 0, st>>>(c, b, q);
+}
+
+}  // namespace
+
+int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int max_cand,
+                  cudaStream_t st) {
+  const int n_sets = b.n_req * c.Hkv;
+  int segs = (max_cand + (1 << c.sum_shift) - 1) >> c.sum_shift;
+  if (segs < 1) segs = 1;                         // the first block also resets the miss queue
+  dim3 grid(segs, n_sets);
+  switch (c.G) {
+    case 1: launch_score_g<1>(c, b, q, grid, st); break;
+    case 2: launch_score_g<2>(c, b, q, grid, st); break;
+    case 4: launch_score_g<4>(c, b, q, grid, st); break;
+    default: launch_score_g<8>(c, b, q, grid, st); break;
+  }
+  k_topk<<<n_sets, kTopkThreads, 0, st>>>(c, b);
+  return 2;
+}
+
+}  // namespace spin

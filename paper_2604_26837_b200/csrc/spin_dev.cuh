@@ -1,0 +1,166 @@
+// Device-side data layout shared by the kernels and the host runtime.
+//
+// A "set" is one (request, layer, kv head).  Everything a set owns in HBM is reached from
+// its SetState and its five directories (two-level indexing, Section 5.4): a directory entry
+// names a fixed-size second-level segment in a shared pool; segments are mapped on demand by
+// the host runtime's bitmap allocators, so metadata grows with the mapped pages.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spin {
+
+constexpr int kHeadDim = 128;
+constexpr int kPageTokens = 16;
+constexpr int kRowBytes = kHeadDim * 2;                     // one K or V row, bf16
+constexpr int kHalfPageBytes = kPageTokens * kRowBytes;     // K half or V half: 4 KiB
+constexpr int kPageBytes = 2 * kHalfPageBytes;              // K rows then V rows: 8 KiB
+constexpr int kMaxBatch = 256;                              // requests per decode step
+constexpr int kMaxBuckets = 64;
+
+enum : int { kKindPage = 0, kKindToken = 1, kKindCluster = 2 };
+// sticky device error bits (same values as SPIN_DEV_ERR_* of the public header)
+constexpr unsigned kErrBounds = 1u, kErrPageList = 2u, kErrTimeout = 4u;
+constexpr int kChunkPages = 16;                             // pages per attention split
+
+// Per-set scalars (device resident, updated only by kernels).
+struct SetState {
+  int32_t n_tokens;       // tokens appended
+  int32_t n_partitions;   // indexed partitions = rows of the Meta-partition table
+  int32_t n_host_pages;   // entries of the set's CPU page table
+  int32_t tail_first;     // CPU-page-table index of the first tail page
+  int32_t tail_pages;     // tail pages (0/1 for the page-sized kinds)
+  int32_t tail_len;       // tokens in the newest tail page
+  int32_t step;           // decode steps done
+  int32_t slots;          // S: GPU page table entries
+};
+
+// Meta-partition table entry (GPU): token count + residency (Section 5.2).
+struct MetaEntry { int32_t tokens; int32_t resident; };
+// GPU page table entry: page-centric (slot -> owner) with the recency timestamp.
+struct GptEntry { int32_t partition; int32_t phys; int32_t page_idx; int32_t ts; };
+
+struct Counters {
+  unsigned long long set_steps, selected_partitions, selected_pages, tail_pages, hit_pages,
+      miss_pages, evicted_pages, bypass_pages, candidates_scored;
+  unsigned int error_bits;
+  unsigned int pad;
+};
+
+struct FetchItem { int32_t host_page; int32_t gpu_page; };
+
+// Everything a kernel needs to find its data; passed by value (fits the 4 KiB param space
+// together with a Batch).
+struct DevCtx {
+  // geometry
+  int32_t num_layers, Hq, Hkv, G, kind, topk, n_buckets, trace;
+  int32_t seg_shift;            // log2(entries per metadata segment)
+  int32_t sum_shift;            // log2(entries per summary segment)
+  int32_t sum_entry_bytes;      // 512 (min+max) or 256 (key / centroid)
+  int32_t dir_part, dir_slot, dir_page, dir_sum;   // directory lengths per set
+  int32_t max_sel, max_parts, max_pages, tail_cap; // scratch strides per batch set
+  int32_t max_cand;             // score stride per batch set
+  float sm_scale;
+  // pools
+  uint8_t *gpu_pages;           // HBM KV pages (cache slots + tails)
+  uint8_t *host_pages;          // pinned host KV pages (device-visible address)
+  uint8_t *summaries;           // summary segments (64 KiB each)
+  MetaEntry *meta_pool;         // GPU
+  GptEntry *gpt_pool;           // GPU
+  int32_t *off_pool;            // pinned host: Partition Offset table segments
+  int32_t *cpt_pool;            // pinned host: CPU page table segments
+  // per set
+  SetState *state;
+  int32_t *dir_meta, *dir_gpt, *dir_off, *dir_cpt, *dir_sumseg;
+  int32_t *tail_phys;           // [set][tail_cap] GPU pages of the tail
+  int32_t *evict_trace;         // [set][max_slots][2] (trace only)
+  int32_t max_slots;
+  // per-step scratch, indexed by batch set b = i_req * Hkv + head
+  float *scores;                // [b][max_cand]
+  int32_t *sel_ids;             // [b][max_sel]   chosen candidates, ascending
+  int32_t *n_sel;               // [b]
+  int32_t *parts;               // [b][max_parts] partitions for the cache manager
+  uint32_t *part_mask;          // [b][max_parts] token masks (token kind)
+  int32_t *part_state;          // [b][max_parts] 0 hit / 1 admitted / 2 bypassed
+  int32_t *n_parts;             // [b]
+  int32_t *page_src;            // [b][max_pages+tail_cap] >=0 GPU page, <0 ~host page
+  uint32_t *page_mask;          // [b][...]
+  int32_t *page_slot;           // [b][...] set-local slot / -1 bypass / -2 tail
+  int32_t *page_part;           // [b][...] owning partition (-1 tail)
+  int32_t *page_pidx;           // [b][...]
+  int32_t *n_pages;             // [b]
+  FetchItem *fetch_queue;       // misses of the whole batch
+  int32_t *fetch_count;
+  int32_t fetch_cap;
+  float *att_part;              // split-K partials [b][max_chunks][G][kHeadDim + 2]
+  int32_t max_chunks;
+  Counters *counters;
+};
+
+struct Batch {
+  int32_t n_req;
+  int32_t layer;
+  int32_t req[kMaxBatch];
+};
+
+__host__ __device__ inline int set_index(const DevCtx &c, int req, int layer, int head) {
+  return (req * c.num_layers + layer) * c.Hkv + head;
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void dev_error(const DevCtx &c, unsigned bits) {
+  atomicOr(&c.counters->error_bits, bits);
+}
+// Two-level lookups.  A negative directory entry means "not mapped": the caller gets nullptr
+// and records a bounds error instead of touching memory.
+__device__ __forceinline__ MetaEntry *meta_at(const DevCtx &c, int set, int p) {
+  int seg = c.dir_meta[(size_t)set * c.dir_part + (p >> c.seg_shift)];
+  return seg < 0 ? nullptr : c.meta_pool + ((size_t)seg << c.seg_shift) + (p & ((1 << c.seg_shift) - 1));
+}
+__device__ __forceinline__ GptEntry *gpt_at(const DevCtx &c, int set, int s) {
+  int seg = c.dir_gpt[(size_t)set * c.dir_slot + (s >> c.seg_shift)];
+  return seg < 0 ? nullptr : c.gpt_pool + ((size_t)seg << c.seg_shift) + (s & ((1 << c.seg_shift) - 1));
+}
+__device__ __forceinline__ int32_t *off_at(const DevCtx &c, int set, int p) {
+  int seg = c.dir_off[(size_t)set * c.dir_part + (p >> c.seg_shift)];
+  return seg < 0 ? nullptr : c.off_pool + ((size_t)seg << c.seg_shift) + (p & ((1 << c.seg_shift) - 1));
+}
+__device__ __forceinline__ int32_t *cpt_at(const DevCtx &c, int set, int i) {
+  int seg = c.dir_cpt[(size_t)set * c.dir_page + (i >> c.seg_shift)];
+  return seg < 0 ? nullptr : c.cpt_pool + ((size_t)seg << c.seg_shift) + (i & ((1 << c.seg_shift) - 1));
+}
+__device__ __forceinline__ uint8_t *summary_at(const DevCtx &c, int set, int e) {
+  int seg = c.dir_sumseg[(size_t)set * c.dir_sum + (e >> c.sum_shift)];
+  return seg < 0 ? nullptr
+                 : c.summaries + (((size_t)seg << c.sum_shift) + (e & ((1 << c.sum_shift) - 1))) *
+                                     (size_t)c.sum_entry_bytes;
+}
+__device__ __forceinline__ const uint8_t *page_ptr(const DevCtx &c, int src) {
+  return src >= 0 ? c.gpu_pages + (size_t)src * kPageBytes : c.host_pages + (size_t)(~src) * kPageBytes;
+}
+#endif
+
+// ---- kernel launchers (each returns the number of kernels it launched) -----------------
+struct AppendEdgeArgs {     // one (request) per entry; all its kv heads are processed
+  int32_t n_req, layer;
+  int32_t req[kMaxBatch];
+};
+int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
+                       const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,
+                       cudaStream_t st);
+int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bfloat16 *k,
+                       const __nv_bfloat16 *v, int n_new, cudaStream_t st);
+int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
+                           const __nv_bfloat16 *v, const int64_t *dest_row, int n_tokens,
+                           cudaStream_t st);
+int launch_copy_centroids(const DevCtx &c, int req, int layer, const __nv_bfloat16 *cen,
+                          int n_clusters, cudaStream_t st);
+int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int max_cand,
+                  cudaStream_t st);
+int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count);
+size_t cache_smem_bytes(const DevCtx &c);
+int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
+                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st);
+
+}  // namespace spin

@@ -1,0 +1,86 @@
+"""Synthetic driver: feeds a `workloads.Workload` through the library, the way a serving
+engine's attention layer would (prefill appends, then per decode step one appended token and
+one decode call per layer).  Marshalling and input generation only; it never computes any
+stage of the path itself and knows nothing about the CPU oracle.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import torch
+
+import workloads as W
+
+from . import binding as B
+
+
+def context_sizes(w: W.Workload):
+    ctx = [w.request_context(r) for r in range(w.batch)]
+    return ctx
+
+
+def make_spin(w: W.Workload, device="cuda:0", trace: bool = False, sm_scale: float = 0.0,
+              slots_per_set: Optional[int] = None, segment_entries: int = 0) -> "SpinRun":
+    return SpinRun(w, device, trace, sm_scale, slots_per_set, segment_entries)
+
+
+class SpinRun:
+    """A library context sized for one workload, plus the per-step call sequence."""
+
+    def __init__(self, w: W.Workload, device="cuda:0", trace=False, sm_scale=0.0,
+                 slots_per_set=None, segment_entries=0):
+        self.w = w
+        self.device = torch.device(device)
+        T = w.page_tokens
+        ctx = context_sizes(w)
+        sets_per_req = w.num_layers * w.num_kv_heads
+        self.slots = w.slots_per_set if slots_per_set is None else slots_per_set
+        cluster = w.partition_kind == W.PART_CLUSTER_CENTROID
+        pages_per_set = [(c + w.steps + T - 1) // T + 2 for c in ctx]
+        if cluster:
+            pages_per_set = [p + w.num_clusters for p in pages_per_set]
+        host_pages = sum(pages_per_set) * sets_per_req
+        cfg = B.make_config(
+            device=self.device.index or 0, num_layers=w.num_layers, num_q_heads=w.num_q_heads,
+            num_kv_heads=w.num_kv_heads, max_requests=w.batch,
+            max_context_tokens=max(ctx) + w.steps + T, partition_kind=w.partition_kind,
+            topk=w.topk, num_clusters=w.num_clusters if cluster else 0,
+            max_selected_pages=(w.topk * w.max_partition_pages if cluster else 0),
+            max_tail_tokens=(w.steps + T if cluster else 0), lru_buckets=w.lru_buckets,
+            segment_entries=segment_entries, sm_scale=sm_scale, trace=1 if trace else 0,
+            gpu_cache_pages=self.slots * sets_per_req * w.batch, host_pages=host_pages)
+        self.spin = B.Spin(cfg, self.device)
+        self.reqs: List[int] = [self.spin.request_open(self.slots) for _ in range(w.batch)]
+        self.ctx = ctx
+        self.step_no = 0
+
+    # -- inputs (synthetic, generated on the device) ------------------------------------
+    def gen_prefill(self, r: int, layer: int):
+        w = self.w
+        k, v = W.kv_tokens(w, r, layer, 0, self.ctx[r], self.device)
+        if w.partition_kind == W.PART_CLUSTER_CENTROID:
+            tp = W.cluster_assignment(w, r, layer, self.ctx[r], self.device).contiguous()
+            cen = W.centroids(w, r, layer, self.device).contiguous()
+            return k.contiguous(), v.contiguous(), tp, cen
+        return k.contiguous(), v.contiguous(), None, None
+
+    def gen_step_tokens(self, layer: int, step: int):
+        ks, vs = [], []
+        for r in range(self.w.batch):
+            k, v = W.kv_tokens(self.w, r, layer, self.ctx[r] + step, 1, self.device)
+            ks.append(k)
+            vs.append(v)
+        return torch.cat(ks).contiguous(), torch.cat(vs).contiguous()      # [B][Hkv][d]
+
+    # -- calls -----------------------------------------------------------------------------
+    def prefill(self, r: int, layer: int, k, v, tp=None, cen=None, stream=None):
+        self.spin.append_kv(self.reqs[r], layer, k, v, k.shape[0], tp, cen, stream)
+
+    def append(self, layer: int, k_new, v_new, stream=None):
+        self.spin.append_kv_batch(layer, self.reqs, k_new, v_new, stream)
+
+    def decode(self, layer: int, q, out, stream=None):
+        self.spin.decode_step(layer, self.reqs, q, out, stream)
+
+    def close(self):
+        self.spin.close()

@@ -1,0 +1,186 @@
+"""Parity of the CUDA library against the CPU oracle, step by step, through the C ABI.
+
+Integer results (selections, partitions, hit/miss/bypass classes, evictions, page lists,
+GPU page table contents, residency bits, counters) and fp32 scores are compared bit for bit;
+attention outputs within max-abs 2e-2 and mean-abs 2e-3 (bf16 K/V, fp32 accumulation).
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import spin_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+def _wl(kind, **kw):
+    base = dict(name="t", seed=77, batch=2, num_layers=2, num_q_heads=8, num_kv_heads=2,
+                head_dim=128, page_tokens=16, context=16 * 40 + 5, partition_kind=kind, topk=6,
+                slots_per_set=16, lru_buckets=4, steps=24, drift=0.25, kv_recipe="normal")
+    base.update(kw)
+    return W.Workload(**base)
+
+
+def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0):
+    from paper_2604_26837_b200.driver import SpinRun
+    dev = "cuda:0"
+    run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
+                  segment_entries=segment_entries)
+    S = run.slots
+    orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                                      w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
+    oreq = [orc.request_open(S) for _ in range(w.batch)]
+    for r in range(w.batch):
+        for l in range(w.num_layers):
+            k, v, tp, cen = run.gen_prefill(r, l)
+            run.prefill(r, l, k, v, tp, cen)
+            if tp is not None:
+                orc.append_kv(oreq[r], l, W.to_bits(k), W.to_bits(v), tp.cpu().numpy(), W.to_bits(cen))
+            else:
+                orc.append_kv(oreq[r], l, W.to_bits(k), W.to_bits(v))
+    qs = {(r, l): W.QueryStream(w, r, l, dev) for r in range(w.batch) for l in range(w.num_layers)}
+    out = torch.zeros(w.batch, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    cap_sel = w.topk
+    cap_pages = w.topk * max(1, w.max_partition_pages) + (w.steps + 16) // 16 + 2
+    worst_abs, worst_mean, rel_num, rel_den = 0.0, 0.0, 0.0, 0.0
+    for step in range(w.steps):
+        for l in range(w.num_layers):
+            kn, vn = run.gen_step_tokens(l, step)
+            run.append(l, kn, vn)
+            kb, vb = W.to_bits(kn), W.to_bits(vn)
+            for r in range(w.batch):
+                orc.append_kv(oreq[r], l, kb[r:r + 1], vb[r:r + 1])
+            q = torch.stack([qs[(r, l)].next() for r in range(w.batch)]).contiguous()
+            run.decode(l, q, out)
+            ref = orc.decode_step(l, oreq, W.to_bits(q))
+            torch.cuda.synchronize()
+            got = out.float().cpu().numpy().astype(np.float64)
+            err = np.abs(got - ref)
+            worst_abs, worst_mean = max(worst_abs, err.max()), max(worst_mean, err.mean())
+            rel_num += float((err ** 2).sum())
+            rel_den += float((ref ** 2).sum())
+            for r in range(w.batch):
+                for h in range(w.num_kv_heads):
+                    tr = orc.last_trace[(oreq[r], l, h)]
+                    st = orc.set(oreq[r], l, h)
+                    ncand = len(tr.scores)
+                    d = run.spin.debug_dump(run.reqs[r], l, h, cap_sel, cap_pages, S,
+                                            st.n_partitions() + 1, ncand + 1)
+                    where = f"step {step} layer {l} req {r} head {h}"
+                    assert np.array_equal(d["scores"].view(np.uint32), tr.scores.view(np.uint32)), where
+                    assert list(d["selected"]) == list(tr.selected), where
+                    assert list(d["parts"]) == list(tr.partitions), where
+                    cls = {0: [], 1: [], 2: []}
+                    for p, s_ in zip(d["parts"], d["part_state"]):
+                        cls[int(s_)].append(int(p))
+                    assert cls[0] == tr.hits, where
+                    assert sorted(cls[1] + cls[2]) == tr.misses and cls[2] == tr.bypass, where
+                    pages = list(zip(d["page_partition"].tolist(), d["page_idx"].tolist(),
+                                     d["page_mask"].tolist(), d["page_slot"].tolist()))
+                    assert pages == tr.pages, where
+                    assert list(d["slot_partition"]) == list(tr.slot_part), where
+                    assert list(d["slot_page_idx"]) == list(tr.slot_pidx), where
+                    assert list(d["slot_ts"]) == list(tr.slot_ts), where
+                    ev = [(s_, int(p), int(i)) for s_, (p, i) in
+                          enumerate(zip(d["slot_evicted_partition"], d["slot_evicted_page_idx"])) if p >= 0]
+                    assert ev == tr.evicted, where
+                    assert list(d["part_resident"]) == list(tr.resident), where
+                    assert list(d["part_tokens"]) == st.part_tokens, where
+                    assert d["n_tokens"] == st.n_tokens and d["step"] == st.t, where
+                    if check_bytes and (step % 5 == 0 or step == w.steps - 1):
+                        # Retrieve step 4: every cached slot holds exactly the host page's bytes
+                        for s_ in np.nonzero(tr.slot_part >= 0)[0][:: max(1, S // 6)]:
+                            p, i = int(tr.slot_part[s_]), int(tr.slot_pidx[s_])
+                            gpu = run.spin.debug_read_page(run.reqs[r], l, h, slot=int(s_))
+                            host = run.spin.debug_read_page(run.reqs[r], l, h, partition=p, page_idx=i)
+                            page = st.cpu_page_table[st.part_offset[p] + i]
+                            valid = min(16, st.part_tokens[p] - 16 * i)
+                            assert np.array_equal(gpu, host), where
+                            assert np.array_equal(gpu[0][:valid], st.page_k[page][:valid]), where
+                            assert np.array_equal(gpu[1][:valid], st.page_v[page][:valid]), where
+    stats = run.spin.stats()
+    assert stats["error_bits"] == 0
+    for key in ("selected_partitions", "selected_pages", "tail_pages", "hit_pages", "miss_pages",
+                "evicted_pages", "bypass_pages"):
+        assert stats[key] == orc.counters[key], key
+    assert stats["set_steps"] == orc.counters["steps"]
+    assert stats["pcie_bytes"] == orc.step_bytes()["pcie"]
+    assert worst_abs <= MAX_ABS * tol_scale and worst_mean <= MEAN_ABS * tol_scale, (worst_abs, worst_mean)
+    run.close()
+    return dict(max_abs=worst_abs, mean_abs=worst_mean, rel_l2=math.sqrt(rel_num / max(rel_den, 1e-30)),
+                stats=stats)
+
+
+@pytest.mark.parametrize("sm_scale", [0.0, 1.0])
+def test_page_minmax_small(sm_scale):
+    r = run_parity(_wl(W.PART_PAGE_MINMAX), sm_scale=sm_scale)
+    assert r["rel_l2"] < 2e-2
+
+
+def test_page_minmax_outlier_keys_gqa4_many_buckets():
+    w = _wl(W.PART_PAGE_MINMAX, num_q_heads=8, num_kv_heads=2, kv_recipe="outlier", outlier_channels=4,
+            lru_buckets=64, steps=80, topk=8, slots_per_set=24, drift=0.1, context=16 * 70 + 15)
+    run_parity(w, sm_scale=0.0)
+
+
+def test_page_minmax_step_counter_passes_bucket_count_and_segments_are_crossed():
+    # 16-entry segments: tables span several second-level segments; n=3 buckets: demotion active
+    w = _wl(W.PART_PAGE_MINMAX, lru_buckets=3, steps=40, topk=12, slots_per_set=40, context=16 * 100 + 1,
+            batch=3, num_layers=1)
+    run_parity(w, segment_entries=16)
+
+
+def test_page_minmax_overflowing_budget_bypasses():
+    w = _wl(W.PART_PAGE_MINMAX, topk=10, slots_per_set=7, steps=12)
+    r = run_parity(w)
+    assert r["stats"]["bypass_pages"] > 0
+
+
+def test_page_minmax_single_bucket_and_gqa1_gqa8():
+    run_parity(_wl(W.PART_PAGE_MINMAX, lru_buckets=1, steps=10, num_q_heads=2, num_kv_heads=2))
+    run_parity(_wl(W.PART_PAGE_MINMAX, steps=6, num_q_heads=16, num_kv_heads=2))
+
+
+def test_empty_and_short_contexts():
+    # fewer candidates than top-k, and a context shorter than one page (no candidate at all)
+    run_parity(_wl(W.PART_PAGE_MINMAX, context=16 * 3 + 2, topk=8, steps=20))
+    run_parity(_wl(W.PART_PAGE_MINMAX, context=3, topk=4, steps=30, batch=1, num_layers=1))
+
+
+@pytest.mark.parametrize("sm_scale", [0.0, 1.0])
+def test_token_dot(sm_scale):
+    w = _wl(W.PART_TOKEN_DOT, topk=40, slots_per_set=30, kv_recipe="page_centre", steps=20,
+            num_q_heads=4, num_kv_heads=1, context=16 * 60 + 9)
+    run_parity(w, sm_scale=sm_scale)
+
+
+def test_token_dot_overflow_and_ties():
+    # i.i.d. keys spread the chosen tokens over more pages than the budget holds
+    w = _wl(W.PART_TOKEN_DOT, topk=64, slots_per_set=20, steps=10, context=16 * 50)
+    r = run_parity(w)
+    assert r["stats"]["bypass_pages"] > 0
+
+
+@pytest.mark.parametrize("sm_scale", [0.0, 1.0])
+def test_cluster_centroid(sm_scale):
+    w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=37, topk=5, slots_per_set=30,
+            context=16 * 50 + 3, steps=40, max_partition_pages=8, lru_buckets=8)
+    run_parity(w, sm_scale=sm_scale)
+
+
+def test_cluster_centroid_tight_budget_with_empty_clusters():
+    # 300 clusters over 400 tokens: many empty and single-token clusters; budget overflows
+    w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=300, topk=20, slots_per_set=12,
+            context=400, steps=20, max_partition_pages=4, batch=1)
+    run_parity(w)
+
+
+def test_tiny_configuration_full_size():
+    # the first benchmark configuration as stated: 4096-token context, top-16, 64 slots, 8 buckets
+    r = run_parity(W.CONFIGS["c1"], check_bytes=False)
+    assert r["stats"]["set_steps"] == 32 and r["stats"]["evicted_pages"] > 0
