@@ -102,7 +102,8 @@ int compute_geometry(const spin_config &cfg, Geometry &g, std::string &err) {
   g.tail_cap = cluster ? (int32_t)std::max<int64_t>(1, (cfg.max_tail_tokens + kPageTokens - 1) / kPageTokens) : 1;
   g.pages_per_set = cluster ? ctx_pages + cfg.num_clusters + g.tail_cap + 1 : ctx_pages + 1;
   g.parts_per_set = cluster ? cfg.num_clusters : g.pages_per_set;
-  g.max_slots = std::max<int64_t>(1, std::min<int64_t>(g.pages_per_set, cfg.gpu_cache_pages));
+  // a budget beyond the set's own page count is never useful, but small sets may ask for it
+  g.max_slots = std::max<int64_t>(1, std::min<int64_t>(std::max<int64_t>(g.pages_per_set, 256), cfg.gpu_cache_pages));
   g.sum_entries = cfg.partition_kind == SPIN_PART_PAGE_MINMAX ? 128 : 256;
   g.sum_shift = ilog2(g.sum_entries);
   g.sum_entry_bytes = cfg.partition_kind == SPIN_PART_PAGE_MINMAX ? 2 * kRowBytes : kRowBytes;
