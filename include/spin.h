@@ -196,6 +196,21 @@ SPIN_API int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_i
 /* Counters and sticky device error bits.  Synchronises the device. */
 SPIN_API int spin_stats(spin_ctx *ctx, spin_stats_t *out);
 
+/* Per-kernel timing (tracing aid, off by default).  spin_profile(ctx, 1) synchronises, clears
+ * the record and makes every later append / decode call record a CUDA event after each kernel
+ * it launches on the caller's stream (up to 32768 marks, then recording stops);
+ * spin_profile_read() synchronises and returns, per kernel, its launches and the summed
+ * event-to-event time.  Kernel order: 0 append, 1 score, 2 top-k, 3 cache manager (LRU +
+ * translation), 4 page fetch, 5 attention splits, 6 attention merge. */
+typedef struct spin_profile_t {
+  uint32_t struct_size;
+  uint32_t n_kernels;
+  uint64_t launches[8];
+  double ms[8];
+} spin_profile_t;
+SPIN_API int spin_profile(spin_ctx *ctx, int32_t enable);
+SPIN_API int spin_profile_read(spin_ctx *ctx, spin_profile_t *out);
+
 /* Logical state of one set (see spin_dump_t).  Synchronises the device. */
 SPIN_API int spin_debug_dump(spin_ctx *ctx, int32_t req, int32_t layer, int32_t kv_head, spin_dump_t *d);
 

@@ -23,8 +23,9 @@ PAGE_BYTES = 8192
 
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open",
            "spin_request_close", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
-           "spin_stats", "spin_debug_dump", "spin_debug_read_page", "spin_last_error",
-           "spin_version"]
+           "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
+           "spin_debug_read_page", "spin_last_error", "spin_version"]
+KERNEL_NAMES = ["append", "score", "topk", "cache", "fetch", "attn_split", "attn_merge"]
 
 
 class SpinError(RuntimeError):
@@ -52,6 +53,11 @@ class spin_stats_t(C.Structure):
                                   "candidates_scored", "pcie_bytes", "hbm_bytes", "kernel_launches",
                                   "gpu_meta_bytes", "host_meta_bytes", "summary_bytes",
                                   "gpu_pages_in_use", "host_pages_in_use")]
+
+
+class spin_profile_t(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("n_kernels", C.c_uint32),
+                ("launches", C.c_uint64 * 8), ("ms", C.c_double * 8)]
 
 
 _I32P = C.POINTER(C.c_int32)
@@ -97,6 +103,8 @@ def load() -> C.CDLL:
     lib.spin_append_kv_batch.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
     lib.spin_decode_step.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
     lib.spin_stats.argtypes = [vp, C.POINTER(spin_stats_t)]
+    lib.spin_profile.argtypes = [vp, i32]
+    lib.spin_profile_read.argtypes = [vp, C.POINTER(spin_profile_t)]
     lib.spin_debug_dump.argtypes = [vp, i32, i32, i32, C.POINTER(spin_dump_t)]
     lib.spin_debug_read_page.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
     lib.spin_last_error.argtypes = [vp]
@@ -213,6 +221,16 @@ class Spin:
         s.struct_size = C.sizeof(spin_stats_t)
         self._ck(self.lib.spin_stats(self.h, C.byref(s)))
         return {n: getattr(s, n) for n, _ in spin_stats_t._fields_ if n != "struct_size"}
+
+    def profile(self, enable: bool):
+        self._ck(self.lib.spin_profile(self.h, 1 if enable else 0))
+
+    def profile_read(self) -> dict:
+        """Per kernel: (launches, total ms) between CUDA events recorded on the stream."""
+        p = spin_profile_t()
+        p.struct_size = C.sizeof(spin_profile_t)
+        self._ck(self.lib.spin_profile_read(self.h, C.byref(p)))
+        return {KERNEL_NAMES[i]: (int(p.launches[i]), float(p.ms[i])) for i in range(p.n_kernels)}
 
     def debug_dump(self, req: int, layer: int, kv_head: int, cap_selected: int, cap_pages: int,
                    cap_slots: int, cap_partitions: int, cap_scores: int = 0) -> dict:

@@ -168,6 +168,7 @@ struct spin_ctx {
   int sm_count = 148;
   uint64_t launches = 0;
   size_t dir_bytes_in_use = 0;
+  Prof prof;
 };
 
 namespace {
@@ -355,12 +356,12 @@ int append_paged_device(spin_ctx *ctx, int req, int layer, const __nv_bfloat16 *
   if (rc) return rc;
   const int64_t j_end = (n0 + n - 1) / kPageTokens;
   // pages strictly between the old tail page and the newest page: complete, all rows new
-  ctx->launches += launch_append_bulk(ctx->d, req, layer, k, v, (int)(j0 + 1), (int)(j_end - (j0 + 1)), (int)n0, st);
+  ctx->launches += launch_append_bulk(ctx->d, req, layer, k, v, (int)(j0 + 1), (int)(j_end - (j0 + 1)), (int)n0, st, &ctx->prof);
   AppendEdgeArgs a{};
   a.n_req = 1;
   a.layer = layer;
   a.req[0] = req;
-  ctx->launches += launch_append_edge(ctx->d, a, k, v, (int)n, st);
+  ctx->launches += launch_append_edge(ctx->d, a, k, v, (int)n, st, &ctx->prof);
   return SPIN_OK;
 }
 
@@ -497,8 +498,47 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
 
 }  // namespace
 
+namespace spin {
+void Prof::mark(cudaStream_t st, int kernel) {
+  if (!ev) {
+    ev = new cudaEvent_t[kMaxMarks];
+    id = new int[kMaxMarks];
+    for (size_t i = 0; i < kMaxMarks; ++i) cudaEventCreate(&ev[i]);
+  }
+  if (used >= kMaxMarks) return;
+  cudaEventRecord(ev[used], st);
+  id[used++] = kernel;
+}
+}  // namespace spin
+
 // ---------------------------------------------------------------------------------------
 extern "C" {
+
+int spin_profile(spin_ctx *ctx, int32_t enable) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  CK(cudaDeviceSynchronize());
+  ctx->prof.on = enable != 0;
+  ctx->prof.used = 0;
+  return SPIN_OK;
+}
+
+int spin_profile_read(spin_ctx *ctx, spin_profile_t *out) {
+  if (!ctx || !out) return SPIN_ERR_INVALID;
+  if (out->struct_size != sizeof(spin_profile_t)) return fail(ctx, SPIN_ERR_INVALID, "spin_profile_t.struct_size mismatch");
+  CK(cudaDeviceSynchronize());
+  out->n_kernels = kProfKernels;
+  for (int i = 0; i < 8; ++i) { out->launches[i] = 0; out->ms[i] = 0.0; }
+  const Prof &p = ctx->prof;
+  for (size_t i = 1; i < p.used; ++i) {
+    if (p.id[i] < 0) continue;
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, p.ev[i - 1], p.ev[i]));
+    out->launches[p.id[i]] += 1;
+    out->ms[p.id[i]] += ms;
+  }
+  return SPIN_OK;
+}
+
 
 const char *spin_version(void) { return "spin-b200 0.1"; }
 
@@ -605,6 +645,11 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
 int spin_destroy(spin_ctx *ctx) {
   if (!ctx) return SPIN_ERR_INVALID;
   cudaDeviceSynchronize();
+  if (ctx->prof.ev) {
+    for (size_t i = 0; i < Prof::kMaxMarks; ++i) cudaEventDestroy(ctx->prof.ev[i]);
+    delete[] ctx->prof.ev;
+    delete[] ctx->prof.id;
+  }
   if (ctx->host_base) cudaFreeHost(ctx->host_base);
   delete ctx;
   return SPIN_OK;
@@ -734,7 +779,7 @@ int spin_append_kv(spin_ctx *ctx, int32_t req, int32_t layer, const void *k, con
       if (rc) return rc;
       AppendEdgeArgs a{};
       a.n_req = 1; a.layer = layer; a.req[0] = req;
-      ctx->launches += launch_append_edge(ctx->d, a, kk, vv, (int)m, st);
+      ctx->launches += launch_append_edge(ctx->d, a, kk, vv, (int)m, st, &ctx->prof);
     } else {
       rc = append_paged_device(ctx, req, layer, kk, vv, m, st);
       if (rc) return rc;
@@ -774,7 +819,8 @@ int spin_append_kv_batch(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, i
     kk = ctx->stage_k;
     vv = ctx->stage_v;
   }
-  ctx->launches += launch_append_edge(ctx->d, a, kk, vv, 1, st);
+  prof_mark(&ctx->prof, st, -1);
+  ctx->launches += launch_append_edge(ctx->d, a, kk, vv, 1, st, &ctx->prof);
   CK(cudaGetLastError());
   return SPIN_OK;
 }
@@ -808,9 +854,10 @@ int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   const bool q_dev = is_device_ptr(q), out_dev = is_device_ptr(out);
   if (!q_dev) { CK(cudaMemcpyAsync(ctx->stage_q, q, qbytes, cudaMemcpyHostToDevice, st)); qd = ctx->stage_q; }
   if (!out_dev) od = ctx->stage_out;
-  ctx->launches += launch_select(ctx->d, b, qd, (int)max_cand, st);
-  ctx->launches += launch_cache(ctx->d, b, st, ctx->sm_count);
-  ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, st);
+  prof_mark(&ctx->prof, st, -1);
+  ctx->launches += launch_select(ctx->d, b, qd, (int)max_cand, st, &ctx->prof);
+  ctx->launches += launch_cache(ctx->d, b, st, ctx->sm_count, &ctx->prof);
+  ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, st, &ctx->prof);
   if (!out_dev) CK(cudaMemcpyAsync(out, ctx->stage_out, qbytes, cudaMemcpyDeviceToHost, st));
   CK(cudaGetLastError());
   return SPIN_OK;

@@ -206,15 +206,17 @@ k_copy_centroids(DevCtx c, int req, int layer, const __nv_bfloat16 *__restrict__
 
 int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,
-                       cudaStream_t st) {
+                       cudaStream_t st, Prof *prof) {
   if (n_pages <= 0) return 0;
   k_append_bulk<<<dim3(n_pages, c.Hkv), 256, 0, st>>>(c, req, layer, k, v, first_page, first_token_of_call);
+  prof_mark(prof, st, kProfAppend);
   return 1;
 }
 
 int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bfloat16 *k,
-                       const __nv_bfloat16 *v, int n_new, cudaStream_t st) {
+                       const __nv_bfloat16 *v, int n_new, cudaStream_t st, Prof *prof) {
   k_append_edge<<<dim3(c.Hkv, a.n_req), 256, 0, st>>>(c, a, k, v, n_new);
+  prof_mark(prof, st, kProfAppend);
   return 1;
 }
 

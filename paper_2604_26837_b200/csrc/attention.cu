@@ -154,7 +154,7 @@ k_attn_merge(DevCtx c, Batch bt, __nv_bfloat16 *__restrict__ out) {
 }  // namespace
 
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
-                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st) {
+                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st, Prof *prof) {
   const int n_sets = b.n_req * c.Hkv;
   int chunks = (max_pages_hint + kChunkPages - 1) / kChunkPages;
   if (chunks < 1) chunks = 1;
@@ -166,7 +166,9 @@ int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
     case 4: k_attn_split<4><<<grid, kAttnWarps * 32, 0, st>>>(c, b, q); break;
     default: k_attn_split<8><<<grid, kAttnWarps * 32, 0, st>>>(c, b, q); break;
   }
+  prof_mark(prof, st, kProfAttnSplit);
   k_attn_merge<<<dim3(c.G, n_sets), kHeadDim, 0, st>>>(c, b, out);
+  prof_mark(prof, st, kProfAttnMerge);
   return 2;
 }
 

@@ -330,7 +330,7 @@ size_t cache_smem_bytes(const DevCtx &c) {
   return (size_t)(5 * c.max_parts + 1 + c.max_pages) * 4 + (size_t)((c.max_slots + 31) / 32) * 4 + 16;
 }
 
-int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count) {
+int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count, Prof *prof) {
   static size_t configured = 0;
   const size_t smem = cache_smem_bytes(c);
   if (smem > configured) {
@@ -338,7 +338,9 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count)
     configured = smem;
   }
   k_cache<<<b.n_req * c.Hkv, kCacheThreads, smem, st>>>(c, b);
+  prof_mark(prof, st, kProfCache);
   k_fetch<<<sm_count * 4, 256, 0, st>>>(c);
+  prof_mark(prof, st, kProfFetch);
   return 2;
 }
 

@@ -242,7 +242,7 @@ void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, dim
 }  // namespace
 
 int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int max_cand,
-                  cudaStream_t st) {
+                  cudaStream_t st, Prof *prof) {
   const int n_sets = b.n_req * c.Hkv;
   int segs = (max_cand + (1 << c.sum_shift) - 1) >> c.sum_shift;
   if (segs < 1) segs = 1;                         // the first block also resets the miss queue
@@ -253,7 +253,9 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int m
     case 4: launch_score_g<4>(c, b, q, grid, st); break;
     default: launch_score_g<8>(c, b, q, grid, st); break;
   }
+  prof_mark(prof, st, kProfScore);
   k_topk<<<n_sets, kTopkThreads, 0, st>>>(c, b);
+  prof_mark(prof, st, kProfTopk);
   return 2;
 }
 

@@ -141,6 +141,19 @@ __device__ __forceinline__ const uint8_t *page_ptr(const DevCtx &c, int src) {
 }
 #endif
 
+// Optional per-kernel timing: an event after every launch; durations are read afterwards.
+enum : int { kProfAppend = 0, kProfScore, kProfTopk, kProfCache, kProfFetch, kProfAttnSplit,
+             kProfAttnMerge, kProfKernels };
+struct Prof {
+  bool on = false;
+  static constexpr size_t kMaxMarks = 1 << 15;
+  cudaEvent_t *ev = nullptr;       // kMaxMarks events, created on first use
+  int *id = nullptr;               // kernel that ended at mark i (-1 = start of a sequence)
+  size_t used = 0;
+  void mark(cudaStream_t st, int kernel);
+};
+inline void prof_mark(Prof *p, cudaStream_t st, int kernel) { if (p && p->on) p->mark(st, kernel); }
+
 // ---- kernel launchers (each returns the number of kernels it launched) -----------------
 struct AppendEdgeArgs {     // one (request) per entry; all its kv heads are processed
   int32_t n_req, layer;
@@ -148,19 +161,19 @@ struct AppendEdgeArgs {     // one (request) per entry; all its kv heads are pro
 };
 int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,
-                       cudaStream_t st);
+                       cudaStream_t st, Prof *prof);
 int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bfloat16 *k,
-                       const __nv_bfloat16 *v, int n_new, cudaStream_t st);
+                       const __nv_bfloat16 *v, int n_new, cudaStream_t st, Prof *prof);
 int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                            const __nv_bfloat16 *v, const int64_t *dest_row, int n_tokens,
                            cudaStream_t st);
 int launch_copy_centroids(const DevCtx &c, int req, int layer, const __nv_bfloat16 *cen,
                           int n_clusters, cudaStream_t st);
 int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int max_cand,
-                  cudaStream_t st);
-int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count);
+                  cudaStream_t st, Prof *prof);
+int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count, Prof *prof);
 size_t cache_smem_bytes(const DevCtx &c);
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
-                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st);
+                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st, Prof *prof);
 
 }  // namespace spin

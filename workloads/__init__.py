@@ -190,6 +190,21 @@ def outlier_channels(w: Workload, layer: int, head: int) -> List[int]:
     return sorted(chans)
 
 
+_SCALE_CACHE: dict = {}
+
+
+def _outlier_scale(w: Workload, layer: int, device) -> torch.Tensor:
+    """fp32 [num_kv_heads][head_dim]: outlier_scale on the outlier channels, 1 elsewhere."""
+    key = (w.seed, w.num_kv_heads, w.head_dim, w.outlier_channels, w.outlier_scale, layer, str(device))
+    if key not in _SCALE_CACHE:
+        s = torch.ones(w.num_kv_heads, w.head_dim, dtype=torch.float32)
+        for h in range(w.num_kv_heads):
+            for c in outlier_channels(w, layer, h):
+                s[h, c] = w.outlier_scale
+        _SCALE_CACHE[key] = s.to(device)
+    return _SCALE_CACHE[key]
+
+
 def centroids(w: Workload, req: int, layer: int, device="cpu") -> torch.Tensor:
     """Mixture centroids of one request: bf16 [num_clusters][num_kv_heads][head_dim]."""
     n = w.num_clusters * w.num_kv_heads * w.head_dim
@@ -221,10 +236,7 @@ def kv_tokens(w: Workload, req: int, layer: int, first_token: int, n_tokens: int
     if w.kv_recipe == "normal":
         k = zk
     elif w.kv_recipe == "outlier":
-        k = zk.clone()
-        for h in range(H):
-            for c in outlier_channels(w, layer, h):
-                k[:, h, c] *= w.outlier_scale
+        k = zk * _outlier_scale(w, layer, device)
     elif w.kv_recipe == "page_centre":
         T = w.page_tokens
         p0 = first_token // T
