@@ -220,6 +220,32 @@ SPIN_API int spin_debug_dump(spin_ctx *ctx, int32_t req, int32_t layer, int32_t 
 SPIN_API int spin_debug_read_page(spin_ctx *ctx, int32_t req, int32_t layer, int32_t kv_head,
                          int32_t slot, int32_t partition, int32_t page_idx, void *out);
 
+/* Paged attention that allocates nothing (the paper has no counterpart: it is an addition for
+ * callers that cannot allocate GPU memory -- code that runs inside another component's fixed
+ * memory budget, or on a path where touching an allocator is forbidden -- and therefore
+ * cannot create a context, whose scratch comes out of a caller-allocated pool).
+ * It runs the same split-K attention + log-sum-exp merge as spin_decode_step's last stage over
+ * page lists the caller supplies; the split-K partials go to an 8 MiB array built into the
+ * library image (every GPU that loads the library holds it until the process exits).
+ *   q, out      bf16 [n_sets][group][128], device pointers (out is written)
+ *   page_pool   device pointer to 8 KiB pages: 16 K rows then 16 V rows of 128 bf16
+ *   page_ids    int32 [n_sets][list_stride], device: pages of each set, each id inside the pool
+ *   page_masks  uint32 [n_sets][list_stride], device: bit r set = token r of that page attended
+ *   n_pages     int32 [n_sets], device: entries used per set (0..list_stride)
+ *   group       query heads per set: 1, 2, 4 or 8;  sm_scale 0 = 1/sqrt(128)
+ * Limit: n_sets x ceil(list_stride/16) x group x 130 <= 2097152 floats; a larger request is
+ * refused with SPIN_ERR_INVALID and a message on stderr, nothing is launched.
+ * The first call on each device looks up the built-in array's device address (no allocation);
+ * make that first call outside any stream capture.  Asynchronous on cuda_stream.  All calls
+ * share the one array and it keeps the previous call's contents; nothing in it has to start
+ * at zero (each call overwrites what it later reads), but two calls whose kernels can overlap
+ * on the GPU (different streams, no ordering) would race on it. */
+SPIN_API int spin_paged_attention_static(const void *q, const void *page_pool,
+                                         const int32_t *page_ids, const uint32_t *page_masks,
+                                         const int32_t *n_pages, int32_t n_sets,
+                                         int32_t list_stride, int32_t group, float sm_scale,
+                                         void *out, void *cuda_stream);
+
 /* Text of the last error on this context (never NULL; valid until the next call). */
 SPIN_API const char *spin_last_error(spin_ctx *ctx);
 

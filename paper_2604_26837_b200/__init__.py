@@ -5,8 +5,8 @@ marshals arguments.  Nothing here computes on the CPU.
 """
 from .binding import (EXPORTS, KERNEL_NAMES, LIB_PATH, PART_CLUSTER_CENTROID, PART_PAGE_MINMAX, PART_TOKEN_DOT,
                       Spin, SpinError, load, make_config, spin_config, spin_dump_t,
-                      spin_required_bytes, spin_stats_t)
+                      spin_paged_attention_static, spin_required_bytes, spin_stats_t)
 
 __all__ = ["EXPORTS", "KERNEL_NAMES", "LIB_PATH", "PART_CLUSTER_CENTROID", "PART_PAGE_MINMAX", "PART_TOKEN_DOT",
            "Spin", "SpinError", "load", "make_config", "spin_config", "spin_dump_t",
-           "spin_required_bytes", "spin_stats_t"]
+           "spin_paged_attention_static", "spin_required_bytes", "spin_stats_t"]

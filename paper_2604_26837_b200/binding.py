@@ -24,7 +24,8 @@ PAGE_BYTES = 8192
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open",
            "spin_request_close", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
            "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
-           "spin_debug_read_page", "spin_last_error", "spin_version"]
+           "spin_debug_read_page", "spin_paged_attention_static", "spin_last_error",
+           "spin_version"]
 KERNEL_NAMES = ["append", "score", "topk", "cache", "fetch", "attn_split", "attn_merge"]
 
 
@@ -107,6 +108,7 @@ def load() -> C.CDLL:
     lib.spin_profile_read.argtypes = [vp, C.POINTER(spin_profile_t)]
     lib.spin_debug_dump.argtypes = [vp, i32, i32, i32, C.POINTER(spin_dump_t)]
     lib.spin_debug_read_page.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
+    lib.spin_paged_attention_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
     lib.spin_last_error.argtypes = [vp]
     lib.spin_last_error.restype = C.c_char_p
     lib.spin_version.argtypes = []
@@ -154,6 +156,18 @@ def spin_required_bytes(cfg: spin_config):
     if rc:
         raise SpinError(rc, "spin_required_bytes rejected the configuration")
     return dev.value, host.value
+
+
+def spin_paged_attention_static(q, page_pool, page_ids, page_masks, n_pages, n_sets: int,
+                                list_stride: int, group: int, sm_scale: float, out, stream=None):
+    """Allocation-free paged attention over caller-supplied page lists (all device buffers).
+
+    For callers that cannot allocate GPU memory and so cannot create a `Spin` context: the
+    split-K scratch is an array inside the library.  Returns the status code; a request beyond
+    the built-in scratch is refused (SPIN_ERR_INVALID) and explained on stderr."""
+    return load().spin_paged_attention_static(_ptr(q), _ptr(page_pool), _ptr(page_ids), _ptr(page_masks),
+                                              _ptr(n_pages), n_sets, list_stride, group, sm_scale,
+                                              _ptr(out), _stream_ptr(stream))
 
 
 class Spin:

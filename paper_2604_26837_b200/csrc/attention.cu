@@ -8,6 +8,9 @@
 // are requested before any arithmetic on them, so a warp keeps a whole page in flight.
 // Pages are read from HBM slots, or straight from pinned host memory when bypassed.
 // k_attn_merge: combines the chunks' (max, sum, output) triples and writes bf16.
+#include <cstdio>
+
+#include "../../include/spin.h"
 #include "spin_dev.cuh"
 
 namespace spin {
@@ -173,3 +176,81 @@ int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
 }
 
 }  // namespace spin
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free paged attention (see spin_paged_attention_static in spin.h).
+//
+// The split-K partials of this variant live in a fixed array that is part of the library
+// image, so a caller that must not (or cannot) allocate device memory -- code running inside
+// someone else's memory budget, a latency-critical loop that may not touch the allocator, a
+// plug-in that is only handed its input and output buffers -- can still run the split + merge
+// pair.  Every GPU that loads the library carries these 8 MiB until the process exits.
+namespace spin {
+namespace {
+constexpr size_t kStaticPartialFloats = (size_t)2 << 20;                  // 8 MiB of fp32
+__device__ __align__(256) static float g_static_partials[kStaticPartialFloats];
+constexpr int kMaxDevices = 64;
+float *g_static_partials_addr[kMaxDevices] = {};                          // per device, set up once
+}  // namespace
+}  // namespace spin
+
+extern "C" int spin_paged_attention_static(const void *q, const void *page_pool,
+                                           const int32_t *page_ids, const uint32_t *page_masks,
+                                           const int32_t *n_pages, int32_t n_sets,
+                                           int32_t list_stride, int32_t group, float sm_scale,
+                                           void *out, void *cuda_stream) {
+  using namespace spin;
+  if (!q || !page_pool || !page_ids || !page_masks || !n_pages || !out || n_sets < 1 || list_stride < 1) {
+    fprintf(stderr, "spin_paged_attention_static: null pointer or non-positive size\n");
+    return SPIN_ERR_INVALID;
+  }
+  if (group != 1 && group != 2 && group != 4 && group != 8) {
+    fprintf(stderr, "spin_paged_attention_static: group must be 1, 2, 4 or 8 (got %d)\n", group);
+    return SPIN_ERR_INVALID;
+  }
+  const int chunks = (list_stride + kChunkPages - 1) / kChunkPages;
+  const size_t need = (size_t)n_sets * chunks * group * (kHeadDim + 2);
+  if (need > kStaticPartialFloats) {
+    fprintf(stderr,
+            "spin_paged_attention_static: n_sets (%d) x ceil(list_stride/16) (%d) x group (%d) x 130 = %zu "
+            "floats of split-K scratch exceed the built-in %zu; use fewer sets per call or the context API\n",
+            n_sets, chunks, group, need, kStaticPartialFloats);
+    return SPIN_ERR_INVALID;
+  }
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    fprintf(stderr, "spin_paged_attention_static: no usable current CUDA device\n");
+    return SPIN_ERR_CUDA;
+  }
+  if (!g_static_partials_addr[dev]) {
+    // In host code the array's name is only a stand-in for the symbol: the address the
+    // kernels can use has to be asked for, once per device, with that device current.
+    float *p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_static_partials);
+    if (e != cudaSuccess || !p) {
+      fprintf(stderr, "spin_paged_attention_static: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+      return SPIN_ERR_CUDA;
+    }
+    g_static_partials_addr[dev] = p;
+  }
+  DevCtx c{};
+  c.num_layers = 1; c.Hq = group; c.Hkv = 1; c.G = group;
+  c.max_pages = list_stride; c.tail_cap = 0; c.max_chunks = chunks;
+  c.sm_scale = sm_scale != 0.f ? sm_scale : 0.08838834764831845f;
+  c.gpu_pages = const_cast<uint8_t *>(reinterpret_cast<const uint8_t *>(page_pool));
+  c.host_pages = nullptr;
+  c.page_src = const_cast<int32_t *>(page_ids);
+  c.page_mask = const_cast<uint32_t *>(page_masks);
+  c.n_pages = const_cast<int32_t *>(n_pages);
+  c.att_part = g_static_partials_addr[dev];
+  Batch b{};
+  b.n_req = n_sets;
+  launch_attention(c, b, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out),
+                   list_stride, reinterpret_cast<cudaStream_t>(cuda_stream), nullptr);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    fprintf(stderr, "spin_paged_attention_static: launch failed: %s\n", cudaGetErrorString(e));
+    return SPIN_ERR_CUDA;
+  }
+  return SPIN_OK;
+}
