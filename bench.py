@@ -174,6 +174,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--context", type=int, default=0, help="override the context length (smaller captures)")
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--fetch-mode", type=int, default=0, help="0 fused into attention, 1 separate copy kernel")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -223,7 +224,7 @@ def main():
     e2e_steps = 0 if args.no_e2e else K
     total_steps = P + Wm + K + K + prof_steps + (Wm + e2e_steps)
     w = W.scaled(base, seed=base.seed + 1000 * rank, steps=total_steps)
-    run = SpinRun(w, device)
+    run = SpinRun(w, device, fetch_mode=args.fetch_mode)
     stream = torch.cuda.Stream(device)
     B, L = w.batch, w.num_layers
 
@@ -250,10 +251,17 @@ def main():
                 for r in range(B):
                     q_all[s, l, r] = qstreams[(r, l)].next()
         out = torch.zeros(B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=device)
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        flush = torch.empty(64 << 20, dtype=torch.int32, device=device)        # 256 MiB
     torch.cuda.synchronize(device)
     pcie_gbs = measure_pcie_gbs(torch, device, stream)
     cur = [0]
+
+    def flush_l2_fn():
+        # write 256 MiB (> 126 MB L2), then read it back so that the L2 is left full of CLEAN
+        # lines, as it is after the weights of a model's other layers have streamed through;
+        # a write-only flush would leave dirty lines whose write-back taxes the timed kernels
+        flush.zero_()
+        flush.max()
 
     def one_step(s):
         for l in range(L):
@@ -265,7 +273,7 @@ def main():
         with torch.cuda.stream(stream):
             for _ in range(n):
                 if flush_l2:
-                    flush.zero_()
+                    flush_l2_fn()
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
                 one_step(cur[0])
@@ -316,7 +324,7 @@ def main():
         e2e_times = []
         with torch.cuda.stream(stream):
             for i in range(Wm + e2e_steps):
-                flush.zero_()
+                flush_l2_fn()
                 stream.synchronize()
                 t0 = time.perf_counter()
                 for l in range(L):
@@ -354,26 +362,40 @@ def main():
     t_step = elapsed_ms * 1e-3 / K
     dp = {k: stp1[k] - stp0[k] for k in stp0 if k != "error_bits"}
     kern = {}
-    bytes_of = dict(score=dp["candidates_scored"] * (512 if w.partition_kind == 0 else 256),
-                    fetch=(dp["miss_pages"] - dp["bypass_pages"]) * PAGE_BYTES,
-                    attn_split=(dp["selected_pages"] + dp["tail_pages"]) * PAGE_BYTES)
+    miss_b = dp["miss_pages"] * PAGE_BYTES
+    admit_b = (dp["miss_pages"] - dp["bypass_pages"]) * PAGE_BYTES
+    kv_b = (dp["selected_pages"] + dp["tail_pages"]) * PAGE_BYTES
+    fused = args.fetch_mode == 0
+    # algorithmic bytes per kernel over the profiled steps: (HBM bytes, host-link bytes)
+    bytes_of = dict(score=(dp["candidates_scored"] * (512 if w.partition_kind == 0 else 256), 0),
+                    fetch=(admit_b, admit_b),
+                    attn_split=((kv_b - miss_b + admit_b, miss_b) if fused else (kv_b - (miss_b - admit_b), miss_b - admit_b)))
     tot_ms = sum(ms for _, ms in prof.values()) or 1.0
     for name, (n, ms) in prof.items():
-        kern[name] = dict(launches=n, avg_us=1e3 * ms / max(n, 1), share=ms / tot_ms)
-        if name in bytes_of and n:
-            kern[name]["gbs"] = bytes_of[name] / (ms * 1e-3) / 1e9
-    top = max(("fetch", "score", "attn_split"), key=lambda k_: kern[k_]["share"] if k_ in kern else 0)
-    bound = "pcie" if top == "fetch" else "hbm"
+        if not n:
+            continue
+        kern[name] = dict(launches=n, avg_us=1e3 * ms / n, share=ms / tot_ms)
+        if name in bytes_of:
+            hb, pb = bytes_of[name]
+            t_h, t_p = hb / (peaks["hbm_gbs"] * 1e9), pb / (pcie_gbs * 1e9)
+            kern[name].update(hbm_gbs=hb / (ms * 1e-3) / 1e9, pcie_gbs=pb / (ms * 1e-3) / 1e9,
+                              bound="pcie" if t_p > t_h else "hbm", roof_frac=max(t_h, t_p) / (ms * 1e-3))
+    top = max((k_ for k_ in ("fetch", "score", "attn_split") if k_ in kern), key=lambda k_: kern[k_]["share"])
+    bound = kern[top]["bound"]
     peak = pcie_gbs if bound == "pcie" else peaks["hbm_gbs"]
+    achieved = kern[top]["pcie_gbs"] if bound == "pcie" else kern[top]["hbm_gbs"]
     traffic = (NCU_TRAFFIC.get(args.workload) or {}).get(top) if not (args.context or args.batch) else None
-    roofline = dict(kernel="k_" + top, bound=bound, achieved=kern[top].get("gbs"), peak=peak, unit="GB/s",
-                    frac=(kern[top]["gbs"] / peak) if kern[top].get("gbs") else None, traffic=traffic,
+    names = dict(fetch="k_fetch", score="k_score", attn_split="k_attn (attention + page fetch)" if fused else "k_attn")
+    roofline = dict(kernel=names[top], bound=bound, achieved=achieved, peak=peak, unit="GB/s",
+                    frac=kern[top]["roof_frac"], traffic=traffic,
                     peak_source=("pinned H2D copy measured in this run" if bound == "pcie" else peaks["source"]),
-                    avg_launch_us=kern[top]["avg_us"], bytes_per_launch=bytes_of[top] / max(kern[top]["launches"], 1))
+                    avg_launch_us=kern[top]["avg_us"],
+                    hbm_bytes_per_launch=bytes_of[top][0] / kern[top]["launches"],
+                    pcie_bytes_per_launch=bytes_of[top][1] / kern[top]["launches"])
     line = dict(
         metric=metric, value=value, unit=unit, n_gpus=world, steps=K, warmup=Wm, ms_per_step=elapsed_ms / K,
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16 in, f32 accumulate", data="synthetic",
-        config=dict(cfg_desc, primed_steps=P, l2="flushed between timed steps (256 MiB memset, untimed)",
+        config=dict(cfg_desc, primed_steps=P, l2="flushed between timed steps (256 MiB written then read back, untimed)",
                     note="single-layer config: tokens/s is per-layer-step throughput"),
         p50_tpot_ms=statistics.median(per_step), ms_per_step_noflush=noflush_ms,
         gpu_launches=int(d["kernel_launches"]), clocks=clocks,

@@ -93,6 +93,9 @@ typedef struct spin_config {
   int32_t segment_entries;      /* entries per second-level segment, power of two; 0 = 256 */
   float sm_scale;               /* softmax scale; 0 = 1/sqrt(head_dim) */
   int32_t trace;                /* != 0: record per-step eviction traces for spin_debug_dump */
+  int32_t fetch_mode;           /* 0: missed pages are fetched inside the attention kernel (they
+                                   cross the host link while the hits are attended from HBM);
+                                   1: by a separate persistent warp-per-page copy kernel */
   int64_t gpu_cache_pages;      /* HBM pages (8 KiB each) shared by all sets' cache slots */
   int64_t host_pages;           /* pinned host pages (8 KiB each) for the complete KV */
   void *hbm_pool;               /* device pointer, 256-byte aligned, caller-owned */
@@ -225,7 +228,7 @@ SPIN_API int spin_debug_read_page(spin_ctx *ctx, int32_t req, int32_t layer, int
  * memory budget, or on a path where touching an allocator is forbidden -- and therefore
  * cannot create a context, whose scratch comes out of a caller-allocated pool).
  * It runs the same split-K attention + log-sum-exp merge as spin_decode_step's last stage over
- * page lists the caller supplies; the split-K partials go to an 8 MiB array built into the
+ * page lists the caller supplies; the split-K partials and counters use an 8 MiB array built into the
  * library image (every GPU that loads the library holds it until the process exits).
  *   q, out      bf16 [n_sets][group][128], device pointers (out is written)
  *   page_pool   device pointer to 8 KiB pages: 16 K rows then 16 V rows of 128 bf16
@@ -233,13 +236,15 @@ SPIN_API int spin_debug_read_page(spin_ctx *ctx, int32_t req, int32_t layer, int
  *   page_masks  uint32 [n_sets][list_stride], device: bit r set = token r of that page attended
  *   n_pages     int32 [n_sets], device: entries used per set (0..list_stride)
  *   group       query heads per set: 1, 2, 4 or 8;  sm_scale 0 = 1/sqrt(128)
- * Limit: n_sets x ceil(list_stride/16) x group x 130 <= 2097152 floats; a larger request is
- * refused with SPIN_ERR_INVALID and a message on stderr, nothing is launched.
+ * Limit: n_sets x ceil(list_stride/8) x group x 130 + n_sets (rounded up to 64) <= 2097152
+ * four-byte words; a larger request is refused with SPIN_ERR_INVALID and a message on stderr,
+ * nothing is launched.
  * The first call on each device looks up the built-in array's device address (no allocation);
  * make that first call outside any stream capture.  Asynchronous on cuda_stream.  All calls
- * share the one array and it keeps the previous call's contents; nothing in it has to start
- * at zero (each call overwrites what it later reads), but two calls whose kernels can overlap
- * on the GPU (different streams, no ordering) would race on it. */
+ * share the one array and it keeps the previous call's contents; the call clears the per-set
+ * arrival counters at its start (the only part that must begin at zero) and overwrites what
+ * else it later reads, but two calls whose kernels can overlap on the GPU (different streams,
+ * no ordering) would race on it. */
 SPIN_API int spin_paged_attention_static(const void *q, const void *page_pool,
                                          const int32_t *page_ids, const uint32_t *page_masks,
                                          const int32_t *n_pages, int32_t n_sets,

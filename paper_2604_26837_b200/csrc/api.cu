@@ -132,7 +132,7 @@ int compute_geometry(const spin_config &cfg, Geometry &g, std::string &err) {
   g.n_cpt_segs = (cfg.host_pages + g.seg - 1) / g.seg + g.n_sets;
   g.fetch_cap = (int64_t)g.max_batch_sets * g.max_pages;
   g.stage_tokens = 2048;
-  if ((size_t)(5 * g.max_parts + 1 + g.max_pages) * 4 + (size_t)((g.max_slots + 31) / 32) * 4 > 200 * 1024)
+  if ((size_t)(6 * g.max_parts + 1 + g.max_pages) * 4 + (size_t)((g.max_slots + 31) / 32) * 4 > 200 * 1024)
     return bad("topk / max_selected_pages / budget too large for the cache kernel's shared memory");
   return SPIN_OK;
 }
@@ -214,6 +214,8 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.n_parts = a.take<int32_t>(B);
   d.page_src = a.take<int32_t>(B * PL);
   d.page_mask = a.take<uint32_t>(B * PL);
+  d.page_fill = a.take<int32_t>(B * PL);
+  d.page_desc = a.take<int4>(B * PL);
   d.page_slot = a.take<int32_t>(B * PL);
   d.page_part = a.take<int32_t>(B * PL);
   d.page_pidx = a.take<int32_t>(B * PL);
@@ -221,6 +223,7 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.fetch_queue = a.take<FetchItem>((size_t)g.fetch_cap);
   d.fetch_count = a.take<int32_t>(1);
   d.att_part = a.take<float>(B * g.max_chunks * G * (kHeadDim + 2));
+  d.att_count = a.take<int32_t>(B);
   d.counters = a.take<Counters>(1);
   __nv_bfloat16 *sq = a.take<__nv_bfloat16>((size_t)cfg.max_requests * cfg.num_q_heads * kHeadDim);
   __nv_bfloat16 *so = a.take<__nv_bfloat16>((size_t)cfg.max_requests * cfg.num_q_heads * kHeadDim);
@@ -611,6 +614,9 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   d.max_sel = g.max_sel; d.max_parts = g.max_parts; d.max_pages = g.max_pages; d.tail_cap = g.tail_cap;
   d.max_cand = (int32_t)g.max_cand; d.max_slots = (int32_t)g.max_slots; d.max_chunks = g.max_chunks;
   d.fetch_cap = (int32_t)g.fetch_cap;
+  d.n_gpu_pages = (int32_t)g.n_gpu_pages_total;
+  d.n_host_pages = (int32_t)cfg->host_pages;
+  d.fetch_mode = cfg->fetch_mode ? 1 : 0;
   d.sm_scale = cfg->sm_scale != 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)kHeadDim);
 
   // directories start unmapped (-1); states, counters and the miss queue start at zero
@@ -620,6 +626,11 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   fill(d.dir_gpt, 0xff, (size_t)g.n_sets * g.dir_slot * 4);
   fill(d.dir_cpt, 0xff, (size_t)g.n_sets * g.dir_page * 4);
   fill(d.dir_sumseg, 0xff, (size_t)g.n_sets * g.dir_sum * 4);
+  // every byte a kernel may read as K/V is finite from the start (rows past a page's valid
+  // tokens are masked out of the softmax but still enter the P*V tiles with weight 0)
+  fill(d.gpu_pages, 0, (size_t)g.n_gpu_pages_total * kPageBytes);
+  memset(ctx->host_base, 0, ctx->host_bytes);
+  fill(d.att_count, 0, (size_t)g.max_batch_sets * 4);
   fill(d.state, 0, (size_t)g.n_sets * sizeof(SetState));
   fill(d.counters, 0, sizeof(Counters));
   fill(d.fetch_count, 0, 4);
@@ -834,6 +845,7 @@ int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   b.n_req = n_req;
   b.layer = layer;
   int64_t max_cand = 0, max_pages = 0;
+  bool may_be_empty = false;
   for (int i = 0; i < n_req; ++i) {
     int rc = validate_req_layer(ctx, req_ids[i], layer);
     if (rc) return rc;
@@ -846,6 +858,7 @@ int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
                         ? ctx->g.max_pages
                         : std::min<int64_t>(ctx->cfg.topk, L.n_partitions);
     max_pages = std::max(max_pages, pages + L.tail_pages);
+    may_be_empty = may_be_empty || L.n_tokens == 0;
     L.last_batch_pos = i;
   }
   const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
@@ -857,7 +870,7 @@ int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   prof_mark(&ctx->prof, st, -1);
   ctx->launches += launch_select(ctx->d, b, qd, (int)max_cand, st, &ctx->prof);
   ctx->launches += launch_cache(ctx->d, b, st, ctx->sm_count, &ctx->prof);
-  ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, st, &ctx->prof);
+  ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, may_be_empty, st, &ctx->prof);
   if (!out_dev) CK(cudaMemcpyAsync(out, ctx->stage_out, qbytes, cudaMemcpyDeviceToHost, st));
   CK(cudaGetLastError());
   return SPIN_OK;

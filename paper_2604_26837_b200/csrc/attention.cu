@@ -1,13 +1,19 @@
-// Attention over the selected pages plus the local tail (Section 4.1 "Attention"): paged GQA
-// decode attention, split over chunks of the page list and merged by log-sum-exp.
+// Attention over the selected pages plus the local tail (Section 4.1 "Attention"), fused with
+// the page fetch of Retrieve step 4 (Section 5.2): paged GQA decode attention, split over
+// chunks of the page list and merged by log-sum-exp.
 //
-// k_attn_split: one CTA per (set, chunk of 16 pages); each warp walks pages of the chunk.
-// A half-warp owns one token row at a time: lane l holds channels 8l..8l+7 of the K and V
-// row (one 16-byte load each), dots them with the group's query heads, reduces over the 16
-// lanes and folds the row into a running (max, sum, weighted V) per head.  A page's 8 KiB
-// are requested before any arithmetic on them, so a warp keeps a whole page in flight.
-// Pages are read from HBM slots, or straight from pinned host memory when bypassed.
-// k_attn_merge: combines the chunks' (max, sum, output) triples and writes bf16.
+// k_attn: one CTA (4 warps) per (set, chunk of 8 pages).  Each warp owns two pages of the
+// chunk.  It requests both pages at once with 16-byte cp.async copies into XOR-swizzled
+// shared memory (a page is one contiguous 8 KiB run: 16 K rows then 16 V rows) -- from an
+// HBM slot for a hit, straight from pinned host memory for a miss -- so every missed page of
+// the step is in flight on the host link while the hits are being attended from HBM.  A
+// missed page that was admitted to the cache is written from shared memory into its HBM
+// slot after use (that is the fetch); a bypassed page is only attended.  QK^T and PV run on
+// mma.sync m16n8k16 bf16 tiles with fp32 accumulators (query heads padded to M = 16, the
+// page's 16 tokens as N resp. K): at ~4 flop/byte the kernel is HBM/PCIe bound and tensor
+// tiles are used to take instruction issue off the critical path, which is also why the
+// 64..128-row tcgen05 tiles (>90% padding at GQA 4) are not.  The last CTA of a set to finish
+// (a counter cleared by the cache-manager kernel) merges the set's partials and writes bf16.
 #include <cstdio>
 
 #include "../../include/spin.h"
@@ -20,159 +26,334 @@ namespace {
 constexpr int kAttnWarps = 4;
 constexpr int kPartStride = kHeadDim + 2;       // per head: 128 outputs, max, sum
 
-__device__ __forceinline__ void unpack8(uint4 raw, float *f) {
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Byte offset of the 16-byte piece `chunk` (0..15) of row `row` (0..31: K rows, then V rows)
+// inside a page staged in shared memory.  Pieces are XOR-swizzled by the row so that the 8
+// rows an ldmatrix touches fall into 8 different bank groups.
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+  return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+}
+
+// One warp requests one page: 16 copies of 16 bytes per lane, 512 contiguous bytes per instruction.
+__device__ __forceinline__ void request_page(uint32_t sdst, const uint8_t *src, int lane) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    f[2 * i] = __uint_as_float(w[i] << 16);
-    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  for (int j = 0; j < 16; ++j) {
+    const int piece = j * 32 + lane;              // 0..511
+    const int row = piece >> 4, chunk = piece & 15;
+    cp_async16(sdst + swz(row, chunk), src + (size_t)piece * 16);
+  }
+}
+
+struct WarpAcc {
+  float m, l;                 // running max (base-2 logits) and partial sum of this lane's row
+  float o[16][4];             // 16 n-tiles of 8 channels; [.][0..1] = row lane/4, [.][2..3] = row+8 (unused, zero)
+};
+
+// Attend one staged page: S = Q K^T (16 x 16), online softmax, O += P V.
+__device__ __forceinline__ void attend_page(uint32_t spage, const uint32_t (&qa)[8][2], uint32_t mask,
+                                            float scale2, WarpAcc &acc, int lane) {
+  float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+  const int mat = lane >> 3, r8 = lane & 7;
+  {
+    const int token = r8 + ((mat >> 1) << 3);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4(spage + swz(token, 2 * ks + (mat & 1)), b0, b1, b2, b3);
+      mma_bf16(s[0], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+      mma_bf16(s[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+    }
+  }
+  // this lane's row = lane/4; its tokens: nt*8 + (lane%4)*2 + {0,1}
+  float p[2][2];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int tok = nt * 8 + (lane & 3) * 2 + j;
+      const float v = ((mask >> tok) & 1u) ? s[nt][j] * scale2 : -INFINITY;
+      p[nt][j] = v;
+      mx = fmaxf(mx, v);
+    }
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+  const float mn = fmaxf(acc.m, mx);
+  const float base = mn == -INFINITY ? 0.f : mn;           // all masked so far: every p is 0
+  const float corr = exp2f(acc.m - base);                  // acc.m = -inf -> 0
+  float psum = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      p[nt][j] = exp2f(p[nt][j] - base);
+      psum += p[nt][j];
+    }
+  acc.l = acc.l * corr + psum;
+  acc.m = mn;
+  const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]), pa2 = pack_bf16(p[1][0], p[1][1]);
+  {
+    const int token = r8 + ((mat & 1) << 3);
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4_trans(spage + swz(kPageTokens + token, 2 * nb + (mat >> 1)), b0, b1, b2, b3);
+      acc.o[2 * nb][0] *= corr; acc.o[2 * nb][1] *= corr;
+      acc.o[2 * nb + 1][0] *= corr; acc.o[2 * nb + 1][1] *= corr;
+      mma_bf16(acc.o[2 * nb], pa0, 0u, pa2, 0u, b0, b1);
+      mma_bf16(acc.o[2 * nb + 1], pa0, 0u, pa2, 0u, b2, b3);
+    }
+  }
+}
+
+// Retrieve step 4 for one admitted miss: the staged page goes to its HBM slot.
+__device__ __forceinline__ void store_page(const uint8_t *spage_generic, uint8_t *dst, int lane) {
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const int piece = j * 32 + lane;
+    const int row = piece >> 4, chunk = piece & 15;
+    *reinterpret_cast<uint4 *>(dst + (size_t)piece * 16) =
+        *reinterpret_cast<const uint4 *>(spage_generic + swz(row, chunk));
   }
 }
 
 template <int G>
 __global__ void __launch_bounds__(kAttnWarps * 32)
-k_attn_split(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
+k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out) {
+  extern __shared__ __align__(128) uint8_t smem_pages[];          // [8][8192]
   __shared__ float sh[kAttnWarps][G][kPartStride];
-  const int b = blockIdx.y, chunk = blockIdx.x;
+  __shared__ int sh_last;
+  const int b = blockIdx.x, chunk = blockIdx.y;       // chunk-major launch order: chunk 0 of every set first
   const int np = c.n_pages[b];
   const int first = chunk * kChunkPages;
   if (first >= np) return;
   const int last = min(np, first + kChunkPages);
   const int i_req = b / c.Hkv, head = b % c.Hkv;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, l16 = lane & 15, half = lane >> 4;
-  const uint32_t row_mask = 0xffffu << (lane & 16);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t pl = (size_t)b * (c.max_pages + c.tail_cap);
 
-  // logits in base 2: q is pre-scaled by sm_scale * log2(e)
-  const float qs = c.sm_scale * 1.4426950408889634f;
-  float qf[G][8], m[G], l[G], o[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    unpack8(*reinterpret_cast<const uint4 *>(q + ((size_t)i_req * c.Hq + head * G + g) * kHeadDim + l16 * 8), qf[g]);
-    m[g] = -INFINITY;
-    l[g] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) { qf[g][i] *= qs; o[g][i] = 0.f; }
+  // the warp's two pages; the one that has to cross the host link is waited for last
+  int pg[2] = {first + warp, first + warp + kAttnWarps};
+  int n_mine = (pg[0] < last) + (pg[1] < last);
+  int src[2] = {0, 0}, fill[2] = {-1, -1};
+  uint32_t mask[2] = {0, 0};
+  for (int i = 0; i < n_mine; ++i) {
+    if (c.page_desc) {                      // work-ordered descriptors written by the cache manager
+      const int4 dsc = c.page_desc[pl + pg[i]];
+      src[i] = dsc.x; fill[i] = dsc.y; mask[i] = (uint32_t)dsc.z;
+    } else {                                // plain lists, attended in the order given
+      src[i] = c.page_src[pl + pg[i]];
+      mask[i] = c.page_mask[pl + pg[i]];
+    }
+    // a descriptor that points outside the pools is dropped (and reported), never followed
+    const bool ok = (src[i] >= 0 ? src[i] < c.n_gpu_pages : ~src[i] < c.n_host_pages) && fill[i] < c.n_host_pages;
+    if (!ok) { if (lane == 0) dev_error(c, kErrBounds); src[i] = 0; fill[i] = -1; mask[i] = 0; }
+  }
+  if (n_mine == 2 && (fill[0] >= 0 || src[0] < 0) && !(fill[1] >= 0 || src[1] < 0)) {
+    int t = src[0]; src[0] = src[1]; src[1] = t;
+    t = fill[0]; fill[0] = fill[1]; fill[1] = t;
+    uint32_t u = mask[0]; mask[0] = mask[1]; mask[1] = u;
+  }
+  uint8_t *spage[2] = {smem_pages + (size_t)(2 * warp) * kPageBytes, smem_pages + (size_t)(2 * warp + 1) * kPageBytes};
+  for (int i = 0; i < 2; ++i) {
+    if (i < n_mine) {
+      const uint8_t *from = fill[i] >= 0 ? c.host_pages + (size_t)fill[i] * kPageBytes : page_ptr(c, src[i]);
+      request_page(smem_u32(spage[i]), from, lane);
+    }
+    cp_async_commit();
   }
 
-  for (int pg = first + warp; pg < last; pg += kAttnWarps) {
-    const uint8_t *page = page_ptr(c, c.page_src[pl + pg]);
-    const uint32_t mask = c.page_mask[pl + pg];
-    uint4 kraw[8], vraw[8];
+  // Q as A-operand fragments: row = lane/4 (query head, zero beyond G), 8 k-steps of 16 channels
+  uint32_t qa[8][2];
+  {
+    const int row = lane >> 2;
+    const uint32_t *qrow = reinterpret_cast<const uint32_t *>(q + ((size_t)i_req * c.Hq + head * G + (row < G ? row : 0)) * kHeadDim);
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int row = 2 * it + half;
-      if ((mask >> row) & 1u) {
-        kraw[it] = *reinterpret_cast<const uint4 *>(page + row * kRowBytes + l16 * 16);
-        vraw[it] = *reinterpret_cast<const uint4 *>(page + kHalfPageBytes + row * kRowBytes + l16 * 16);
-      }
-    }
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int row = 2 * it + half;
-      if (!((mask >> row) & 1u)) continue;
-      float kf[8], vf[8];
-      unpack8(kraw[it], kf);
-      unpack8(vraw[it], vf);
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float s = qf[g][0] * kf[0];
-#pragma unroll
-        for (int i = 1; i < 8; ++i) s = fmaf(qf[g][i], kf[i], s);
-        s += __shfl_xor_sync(row_mask, s, 1);
-        s += __shfl_xor_sync(row_mask, s, 2);
-        s += __shfl_xor_sync(row_mask, s, 4);
-        s += __shfl_xor_sync(row_mask, s, 8);
-        const float mn = fmaxf(m[g], s);
-        const float corr = exp2f(m[g] - mn), p = exp2f(s - mn);
-        l[g] = l[g] * corr + p;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[g][i] = fmaf(o[g][i], corr, p * vf[i]);
-        m[g] = mn;
-      }
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = row < G ? qrow[ks * 8 + (lane & 3)] : 0u;
+      qa[ks][1] = row < G ? qrow[ks * 8 + 4 + (lane & 3)] : 0u;
     }
   }
-  // fold the two half-warps, then the warps of the CTA
+  WarpAcc acc;
+  acc.m = -INFINITY;
+  acc.l = 0.f;
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const float m2 = __shfl_xor_sync(0xffffffffu, m[g], 16);
-    const float l2 = __shfl_xor_sync(0xffffffffu, l[g], 16);
-    const float mn = fmaxf(m[g], m2);
-    const float a = m[g] == -INFINITY ? 0.f : exp2f(m[g] - mn);
-    const float a2 = m2 == -INFINITY ? 0.f : exp2f(m2 - mn);
+  for (int i = 0; i < 16; ++i) { acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f; }
+  const float scale2 = c.sm_scale * 1.4426950408889634f;
+
+  cp_async_wait<1>();
+  __syncwarp();
+  if (n_mine >= 1) {
+    attend_page(smem_u32(spage[0]), qa, mask[0], scale2, acc, lane);
+    if (fill[0] >= 0) store_page(spage[0], c.gpu_pages + (size_t)src[0] * kPageBytes, lane);
+  }
+  cp_async_wait<0>();
+  __syncwarp();
+  if (n_mine >= 2) {
+    attend_page(smem_u32(spage[1]), qa, mask[1], scale2, acc, lane);
+    if (fill[1] >= 0) store_page(spage[1], c.gpu_pages + (size_t)src[1] * kPageBytes, lane);
+  }
+
+  // row sums live in the 4 lanes of a quad
+  acc.l += __shfl_xor_sync(0xffffffffu, acc.l, 1);
+  acc.l += __shfl_xor_sync(0xffffffffu, acc.l, 2);
+  {
+    const int row = lane >> 2;
+    if (row < G) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float o2 = __shfl_xor_sync(0xffffffffu, o[g][i], 16);
-      o[g][i] = o[g][i] * a + o2 * a2;
-    }
-    l[g] = l[g] * a + l2 * a2;
-    m[g] = mn;
-    if (half == 0) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) sh[warp][g][l16 * 8 + i] = o[g][i];
-      if (l16 == 0) { sh[warp][g][kHeadDim] = mn; sh[warp][g][kHeadDim + 1] = l[g]; }
+      for (int nt = 0; nt < 16; ++nt) {
+        sh[warp][row][nt * 8 + (lane & 3) * 2] = acc.o[nt][0];
+        sh[warp][row][nt * 8 + (lane & 3) * 2 + 1] = acc.o[nt][1];
+      }
+      if ((lane & 3) == 0) { sh[warp][row][kHeadDim] = acc.m; sh[warp][row][kHeadDim + 1] = acc.l; }
     }
   }
   __syncthreads();
-  float *out = c.att_part + ((size_t)b * c.max_chunks + chunk) * G * kPartStride;
+  const int n_chunks = (np + kChunkPages - 1) / kChunkPages;
+  float *part = c.att_part + ((size_t)b * c.max_chunks + chunk) * G * kPartStride;
   for (int e = threadIdx.x; e < G * kHeadDim; e += kAttnWarps * 32) {
     const int g = e / kHeadDim, ch = e % kHeadDim;
     float mn = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kAttnWarps; ++w) mn = fmaxf(mn, sh[w][g][kHeadDim]);
-    float acc = 0.f, ls = 0.f;
+    float a_o = 0.f, a_l = 0.f;
 #pragma unroll
     for (int w = 0; w < kAttnWarps; ++w) {
       const float mw = sh[w][g][kHeadDim];
       const float a = mw == -INFINITY ? 0.f : exp2f(mw - mn);
-      acc += sh[w][g][ch] * a;
-      ls += sh[w][g][kHeadDim + 1] * a;
+      a_o += sh[w][g][ch] * a;
+      a_l += sh[w][g][kHeadDim + 1] * a;
     }
-    out[g * kPartStride + ch] = acc;
-    if (ch == 0) { out[g * kPartStride + kHeadDim] = mn; out[g * kPartStride + kHeadDim + 1] = ls; }
+    if (n_chunks == 1) {
+      // only chunk of the set: finish here
+      out[((size_t)i_req * c.Hq + head * G + g) * kHeadDim + ch] = __float2bfloat16(a_l > 0.f ? a_o / a_l : 0.f);
+    } else {
+      part[g * kPartStride + ch] = a_o;
+      if (ch == 0) { part[g * kPartStride + kHeadDim] = mn; part[g * kPartStride + kHeadDim + 1] = a_l; }
+    }
+  }
+  if (n_chunks == 1) return;
+  // the last CTA of the set to get here merges all partials (log-sum-exp)
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) sh_last = atomicAdd(&c.att_count[b], 1) == n_chunks - 1;
+  __syncthreads();
+  if (!sh_last) return;
+  __threadfence();
+  // merge: the per-chunk (max, sum) pairs first, then the outputs, with the loads of a batch
+  // of chunks issued together
+  const float *parts = c.att_part + (size_t)b * c.max_chunks * G * kPartStride;
+  float *s_scale = reinterpret_cast<float *>(smem_pages);         // [n_chunks][G] weights exp2(m_k - m)
+  float *s_m = s_scale + (size_t)n_chunks * G;                    // [n_chunks][G]
+  float *s_l = s_m + (size_t)n_chunks * G;                        // [n_chunks][G]
+  float *s_den = s_l + (size_t)n_chunks * G;                      // [G]
+  for (int e = threadIdx.x; e < n_chunks * G; e += kAttnWarps * 32) {
+    const int k = e / G, g = e % G;
+    const float *pp = parts + ((size_t)k * G + g) * kPartStride;
+    s_m[e] = __ldcg(pp + kHeadDim);
+    s_l[e] = __ldcg(pp + kHeadDim + 1);
+  }
+  __syncthreads();
+  if (threadIdx.x < G) {
+    const int g = threadIdx.x;
+    float mn = -INFINITY;
+    for (int k = 0; k < n_chunks; ++k) mn = fmaxf(mn, s_m[k * G + g]);
+    float den = 0.f;
+    for (int k = 0; k < n_chunks; ++k) {
+      const float mk = s_m[k * G + g];
+      const float a = mk == -INFINITY ? 0.f : exp2f(mk - mn);
+      s_scale[k * G + g] = a;
+      den += s_l[k * G + g] * a;
+    }
+    s_den[g] = den;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < G * kHeadDim; e += kAttnWarps * 32) {
+    const int g = e / kHeadDim, ch = e % kHeadDim;
+    const float *pg_ = parts + g * kPartStride + ch;
+    float a_o = 0.f;
+    int k = 0;
+    for (; k + 8 <= n_chunks; k += 8) {
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = __ldcg(pg_ + (size_t)(k + j) * G * kPartStride);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) a_o = fmaf(v[j], s_scale[(k + j) * G + g], a_o);
+    }
+    for (; k < n_chunks; ++k) a_o = fmaf(__ldcg(pg_ + (size_t)k * G * kPartStride), s_scale[k * G + g], a_o);
+    const float den = s_den[g];
+    out[((size_t)i_req * c.Hq + head * G + g) * kHeadDim + ch] = __float2bfloat16(den > 0.f ? a_o / den : 0.f);
   }
 }
 
-// grid: (G, batch sets); 128 threads = channels
-__global__ void __launch_bounds__(kHeadDim)
-k_attn_merge(DevCtx c, Batch bt, __nv_bfloat16 *__restrict__ out) {
-  const int b = blockIdx.y, g = blockIdx.x, ch = threadIdx.x;
+// Sets whose page list is empty get a zero output (no CTA of k_attn reaches them).
+__global__ void k_attn_zero_empty(DevCtx c, __nv_bfloat16 *__restrict__ out, int n_sets) {
+  const int b = blockIdx.x;
+  if (b >= n_sets || c.n_pages[b] != 0) return;
   const int i_req = b / c.Hkv, head = b % c.Hkv;
-  const int n_chunks = (c.n_pages[b] + kChunkPages - 1) / kChunkPages;
-  const float *part = c.att_part + ((size_t)b * c.max_chunks * c.G + g) * kPartStride;
-  const size_t stride = (size_t)c.G * kPartStride;
-  float mn = -INFINITY;
-  for (int k = 0; k < n_chunks; ++k) mn = fmaxf(mn, part[k * stride + kHeadDim]);
-  float acc = 0.f, ls = 0.f;
-  for (int k = 0; k < n_chunks; ++k) {
-    const float mk = part[k * stride + kHeadDim];
-    const float a = mk == -INFINITY ? 0.f : exp2f(mk - mn);
-    acc += part[k * stride + ch] * a;
-    ls += part[k * stride + kHeadDim + 1] * a;
+  for (int e = threadIdx.x; e < c.G * kHeadDim; e += blockDim.x)
+    out[((size_t)i_req * c.Hq + head * c.G) * kHeadDim + e] = __float2bfloat16(0.f);
+}
+
+template <int G>
+void launch_attn_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, __nv_bfloat16 *out, dim3 grid,
+                   cudaStream_t st) {
+  static bool configured = false;
+  constexpr int smem = kChunkPages * kPageBytes;
+  if (!configured) {
+    cudaFuncSetAttribute(k_attn<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
   }
-  const float r = ls > 0.f ? acc / ls : 0.f;
-  out[((size_t)i_req * c.Hq + head * c.G + g) * kHeadDim + ch] = __float2bfloat16(r);
+  k_attn<G><<<grid, kAttnWarps * 32, smem, st>>>(c, b, q, out);
 }
 
 }  // namespace
 
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
-                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st, Prof *prof) {
+                     __nv_bfloat16 *out, int max_pages_hint, bool may_be_empty, cudaStream_t st, Prof *prof) {
   const int n_sets = b.n_req * c.Hkv;
   int chunks = (max_pages_hint + kChunkPages - 1) / kChunkPages;
   if (chunks < 1) chunks = 1;
   if (chunks > c.max_chunks) chunks = c.max_chunks;
-  dim3 grid(chunks, n_sets);
+  dim3 grid(n_sets, chunks);
+  int launched = 1;
+  if (may_be_empty) { k_attn_zero_empty<<<n_sets, 128, 0, st>>>(c, out, n_sets); ++launched; }
   switch (c.G) {
-    case 1: k_attn_split<1><<<grid, kAttnWarps * 32, 0, st>>>(c, b, q); break;
-    case 2: k_attn_split<2><<<grid, kAttnWarps * 32, 0, st>>>(c, b, q); break;
-    case 4: k_attn_split<4><<<grid, kAttnWarps * 32, 0, st>>>(c, b, q); break;
-    default: k_attn_split<8><<<grid, kAttnWarps * 32, 0, st>>>(c, b, q); break;
+    case 1: launch_attn_g<1>(c, b, q, out, grid, st); break;
+    case 2: launch_attn_g<2>(c, b, q, out, grid, st); break;
+    case 4: launch_attn_g<4>(c, b, q, out, grid, st); break;
+    default: launch_attn_g<8>(c, b, q, out, grid, st); break;
   }
   prof_mark(prof, st, kProfAttnSplit);
-  k_attn_merge<<<dim3(c.G, n_sets), kHeadDim, 0, st>>>(c, b, out);
-  prof_mark(prof, st, kProfAttnMerge);
-  return 2;
+  return launched;
 }
 
 }  // namespace spin
@@ -180,7 +361,7 @@ int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
 // ---------------------------------------------------------------------------------------
 // Allocation-free paged attention (see spin_paged_attention_static in spin.h).
 //
-// The split-K partials of this variant live in a fixed array that is part of the library
+// The split-K partials and arrival counters of this variant live in a fixed array that is part of the library
 // image, so a caller that must not (or cannot) allocate device memory -- code running inside
 // someone else's memory budget, a latency-critical loop that may not touch the allocator, a
 // plug-in that is only handed its input and output buffers -- can still run the split + merge
@@ -209,12 +390,14 @@ extern "C" int spin_paged_attention_static(const void *q, const void *page_pool,
     return SPIN_ERR_INVALID;
   }
   const int chunks = (list_stride + kChunkPages - 1) / kChunkPages;
-  const size_t need = (size_t)n_sets * chunks * group * (kHeadDim + 2);
+  // layout of the built-in array: [n_sets] arrival counters (as int32), then the partials
+  const size_t counter_floats = ((size_t)n_sets + 63) / 64 * 64;
+  const size_t need = counter_floats + (size_t)n_sets * chunks * group * (kHeadDim + 2);
   if (need > kStaticPartialFloats) {
     fprintf(stderr,
-            "spin_paged_attention_static: n_sets (%d) x ceil(list_stride/16) (%d) x group (%d) x 130 = %zu "
-            "floats of split-K scratch exceed the built-in %zu; use fewer sets per call or the context API\n",
-            n_sets, chunks, group, need, kStaticPartialFloats);
+            "spin_paged_attention_static: n_sets (%d) x ceil(list_stride/8) (%d) x group (%d) x 130 partial "
+            "floats + %zu counters = %zu exceed the built-in %zu; use fewer sets per call or the context API\n",
+            n_sets, chunks, group, counter_floats, need, kStaticPartialFloats);
     return SPIN_ERR_INVALID;
   }
   int dev = -1;
@@ -239,15 +422,28 @@ extern "C" int spin_paged_attention_static(const void *q, const void *page_pool,
   c.sm_scale = sm_scale != 0.f ? sm_scale : 0.08838834764831845f;
   c.gpu_pages = const_cast<uint8_t *>(reinterpret_cast<const uint8_t *>(page_pool));
   c.host_pages = nullptr;
+  c.n_gpu_pages = 0x7fffffff;                               // the caller vouches for the ids
+  c.n_host_pages = 0;
   c.page_src = const_cast<int32_t *>(page_ids);
   c.page_mask = const_cast<uint32_t *>(page_masks);
   c.n_pages = const_cast<int32_t *>(n_pages);
-  c.att_part = g_static_partials_addr[dev];
+  c.page_fill = nullptr;                                    // every listed page is already in the pool
+  c.page_desc = nullptr;                                    // the lists are attended in the order given
+  c.att_count = reinterpret_cast<int32_t *>(g_static_partials_addr[dev]);
+  c.att_part = g_static_partials_addr[dev] + counter_floats;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // the array still holds the previous call's counters: they are the one thing that must
+  // start at zero (a memset of library memory, not an allocation)
+  cudaError_t e = cudaMemsetAsync(c.att_count, 0, counter_floats * sizeof(float), st);
+  if (e != cudaSuccess) {
+    fprintf(stderr, "spin_paged_attention_static: clearing the counters failed: %s\n", cudaGetErrorString(e));
+    return SPIN_ERR_CUDA;
+  }
   Batch b{};
   b.n_req = n_sets;
   launch_attention(c, b, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out),
-                   list_stride, reinterpret_cast<cudaStream_t>(cuda_stream), nullptr);
-  cudaError_t e = cudaGetLastError();
+                   list_stride, true, st, nullptr);
+  e = cudaGetLastError();
   if (e != cudaSuccess) {
     fprintf(stderr, "spin_paged_attention_static: launch failed: %s\n", cudaGetErrorString(e));
     return SPIN_ERR_CUDA;

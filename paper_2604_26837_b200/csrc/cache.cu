@@ -77,7 +77,8 @@ k_cache(DevCtx c, Batch bt) {
   int32_t *s_tokens = s_parts + c.max_parts;        // [max_parts]
   int32_t *s_pageoff = s_tokens + c.max_parts;      // [max_parts + 1]
   int32_t *s_missoff = s_pageoff + c.max_parts + 1; // [max_parts] offset into the free list
-  int32_t *s_state = s_missoff + c.max_parts;       // [max_parts]
+  int32_t *s_missbefore = s_missoff + c.max_parts;  // [max_parts] missed pages of earlier partitions
+  int32_t *s_state = s_missbefore + c.max_parts;    // [max_parts]
   int32_t *s_free = s_state + c.max_parts;          // [max_pages]
   uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_free + c.max_pages);   // [max_slots/32]
   __shared__ uint32_t hist[kMaxBuckets + 2];
@@ -96,6 +97,9 @@ k_cache(DevCtx c, Batch bt) {
   int32_t *page_src = c.page_src + pl, *page_slot = c.page_slot + pl;
   int32_t *page_part = c.page_part + pl, *page_pidx = c.page_pidx + pl;
   uint32_t *page_mask = c.page_mask + pl;
+  int32_t *page_fill = c.page_fill + pl;
+  int4 *page_desc = c.page_desc + pl;
+  if (tid == 0) c.att_count[b] = 0;
 
   // ---- step 1: hit/miss classification, page demand ------------------------------------
   uint32_t run_all = 0, run_miss = 0;
@@ -119,6 +123,7 @@ k_cache(DevCtx c, Batch bt) {
     if (r < np) {
       s_pageoff[r] = run_all + ex_a;
       s_missoff[r] = run_miss + ex_m;
+      s_missbefore[r] = run_miss + ex_m;
     }
     run_all += tot_a;
     run_miss += tot_m;
@@ -230,7 +235,7 @@ k_cache(DevCtx c, Batch bt) {
     }
   } else if (tid == 0) sh_demand = demand;
   __syncthreads();
-  if (tid == 0) sh_qbase = sh_demand > 0 ? atomicAdd(c.fetch_count, sh_demand) : 0;
+  if (tid == 0) sh_qbase = (sh_demand > 0 && c.fetch_mode != 0) ? atomicAdd(c.fetch_count, sh_demand) : 0;
   __syncthreads();
   const int qbase = sh_qbase;
 
@@ -250,11 +255,15 @@ k_cache(DevCtx c, Batch bt) {
                                            : ((1u << valid) - 1u);
     page_part[idx] = p;
     page_pidx[idx] = i;
-    if (state == kHit) continue;
+    page_fill[idx] = -1;
+    // work order of the attention kernel: pages that cross the host link first, so that all
+    // of them are requested by the first CTAs and overlap the hits' HBM traffic
+    const int pos = state == kHit ? demand + (s_pageoff[r] - s_missbefore[r]) + i : s_missbefore[r] + i;
+    if (state == kHit) { page_desc[pos] = make_int4(page_src[idx], -1, (int)page_mask[idx], idx); continue; }
     // lookup step 3: Partition Offset -> slice of the CPU page table (pinned host memory)
     const int32_t *off = off_at(c, set, p);
     const int32_t *hp = off ? cpt_at(c, set, *off + i) : nullptr;
-    if (!hp) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; continue; }
+    if (!hp) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
     const int host_page = *hp;
     if (state == kAdmit) {
       const int slot = s_free[s_missoff[r] + i];
@@ -265,13 +274,19 @@ k_cache(DevCtx c, Batch bt) {
       e->ts = top;
       page_src[idx] = phys;
       page_slot[idx] = slot;
-      const int qi = qbase + s_missoff[r] + i;
-      if (qi < c.fetch_cap) c.fetch_queue[qi] = FetchItem{host_page, phys};
-      else dev_error(c, kErrBounds);
+      if (c.fetch_mode == 0) {
+        page_fill[idx] = host_page;               // the attention kernel brings it in
+      } else {
+        const int qi = qbase + s_missoff[r] + i;
+        if (qi < c.fetch_cap) c.fetch_queue[qi] = FetchItem{host_page, phys};
+        else dev_error(c, kErrBounds);
+      }
+      page_desc[pos] = make_int4(phys, page_fill[idx], (int)page_mask[idx], idx);
       ++my_admit;
     } else {
       page_src[idx] = ~host_page;
       page_slot[idx] = -1;
+      page_desc[pos] = make_int4(~host_page, -1, (int)page_mask[idx], idx);
       ++my_bypass;
     }
   }
@@ -284,6 +299,8 @@ k_cache(DevCtx c, Batch bt) {
     page_src[idx] = c.tail_phys[(size_t)set * c.tail_cap + j];
     page_mask[idx] = j == st.tail_pages - 1 ? ((1u << st.tail_len) - 1u) : 0xffffu;
     page_slot[idx] = -2;
+    page_fill[idx] = -1;
+    page_desc[idx] = make_int4(page_src[idx], -1, (int)page_mask[idx], idx);
     page_part[idx] = -1;
     page_pidx[idx] = j;
   }
@@ -327,7 +344,7 @@ k_fetch(DevCtx c) {
 }  // namespace
 
 size_t cache_smem_bytes(const DevCtx &c) {
-  return (size_t)(5 * c.max_parts + 1 + c.max_pages) * 4 + (size_t)((c.max_slots + 31) / 32) * 4 + 16;
+  return (size_t)(6 * c.max_parts + 1 + c.max_pages) * 4 + (size_t)((c.max_slots + 31) / 32) * 4 + 16;
 }
 
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count, Prof *prof) {
@@ -339,6 +356,7 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count,
   }
   k_cache<<<b.n_req * c.Hkv, kCacheThreads, smem, st>>>(c, b);
   prof_mark(prof, st, kProfCache);
+  if (c.fetch_mode == 0) return 1;
   k_fetch<<<sm_count * 4, 256, 0, st>>>(c);
   prof_mark(prof, st, kProfFetch);
   return 2;

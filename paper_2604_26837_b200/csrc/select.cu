@@ -27,6 +27,44 @@ __device__ __forceinline__ void unpack8(uint4 raw, float *f) {
   }
 }
 
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// Score of one entry for this lane's 8 channels, all G heads; the 16 lanes of the row are
+// combined by the caller-visible butterfly.  For min/max summaries max(q*min, q*max) equals
+// q * (q >= 0 ? max : min) exactly (min <= max and the products are exact), so the operand is
+// picked with one bitwise blend per channel pair on the packed bf16 words (masks precomputed
+// per head) instead of two multiplies and a max per channel.
+template <int G, bool MINMAX>
+__device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, const float (&qf)[G][8],
+                                             const uint32_t (&qsel)[G][4], uint32_t row_mask) {
+  const uint32_t a[4] = {lo.x, lo.y, lo.z, lo.w}, m[4] = {hi.x, hi.y, hi.z, hi.w};
+  float tot = 0.f;
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t w = MINMAX ? ((m[j] & qsel[g][j]) | (a[j] & ~qsel[g][j])) : a[j];
+      x[2 * j] = __uint_as_float(w << 16);
+      x[2 * j + 1] = __uint_as_float(w & 0xffff0000u);
+    }
+    float s = qf[g][0] * x[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) s = fmaf(qf[g][i], x[i], s);     // exact product, one rounding: s + q*x
+    s = s + __shfl_xor_sync(row_mask, s, 1);
+    s = s + __shfl_xor_sync(row_mask, s, 2);
+    s = s + __shfl_xor_sync(row_mask, s, 4);
+    s = s + __shfl_xor_sync(row_mask, s, 8);
+    tot = g == 0 ? s : tot + s;
+  }
+  return tot + 0.0f;                              // -0.0 -> +0.0
+}
+
 template <int G, bool MINMAX>
 __global__ void __launch_bounds__(256)
 k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
@@ -39,49 +77,42 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
   const int e0 = blockIdx.x * seg_entries;
   if (e0 >= n_cand) return;
   const int seg = c.dir_sumseg[(size_t)set * c.dir_sum + blockIdx.x];
-  if (seg < 0) { if (threadIdx.x == 0) dev_error(c, 1u); return; }
+  if (seg < 0) { if (threadIdx.x == 0) dev_error(c, kErrBounds); return; }
   const int lane16 = threadIdx.x & 15, grp = threadIdx.x >> 4;
   // the two 16-lane rows of a warp may leave the loop at different times: each shuffles
   // only among its own lanes
   const uint32_t row_mask = 0xffffu << (threadIdx.x & 16);
 
   float qf[G][8];
+  uint32_t qsel[G][4];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     const uint4 raw = *reinterpret_cast<const uint4 *>(
         q + ((size_t)i_req * c.Hq + head * G + g) * kHeadDim + lane16 * 8);
     unpack8(raw, qf[g]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      qsel[g][j] = (qf[g][2 * j] >= 0.f ? 0x0000ffffu : 0u) | (qf[g][2 * j + 1] >= 0.f ? 0xffff0000u : 0u);
   }
   const int n_here = min(seg_entries, n_cand - e0);
   constexpr int kEntry = MINMAX ? 2 * kRowBytes : kRowBytes;
   const uint8_t *base = c.summaries + ((size_t)seg << c.sum_shift) * kEntry + lane16 * 16;
   float *out = c.scores + (size_t)b * c.max_cand + e0;
 
-#pragma unroll 4
-  for (int e = grp; e < n_here; e += 16) {
-    float a[8], mx[8];
-    unpack8(*reinterpret_cast<const uint4 *>(base + (size_t)e * kEntry), a);
-    if (MINMAX) unpack8(*reinterpret_cast<const uint4 *>(base + (size_t)e * kEntry + kRowBytes), mx);
-    float tot = 0.f;
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float s;
-      if (MINMAX) {
-        s = fmaxf(qf[g][0] * a[0], qf[g][0] * mx[0]);
-#pragma unroll
-        for (int i = 1; i < 8; ++i) s = s + fmaxf(qf[g][i] * a[i], qf[g][i] * mx[i]);
-      } else {
-        s = qf[g][0] * a[0];
-#pragma unroll
-        for (int i = 1; i < 8; ++i) s = s + qf[g][i] * a[i];
-      }
-      s = s + __shfl_xor_sync(row_mask, s, 1);
-      s = s + __shfl_xor_sync(row_mask, s, 2);
-      s = s + __shfl_xor_sync(row_mask, s, 4);
-      s = s + __shfl_xor_sync(row_mask, s, 8);
-      tot = g == 0 ? s : tot + s;
+  // two entries per half-warp and iteration, all their loads issued before any arithmetic
+  for (int e = grp; e < n_here; e += 32) {
+    const bool two = e + 16 < n_here;
+    const uint4 z = make_uint4(0, 0, 0, 0);
+    const uint4 a0 = ld_stream16(base + (size_t)e * kEntry);
+    const uint4 m0 = MINMAX ? ld_stream16(base + (size_t)e * kEntry + kRowBytes) : z;
+    const uint4 a1 = two ? ld_stream16(base + (size_t)(e + 16) * kEntry) : z;
+    const uint4 m1 = (MINMAX && two) ? ld_stream16(base + (size_t)(e + 16) * kEntry + kRowBytes) : z;
+    const float s0 = score_entry<G, MINMAX>(a0, m0, qf, qsel, row_mask);
+    if (lane16 == 0) out[e] = s0;
+    if (two) {
+      const float s1 = score_entry<G, MINMAX>(a1, m1, qf, qsel, row_mask);
+      if (lane16 == 0) out[e + 16] = s1;
     }
-    if (lane16 == 0) out[e] = tot + 0.0f;       // -0.0 -> +0.0
   }
 }
 

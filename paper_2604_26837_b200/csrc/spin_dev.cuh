@@ -22,7 +22,7 @@ constexpr int kMaxBuckets = 64;
 enum : int { kKindPage = 0, kKindToken = 1, kKindCluster = 2 };
 // sticky device error bits (same values as SPIN_DEV_ERR_* of the public header)
 constexpr unsigned kErrBounds = 1u, kErrPageList = 2u, kErrTimeout = 4u;
-constexpr int kChunkPages = 16;                             // pages per attention split
+constexpr int kChunkPages = 8;                              // pages per attention split
 
 // Per-set scalars (device resident, updated only by kernels).
 struct SetState {
@@ -63,6 +63,7 @@ struct DevCtx {
   int32_t max_cand;             // score stride per batch set
   float sm_scale;
   // pools
+  int32_t n_gpu_pages, n_host_pages;   // pool sizes, for range checks
   uint8_t *gpu_pages;           // HBM KV pages (cache slots + tails)
   uint8_t *host_pages;          // pinned host KV pages (device-visible address)
   uint8_t *summaries;           // summary segments (64 KiB each)
@@ -86,6 +87,8 @@ struct DevCtx {
   int32_t *n_parts;             // [b]
   int32_t *page_src;            // [b][max_pages+tail_cap] >=0 GPU page, <0 ~host page
   uint32_t *page_mask;          // [b][...]
+  int32_t *page_fill;           // [b][...] host page to copy into page_src first, or -1
+  int4 *page_desc;              // [b][...] attention's work list, misses first: {page_src, page_fill, mask, list index}
   int32_t *page_slot;           // [b][...] set-local slot / -1 bypass / -2 tail
   int32_t *page_part;           // [b][...] owning partition (-1 tail)
   int32_t *page_pidx;           // [b][...]
@@ -94,7 +97,9 @@ struct DevCtx {
   int32_t *fetch_count;
   int32_t fetch_cap;
   float *att_part;              // split-K partials [b][max_chunks][G][kHeadDim + 2]
+  int32_t *att_count;           // [b] chunks of the set that have finished (zero before attention)
   int32_t max_chunks;
+  int32_t fetch_mode;           // 0: misses are fetched by the attention kernel; 1: by k_fetch
   Counters *counters;
 };
 
@@ -174,6 +179,6 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int m
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count, Prof *prof);
 size_t cache_smem_bytes(const DevCtx &c);
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
-                     __nv_bfloat16 *out, int max_pages_hint, cudaStream_t st, Prof *prof);
+                     __nv_bfloat16 *out, int max_pages_hint, bool may_be_empty, cudaStream_t st, Prof *prof);
 
 }  // namespace spin
