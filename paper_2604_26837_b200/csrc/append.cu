@@ -83,6 +83,8 @@ k_append_edge(DevCtx c, AppendEdgeArgs a, const __nv_bfloat16 *__restrict__ k,
               const __nv_bfloat16 *__restrict__ v, int n_new) {
   __shared__ __align__(16) __nv_bfloat16 krows[kPageTokens][kHeadDim];
   const int head = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
+  pdl_launch_next();
+  pdl_wait_prev();
   const int set = set_index(c, a.req[i], a.layer, head);
   const int r = tid >> 4, piece = tid & 15;
   SetState st = c.state[set];
@@ -215,7 +217,7 @@ int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 
 
 int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int n_new, cudaStream_t st, Prof *prof) {
-  k_append_edge<<<dim3(c.Hkv, a.n_req), 256, 0, st>>>(c, a, k, v, n_new);
+  launch_pdl(k_append_edge, dim3(c.Hkv, a.n_req), dim3(256), 0, st, 1, c, a, k, v, n_new);
   prof_mark(prof, st, kProfAppend);
   return 1;
 }

@@ -152,6 +152,8 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   __shared__ float sh[kAttnWarps][G][kPartStride];
   __shared__ int sh_last;
   const int b = blockIdx.x, chunk = blockIdx.y;       // chunk-major launch order: chunk 0 of every set first
+  pdl_launch_next();
+  pdl_wait_prev();
   const int np = c.n_pages[b];
   const int first = chunk * kChunkPages;
   if (first >= np) return;
@@ -332,7 +334,7 @@ void launch_attn_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, __nv
     cudaFuncSetAttribute(k_attn<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     configured = true;
   }
-  k_attn<G><<<grid, kAttnWarps * 32, smem, st>>>(c, b, q, out);
+  launch_pdl(k_attn<G>, grid, dim3(kAttnWarps * 32), (size_t)smem, st, 1, c, b, q, out);
 }
 
 }  // namespace

@@ -21,7 +21,7 @@ namespace spin {
 
 namespace {
 
-constexpr int kCacheThreads = 256;
+constexpr int kCacheThreads = 512;
 enum : int { kHit = 0, kAdmit = 1, kBypass = 2 };
 
 __device__ __forceinline__ uint32_t block_scan256(uint32_t v, uint32_t *wsum, uint32_t *total) {
@@ -83,11 +83,14 @@ k_cache(DevCtx c, Batch bt) {
   uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_free + c.max_pages);   // [max_slots/32]
   __shared__ uint32_t hist[kMaxBuckets + 2];
   __shared__ uint32_t wsum[33];
+  __shared__ int32_t s_hostpage[kCacheThreads];      // CPU page ids of the first missed pages
   __shared__ int sh_x, sh_demand, sh_evicted, sh_qbase, sh_admit_pages,
       sh_bypass_pages;
 
   const int b = blockIdx.x, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
+  pdl_launch_next();
+  pdl_wait_prev();
   const SetState st = c.state[set];
   const int S = st.slots, n = c.n_buckets, t = st.step;
   const int top = min(t, n - 1);
@@ -147,31 +150,57 @@ k_cache(DevCtx c, Batch bt) {
   for (int i = tid; i < kMaxBuckets + 2; i += kCacheThreads) hist[i] = 0;
   __syncthreads();
 
+  // Retrieve step 3, started early: the Partition Offset / CPU page table entries of the
+  // missed pages live in pinned host memory, two dependent reads over the host link.  They
+  // are issued here and consumed after the table scans below, which hides their latency.
+  int early_i = 0, early_off = -1, early_host = -1;
+  if (tid < demand && np > 0) {
+    const int r = owner_of(s_missbefore, np, tid);
+    early_i = tid - s_missbefore[r];
+    const int32_t *off = off_at(c, set, s_parts[r]);
+    if (off) early_off = *off;
+  }
+
   // ---- step 2: one scan of the GPU page table: promote, demote, histogram ---------------
-  for (int s = tid; s < S; s += kCacheThreads) {
-    GptEntry *e = gpt_at(c, set, s);
-    if (!e) { dev_error(c, kErrBounds); continue; }
-    const int4 raw = *reinterpret_cast<const int4 *>(e);
-    const int part = raw.x, phys = raw.y, pidx = raw.z;
-    int ts = raw.w;
-    if (c.trace) {
-      c.evict_trace[((size_t)set * c.max_slots + s) * 2] = -1;
-      c.evict_trace[((size_t)set * c.max_slots + s) * 2 + 1] = -1;
+  for (int base = 0; base < S; base += kCacheThreads) {
+    const int s = base + tid;
+    int bucket = -2;                                  // -2: nothing to count (hit slot or no slot)
+    GptEntry *e = s < S ? gpt_at(c, set, s) : nullptr;
+    if (s < S && !e) dev_error(c, kErrBounds);
+    if (e) {
+      const int4 raw = *reinterpret_cast<const int4 *>(e);
+      const int part = raw.x, phys = raw.y, pidx = raw.z;
+      int ts = raw.w;
+      if (c.trace) {
+        c.evict_trace[((size_t)set * c.max_slots + s) * 2] = -1;
+        c.evict_trace[((size_t)set * c.max_slots + s) * 2 + 1] = -1;
+      }
+      if (part < 0) {
+        bucket = -1;
+      } else {
+        const int r = find_sorted(s_parts, np, part);
+        if (r >= 0) {
+          atomicOr(&s_hit[s >> 5], 1u << (s & 31));
+          if (ts != top) e->ts = top;
+          const int idx = s_pageoff[r] + pidx;
+          page_src[idx] = phys;
+          page_slot[idx] = s;
+        } else {
+          if (t > n - 1 && ts > 0) { --ts; e->ts = ts; }
+          bucket = ts;
+        }
+      }
     }
-    if (part < 0) { atomicAdd(&hist[0], 1u); continue; }
-    const int r = find_sorted(s_parts, np, part);
-    if (r >= 0) {
-      atomicOr(&s_hit[s >> 5], 1u << (s & 31));
-      if (ts != top) e->ts = top;
-      const int idx = s_pageoff[r] + pidx;
-      page_src[idx] = phys;
-      page_slot[idx] = s;
-    } else {
-      if (t > n - 1 && ts > 0) { --ts; e->ts = ts; }
-      atomicAdd(&hist[ts + 1], 1u);
-    }
+    // slots of one generation share a timestamp: one lane per distinct bucket adds the count
+    const uint32_t same = __match_any_sync(0xffffffffu, bucket);
+    if (bucket >= -1 && (tid & 31) == __ffs(same) - 1) atomicAdd(&hist[bucket + 1], (uint32_t)__popc(same));
   }
   __syncthreads();
+
+  if (early_off >= 0) {
+    const int32_t *hp = cpt_at(c, set, early_off + early_i);
+    if (hp) early_host = *hp;
+  }
 
   // ---- step 3: threshold and eviction; free slots in ascending order --------------------
   if (tid == 0) {
@@ -221,6 +250,8 @@ k_cache(DevCtx c, Batch bt) {
   }
   __syncthreads();
 
+  s_hostpage[tid] = early_host;
+
   // ---- step 4: admission (whole partitions; what does not fit is bypassed) --------------
   if (demand > (int)run_free) {
     if (tid == 0) {
@@ -261,10 +292,15 @@ k_cache(DevCtx c, Batch bt) {
     const int pos = state == kHit ? demand + (s_pageoff[r] - s_missbefore[r]) + i : s_missbefore[r] + i;
     if (state == kHit) { page_desc[pos] = make_int4(page_src[idx], -1, (int)page_mask[idx], idx); continue; }
     // lookup step 3: Partition Offset -> slice of the CPU page table (pinned host memory)
-    const int32_t *off = off_at(c, set, p);
-    const int32_t *hp = off ? cpt_at(c, set, *off + i) : nullptr;
+    const int mi = s_missbefore[r] + i;
+    int host_page = mi < kCacheThreads ? s_hostpage[mi] : -1;
+    const int32_t *hp = &host_page;
+    if (host_page < 0) {                       // beyond the early batch (or it failed): look up now
+      const int32_t *off = off_at(c, set, p);
+      hp = off ? cpt_at(c, set, *off + i) : nullptr;
+      if (hp) host_page = *hp;
+    }
     if (!hp) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
-    const int host_page = *hp;
     if (state == kAdmit) {
       const int slot = s_free[s_missoff[r] + i];
       GptEntry *e = gpt_at(c, set, slot);
@@ -354,7 +390,7 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count,
     cudaFuncSetAttribute(k_cache, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  k_cache<<<b.n_req * c.Hkv, kCacheThreads, smem, st>>>(c, b);
+  launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b);
   prof_mark(prof, st, kProfCache);
   if (c.fetch_mode == 0) return 1;
   k_fetch<<<sm_count * 4, 256, 0, st>>>(c);

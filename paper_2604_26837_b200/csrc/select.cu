@@ -12,7 +12,11 @@
 // select on order-preserving keys followed by one ordered compaction, and emits them in
 // ascending index order.  For token-granular selection it also folds the chosen tokens into
 // their pages with a 16-bit token mask per page.
+#include <cooperative_groups.h>
+
 #include "spin_dev.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace spin {
 
@@ -70,6 +74,8 @@ __global__ void __launch_bounds__(256)
 k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
   const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
+  pdl_launch_next();
+  pdl_wait_prev();
   if (blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *c.fetch_count = 0;   // new step, new miss queue
   const SetState st = c.state[set];
   const int n_cand = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
@@ -151,42 +157,69 @@ __device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t *wsum, uint3
   return res;
 }
 
+// One thread-block cluster per set: the candidates are cut into one contiguous slice per CTA
+// (keys kept in shared memory), every radix pass builds per-CTA histograms that all CTAs sum
+// through distributed shared memory, and the ordered compaction uses the lower-ranked CTAs'
+// counts as its offset.  A cluster of one CTA is the small-set case (a few thousand pages);
+// token-granular selection over 64K+ keys uses 8 CTAs.  Cluster barriers are hardware
+// barriers (no flag spinning); every CTA of a cluster executes the same number of them.
 __global__ void __launch_bounds__(kTopkThreads)
-k_topk(DevCtx c, Batch bt) {
-  __shared__ uint32_t hist[256];
+k_topk(DevCtx c, Batch bt, int keys_cap) {
+  extern __shared__ uint32_t s_keys[];                 // [keys_cap] order-preserving keys of this slice
+  __shared__ uint32_t hist[256];                       // this CTA's histogram (read remotely)
+  __shared__ uint32_t ghist[256];                      // cluster-wide histogram
   __shared__ uint32_t wsum[33];
+  __shared__ uint32_t cnt[2];                          // this CTA's (above threshold, equal) counts
   __shared__ uint32_t sh_prefix, sh_remaining;
-  const int b = blockIdx.x, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const int b = blockIdx.x / C, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
+  pdl_launch_next();
+  pdl_wait_prev();
   const SetState st = c.state[set];
   const int n = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
   const int k = min(c.topk, n);
   const float *scores = c.scores + (size_t)b * c.max_cand;
   int32_t *sel = c.sel_ids + (size_t)b * c.max_sel;
+  const int per = (n + C - 1) / C;
+  const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
+  const bool cached = m <= keys_cap;
 
-  if (tid == 0) {
+  if (tid == 0 && rank == 0) {
     c.n_sel[b] = k;
     atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
   }
+  if (cached)
+    for (int i = tid; i < m; i += kTopkThreads) s_keys[i] = order_key(scores[lo + i]);
+  __syncthreads();
+  auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(scores[lo + i]); };
+
   if (k == n) {
-    for (int i = tid; i < n; i += kTopkThreads) sel[i] = i;
+    for (int i = tid; i < m; i += kTopkThreads) sel[lo + i] = lo + i;
   } else {
     // ---- radix select: key of the k-th best candidate --------------------------------
     uint32_t prefix = 0, mask = 0, remaining = k;
     for (int shift = 24; shift >= 0; shift -= 8) {
       if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      for (int i = tid; i < n; i += kTopkThreads) {
-        const uint32_t key = order_key(scores[i]);
+      for (int i = tid; i < m; i += kTopkThreads) {
+        const uint32_t key = key_at(i);
         if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
-      __syncthreads();
+      cluster.sync();                                   // every CTA's histogram is complete
+      if (tid < 256) {
+        uint32_t tot = 0;
+        for (int r = 0; r < C; ++r) tot += cluster.map_shared_rank(hist, r)[tid];
+        ghist[tid] = tot;
+      }
+      cluster.sync();                                   // remote reads done before hist is reused
       if (tid < 32) {
         // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the
         // top reaches `remaining`
         uint32_t loc[8], sum = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { loc[j] = hist[255 - 8 * tid - j]; sum += loc[j]; }
+        for (int j = 0; j < 8; ++j) { loc[j] = ghist[255 - 8 * tid - j]; sum += loc[j]; }
         uint32_t inc = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -212,13 +245,36 @@ k_topk(DevCtx c, Batch bt) {
       mask |= 255u << shift;
     }
     const uint32_t thr = prefix, need_eq = remaining;
-    // ---- ordered compaction: everything above thr, plus the first need_eq equal to it --
+    // ---- counts of this slice, offsets from the lower-ranked slices ---------------------
+    if (tid < 2) cnt[tid] = 0;
+    __syncthreads();
+    {
+      uint32_t gt = 0, eq = 0;
+      for (int i = tid; i < m; i += kTopkThreads) {
+        const uint32_t key = key_at(i);
+        gt += key > thr;
+        eq += key == thr;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        gt += __shfl_xor_sync(0xffffffffu, gt, o);
+        eq += __shfl_xor_sync(0xffffffffu, eq, o);
+      }
+      if ((tid & 31) == 0) { atomicAdd(&cnt[0], gt); atomicAdd(&cnt[1], eq); }
+    }
+    cluster.sync();
     uint32_t run_gt = 0, run_eq = 0;
-    for (int base = 0; base < n; base += kTopkThreads) {
+    for (int r = 0; r < rank; ++r) {
+      const uint32_t *rc = cluster.map_shared_rank(cnt, r);
+      run_gt += rc[0];
+      run_eq += rc[1];
+    }
+    // ---- ordered compaction: everything above thr, plus the first need_eq equal to it --
+    for (int base = 0; base < m; base += kTopkThreads) {
       const int i = base + tid;
       uint32_t gt = 0, eq = 0;
-      if (i < n) {
-        const uint32_t key = order_key(scores[i]);
+      if (i < m) {
+        const uint32_t key = key_at(i);
         gt = key > thr;
         eq = key == thr;
       }
@@ -226,17 +282,18 @@ k_topk(DevCtx c, Batch bt) {
       const uint32_t ex = block_scan(gt | (eq << 16), wsum, &total);
       const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
       if (gt || (eq && eq_before < need_eq))
-        sel[gt_before + min(eq_before, need_eq)] = i;
+        sel[gt_before + min(eq_before, need_eq)] = lo + i;
       run_gt += total & 0xffffu;
       run_eq += total >> 16;
     }
   }
-  __syncthreads();
+  cluster.sync();            // selections of all slices are written; nobody reads remote smem after this
+  if (rank != 0) return;
 
-  // ---- candidates -> partitions of the cache manager -------------------------------------
+  // ---- candidates -> partitions of the cache manager (first CTA of the cluster) ----------
   int32_t *parts = c.parts + (size_t)b * c.max_parts;
   if (c.kind != kKindToken) {
-    for (int i = tid; i < k; i += kTopkThreads) parts[i] = sel[i];
+    for (int i = tid; i < k; i += kTopkThreads) parts[i] = __ldcg(sel + i);
     if (tid == 0) c.n_parts[b] = k;
     return;
   }
@@ -249,15 +306,15 @@ k_topk(DevCtx c, Batch bt) {
     uint32_t first = 0;
     int tok = 0;
     if (i < k) {
-      tok = sel[i];
-      first = (i == 0) || ((sel[i - 1] >> 4) != (tok >> 4));
+      tok = __ldcg(sel + i);
+      first = (i == 0) || ((__ldcg(sel + i - 1) >> 4) != (tok >> 4));
     }
     uint32_t total;
     const uint32_t ex = block_scan(first, wsum, &total);
     if (i < k) {
-      const uint32_t rank = run + ex + first - 1;
-      if (first) parts[rank] = tok >> 4;
-      atomicOr(&pmask[rank], 1u << (tok & 15));
+      const uint32_t rank_ = run + ex + first - 1;
+      if (first) parts[rank_] = tok >> 4;
+      atomicOr(&pmask[rank_], 1u << (tok & 15));
     }
     run += total;
   }
@@ -266,8 +323,8 @@ k_topk(DevCtx c, Batch bt) {
 
 template <int G>
 void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, dim3 grid, cudaStream_t st) {
-  if (c.kind == kKindPage) k_score<G, true><<<grid, 256, 0, st>>>(c, b, q);
-  else k_score<G, false><<<grid, 256, 0, st>>>(c, b, q);
+  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(256), 0, st, 1, c, b, q);
+  else launch_pdl(k_score<G, false>, grid, dim3(256), 0, st, 1, c, b, q);
 }
 
 }  // namespace
@@ -285,7 +342,17 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int m
     default: launch_score_g<8>(c, b, q, grid, st); break;
   }
   prof_mark(prof, st, kProfScore);
-  k_topk<<<n_sets, kTopkThreads, 0, st>>>(c, b);
+  {
+    // cluster size from the largest candidate count: slices of at most 8192 keys stay in smem
+    int C = 1;
+    while (C < 8 && (max_cand + C - 1) / C > 8192) C *= 2;
+    int keys_cap = (max_cand + C - 1) / C;
+    if (keys_cap > 16384) keys_cap = 0;                  // too many for shared memory: re-read from L2
+    static int smem_set = 0;
+    const int smem = keys_cap * 4;
+    if (smem > smem_set) { cudaFuncSetAttribute(k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); smem_set = smem; }
+    launch_pdl(k_topk, dim3(n_sets * C), dim3(kTopkThreads), (size_t)smem, st, C, c, b, keys_cap);
+  }
   prof_mark(prof, st, kProfTopk);
   return 2;
 }

@@ -141,6 +141,15 @@ __device__ __forceinline__ uint8_t *summary_at(const DevCtx &c, int set, int e) 
                  : c.summaries + (((size_t)seg << c.sum_shift) + (e & ((1 << c.sum_shift) - 1))) *
                                      (size_t)c.sum_entry_bytes;
 }
+// Programmatic dependent launch: the kernels of a decode step are launched back to back with
+// the "programmatic stream serialization" attribute, so a kernel's CTAs may become resident
+// while the previous kernel drains.  pdl_launch_next() lets the next kernel start launching;
+// pdl_wait_prev() blocks until the previous kernel has completed and its writes are visible.
+// Every kernel launched this way calls pdl_wait_prev() before it reads or writes anything
+// another kernel touches.
+__device__ __forceinline__ void pdl_launch_next() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prev() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ const uint8_t *page_ptr(const DevCtx &c, int src) {
   return src >= 0 ? c.gpu_pages + (size_t)src * kPageBytes : c.host_pages + (size_t)(~src) * kPageBytes;
 }
@@ -158,6 +167,32 @@ struct Prof {
   void mark(cudaStream_t st, int kernel);
 };
 inline void prof_mark(Prof *p, cudaStream_t st, int kernel) { if (p && p->on) p->mark(st, kernel); }
+
+// Launch with programmatic stream serialization (and optionally a cluster size).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              int cluster_x, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[na].val.programmaticStreamSerializationAllowed = 1;
+  ++na;
+  if (cluster_x > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = cluster_x;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 // ---- kernel launchers (each returns the number of kernels it launched) -----------------
 struct AppendEdgeArgs {     // one (request) per entry; all its kv heads are processed
