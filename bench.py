@@ -265,8 +265,7 @@ def main():
 
     def one_step(s):
         for l in range(L):
-            run.append(l, k_all[s, l], v_all[s, l], stream)
-            run.decode(l, q_all[s, l], out, stream)
+            run.step(l, k_all[s, l], v_all[s, l], q_all[s, l], out, stream)
 
     def timed_steps(n, flush_l2=True):
         evs = []
@@ -328,8 +327,7 @@ def main():
                 stream.synchronize()
                 t0 = time.perf_counter()
                 for l in range(L):
-                    run.append(l, kh[i, l], vh[i, l], stream)
-                    run.decode(l, qh[i, l], oh, stream)
+                    run.step(l, kh[i, l], vh[i, l], qh[i, l], oh, stream)
                 stream.synchronize()                       # the result is read on the host
                 _ = float(oh[0, 0, 0])
                 if i >= Wm:

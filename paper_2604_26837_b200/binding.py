@@ -23,7 +23,7 @@ PAGE_BYTES = 8192
 
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open",
            "spin_request_close", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
-           "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
+           "spin_decode_step_append", "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
            "spin_debug_read_page", "spin_paged_attention_static", "spin_last_error",
            "spin_version"]
 KERNEL_NAMES = ["append", "score", "topk", "cache", "fetch", "attn_split", "attn_merge"]
@@ -104,6 +104,7 @@ def load() -> C.CDLL:
     lib.spin_append_kv.argtypes = [vp, i32, i32, vp, vp, i64, vp, vp, vp]
     lib.spin_append_kv_batch.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
     lib.spin_decode_step.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
+    lib.spin_decode_step_append.argtypes = [vp, i32, _I32P, i32, vp, vp, vp, vp, vp]
     lib.spin_stats.argtypes = [vp, C.POINTER(spin_stats_t)]
     lib.spin_profile.argtypes = [vp, i32]
     lib.spin_profile_read.argtypes = [vp, C.POINTER(spin_profile_t)]
@@ -230,6 +231,11 @@ class Spin:
         arr = (C.c_int32 * len(req_ids))(*req_ids)
         self._ck(self.lib.spin_decode_step(self.h, layer, arr, len(req_ids), _ptr(q), _ptr(out),
                                            _stream_ptr(stream)))
+
+    def decode_step_append(self, layer: int, req_ids: Sequence[int], k_new, v_new, q, out, stream=None):
+        arr = (C.c_int32 * len(req_ids))(*req_ids)
+        self._ck(self.lib.spin_decode_step_append(self.h, layer, arr, len(req_ids), _ptr(k_new),
+                                                  _ptr(v_new), _ptr(q), _ptr(out), _stream_ptr(stream)))
 
     def stats(self) -> dict:
         s = spin_stats_t()

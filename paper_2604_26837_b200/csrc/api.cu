@@ -169,6 +169,9 @@ struct spin_ctx {
   uint64_t launches = 0;
   size_t dir_bytes_in_use = 0;
   Prof prof;
+  cudaStream_t side = nullptr;       // runs the decode-time append next to Select
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool join_pending = false;
 };
 
 namespace {
@@ -649,6 +652,12 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   ctx->sum_segs.init(g.n_sum_segs);
   ctx->reqs.resize((size_t)cfg->max_requests);
   ctx->sets.resize((size_t)g.n_sets);
+  if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    cudaGetLastError();
+    ctx->side = nullptr;                // no side stream: appends simply stay on the caller's stream
+  }
   *out = ctx;
   return SPIN_OK;
 }
@@ -661,6 +670,9 @@ int spin_destroy(spin_ctx *ctx) {
     delete[] ctx->prof.ev;
     delete[] ctx->prof.id;
   }
+  if (ctx->side) cudaStreamDestroy(ctx->side);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   if (ctx->host_base) cudaFreeHost(ctx->host_base);
   delete ctx;
   return SPIN_OK;
@@ -836,27 +848,65 @@ int spin_append_kv_batch(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, i
   return SPIN_OK;
 }
 
-int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32_t n_req,
-                     const void *q, void *out, void *cuda_stream) {
-  if (!ctx) return SPIN_ERR_INVALID;
+// One decode step, optionally preceded by the append of one token per request.  When the
+// append cannot change what Select sees (no page is completed by it), it runs on the
+// context's side stream concurrently with scoring and top-k and is joined before the cache
+// manager, which hides its host-link write latency.
+static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32_t n_req, const void *k,
+                     const void *v, const void *q, void *out, cudaStream_t st) {
   if (!req_ids || !q || !out || n_req < 1 || n_req > ctx->cfg.max_requests) return fail(ctx, SPIN_ERR_INVALID, "bad batch arguments");
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const bool with_append = k != nullptr;
+  if (with_append && !v) return fail(ctx, SPIN_ERR_INVALID, "k without v");
+  const bool cluster = ctx->cfg.partition_kind == SPIN_PART_CLUSTER_CENTROID;
   Batch b{};
   b.n_req = n_req;
   b.layer = layer;
-  int64_t max_cand = 0, max_pages = 0;
-  bool may_be_empty = false;
+  bool completes_page = false;
   for (int i = 0; i < n_req; ++i) {
     int rc = validate_req_layer(ctx, req_ids[i], layer);
     if (rc) return rc;
     for (int j = 0; j < i; ++j) if (req_ids[j] == req_ids[i]) return fail(ctx, SPIN_ERR_INVALID, "request %d listed twice", req_ids[i]);
     b.req[i] = req_ids[i];
+    const LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
+    if (with_append && cluster && !L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req_ids[i]);
+    if (with_append && L.n_tokens % kPageTokens == 0) completes_page = true;     // a new page starts
+  }
+  if (with_append) {
+    const bool parallel = !completes_page && !ctx->prof.on && ctx->side != nullptr;
+    cudaStream_t as = parallel ? ctx->side : st;
+    if (parallel) {
+      CK(cudaEventRecord(ctx->ev_fork, st));
+      CK(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    }
+    AppendEdgeArgs a{};
+    a.n_req = n_req;
+    a.layer = layer;
+    for (int i = 0; i < n_req; ++i) {
+      a.req[i] = req_ids[i];
+      LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
+      int rc = cluster ? grow_cluster_tail(ctx, req_ids[i], layer, 1, as) : grow_paged(ctx, req_ids[i], layer, L.n_tokens + 1, as);
+      if (rc) return rc;
+    }
+    const __nv_bfloat16 *kk = reinterpret_cast<const __nv_bfloat16 *>(k), *vv = reinterpret_cast<const __nv_bfloat16 *>(v);
+    if (!is_device_ptr(k)) {
+      const size_t bytes = (size_t)n_req * ctx->cfg.num_kv_heads * kRowBytes;
+      CK(cudaMemcpyAsync(ctx->stage_k, k, bytes, cudaMemcpyHostToDevice, as));
+      CK(cudaMemcpyAsync(ctx->stage_v, v, bytes, cudaMemcpyHostToDevice, as));
+      kk = ctx->stage_k;
+      vv = ctx->stage_v;
+    }
+    prof_mark(&ctx->prof, as, -1);
+    ctx->launches += launch_append_edge(ctx->d, a, kk, vv, 1, as, &ctx->prof);
+    if (parallel) CK(cudaEventRecord(ctx->ev_join, ctx->side));
+    ctx->join_pending = parallel;
+  }
+  int64_t max_cand = 0, max_pages = 0;
+  bool may_be_empty = false;
+  for (int i = 0; i < n_req; ++i) {
     LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
     const int64_t cand = ctx->cfg.partition_kind == SPIN_PART_TOKEN_DOT ? (int64_t)L.n_partitions * kPageTokens : L.n_partitions;
     max_cand = std::max(max_cand, cand);
-    int64_t pages = ctx->cfg.partition_kind == SPIN_PART_CLUSTER_CENTROID
-                        ? ctx->g.max_pages
-                        : std::min<int64_t>(ctx->cfg.topk, L.n_partitions);
+    int64_t pages = cluster ? ctx->g.max_pages : std::min<int64_t>(ctx->cfg.topk, L.n_partitions);
     max_pages = std::max(max_pages, pages + L.tail_pages);
     may_be_empty = may_be_empty || L.n_tokens == 0;
     L.last_batch_pos = i;
@@ -869,11 +919,29 @@ int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   if (!out_dev) od = ctx->stage_out;
   prof_mark(&ctx->prof, st, -1);
   ctx->launches += launch_select(ctx->d, b, qd, (int)max_cand, st, &ctx->prof);
+  if (ctx->join_pending) {
+    CK(cudaStreamWaitEvent(st, ctx->ev_join, 0));
+    ctx->join_pending = false;
+  }
   ctx->launches += launch_cache(ctx->d, b, st, ctx->sm_count, &ctx->prof);
   ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, may_be_empty, st, &ctx->prof);
   if (!out_dev) CK(cudaMemcpyAsync(out, ctx->stage_out, qbytes, cudaMemcpyDeviceToHost, st));
   CK(cudaGetLastError());
   return SPIN_OK;
+}
+
+int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32_t n_req,
+                     const void *q, void *out, void *cuda_stream) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  return step_impl(ctx, layer, req_ids, n_req, nullptr, nullptr, q, out, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int spin_decode_step_append(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32_t n_req,
+                            const void *k_new, const void *v_new, const void *q, void *out,
+                            void *cuda_stream) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  if (!k_new || !v_new) return fail(ctx, SPIN_ERR_INVALID, "null k_new / v_new");
+  return step_impl(ctx, layer, req_ids, n_req, k_new, v_new, q, out, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int spin_stats(spin_ctx *ctx, spin_stats_t *out) {

@@ -83,5 +83,9 @@ class SpinRun:
     def decode(self, layer: int, q, out, stream=None):
         self.spin.decode_step(layer, self.reqs, q, out, stream)
 
+    def step(self, layer: int, k_new, v_new, q, out, stream=None):
+        """Append one token per request and decode, in one library call."""
+        self.spin.decode_step_append(layer, self.reqs, k_new, v_new, q, out, stream)
+
     def close(self):
         self.spin.close()

@@ -26,11 +26,12 @@ def _wl(kind, **kw):
     return W.Workload(**base)
 
 
-def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0):
+def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
+               one_call=False, fetch_mode=0):
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
-                  segment_entries=segment_entries)
+                  segment_entries=segment_entries, fetch_mode=fetch_mode)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
@@ -51,12 +52,15 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     for step in range(w.steps):
         for l in range(w.num_layers):
             kn, vn = run.gen_step_tokens(l, step)
-            run.append(l, kn, vn)
             kb, vb = W.to_bits(kn), W.to_bits(vn)
             for r in range(w.batch):
                 orc.append_kv(oreq[r], l, kb[r:r + 1], vb[r:r + 1])
             q = torch.stack([qs[(r, l)].next() for r in range(w.batch)]).contiguous()
-            run.decode(l, q, out)
+            if one_call:                      # spin_decode_step_append: append + decode in one call
+                run.step(l, kn, vn, q, out)
+            else:
+                run.append(l, kn, vn)
+                run.decode(l, q, out)
             ref = orc.decode_step(l, oreq, W.to_bits(q))
             torch.cuda.synchronize()
             got = out.float().cpu().numpy().astype(np.float64)
@@ -122,6 +126,19 @@ def test_page_minmax_small(sm_scale):
     assert r["rel_l2"] < 2e-2
 
 
+@pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_TOKEN_DOT, W.PART_CLUSTER_CENTROID])
+def test_append_and_decode_in_one_call(kind):
+    # 40 steps cross two page boundaries: both the side-stream append and the serialised one run
+    extra = dict(kv_recipe="mixture", num_clusters=23, max_partition_pages=8) if kind == W.PART_CLUSTER_CENTROID else {}
+    run_parity(_wl(kind, steps=40, topk=12 if kind == W.PART_TOKEN_DOT else 6, **extra), one_call=True)
+
+
+def test_separate_fetch_kernel_mode():
+    run_parity(_wl(W.PART_PAGE_MINMAX, steps=30), fetch_mode=1)
+    run_parity(_wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=23, max_partition_pages=8,
+                   steps=20), fetch_mode=1, one_call=True)
+
+
 def test_page_minmax_outlier_keys_gqa4_many_buckets():
     w = _wl(W.PART_PAGE_MINMAX, num_q_heads=8, num_kv_heads=2, kv_recipe="outlier", outlier_channels=4,
             lru_buckets=64, steps=80, topk=8, slots_per_set=24, drift=0.1, context=16 * 70 + 15)
@@ -182,5 +199,5 @@ def test_cluster_centroid_tight_budget_with_empty_clusters():
 
 def test_tiny_configuration_full_size():
     # the first benchmark configuration as stated: 4096-token context, top-16, 64 slots, 8 buckets
-    r = run_parity(W.CONFIGS["c1"], check_bytes=False)
+    r = run_parity(W.CONFIGS["c1"], check_bytes=False, one_call=True)
     assert r["stats"]["set_steps"] == 32 and r["stats"]["evicted_pages"] > 0
