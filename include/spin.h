@@ -198,9 +198,8 @@ SPIN_API int spin_decode_step(spin_ctx *ctx, int32_t layer, const int32_t *req_i
 
 /* The decode loop's usual pair in one call: spin_append_kv_batch(k_new, v_new) followed by
  * spin_decode_step(q, out), same arguments and results.  When the appended tokens complete no
- * page (15 steps out of 16), the append runs on a stream of the context concurrently with
- * scoring and top-k and is joined, by events, before the cache manager; k_new and v_new may be
- * reused as soon as work enqueued on cuda_stream after this call runs.  Asynchronous. */
+ * page (15 steps out of 16), the append runs inside the scoring kernel (one extra CTA per set)
+ * instead of in a launch of its own.  Asynchronous on cuda_stream. */
 SPIN_API int spin_decode_step_append(spin_ctx *ctx, int32_t layer, const int32_t *req_ids,
                                      int32_t n_req, const void *k_new, const void *v_new,
                                      const void *q, void *out, void *cuda_stream);

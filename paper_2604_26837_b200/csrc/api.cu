@@ -169,9 +169,7 @@ struct spin_ctx {
   uint64_t launches = 0;
   size_t dir_bytes_in_use = 0;
   Prof prof;
-  cudaStream_t side = nullptr;       // runs the decode-time append next to Select
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-  bool join_pending = false;
+  int32_t epoch = 0;                 // decode calls so far (value of the per-set ready flags)
 };
 
 namespace {
@@ -227,6 +225,9 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.fetch_count = a.take<int32_t>(1);
   d.att_part = a.take<float>(B * g.max_chunks * G * (kHeadDim + 2));
   d.att_count = a.take<int32_t>(B);
+  d.sel_count = a.take<int32_t>(B);
+  d.ready = a.take<int32_t>(B);
+  d.tail_ready = a.take<int32_t>(B);
   d.counters = a.take<Counters>(1);
   __nv_bfloat16 *sq = a.take<__nv_bfloat16>((size_t)cfg.max_requests * cfg.num_q_heads * kHeadDim);
   __nv_bfloat16 *so = a.take<__nv_bfloat16>((size_t)cfg.max_requests * cfg.num_q_heads * kHeadDim);
@@ -634,6 +635,9 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   fill(d.gpu_pages, 0, (size_t)g.n_gpu_pages_total * kPageBytes);
   memset(ctx->host_base, 0, ctx->host_bytes);
   fill(d.att_count, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.sel_count, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.ready, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.tail_ready, 0, (size_t)g.max_batch_sets * 4);
   fill(d.state, 0, (size_t)g.n_sets * sizeof(SetState));
   fill(d.counters, 0, sizeof(Counters));
   fill(d.fetch_count, 0, 4);
@@ -652,12 +656,6 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   ctx->sum_segs.init(g.n_sum_segs);
   ctx->reqs.resize((size_t)cfg->max_requests);
   ctx->sets.resize((size_t)g.n_sets);
-  if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
-    cudaGetLastError();
-    ctx->side = nullptr;                // no side stream: appends simply stay on the caller's stream
-  }
   *out = ctx;
   return SPIN_OK;
 }
@@ -670,9 +668,6 @@ int spin_destroy(spin_ctx *ctx) {
     delete[] ctx->prof.ev;
     delete[] ctx->prof.id;
   }
-  if (ctx->side) cudaStreamDestroy(ctx->side);
-  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
-  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   if (ctx->host_base) cudaFreeHost(ctx->host_base);
   delete ctx;
   return SPIN_OK;
@@ -848,10 +843,7 @@ int spin_append_kv_batch(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, i
   return SPIN_OK;
 }
 
-// One decode step, optionally preceded by the append of one token per request.  When the
-// append cannot change what Select sees (no page is completed by it), it runs on the
-// context's side stream concurrently with scoring and top-k and is joined before the cache
-// manager, which hides its host-link write latency.
+// One decode step, optionally preceded by the append of one token per request.
 static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32_t n_req, const void *k,
                      const void *v, const void *q, void *out, cudaStream_t st) {
   if (!req_ids || !q || !out || n_req < 1 || n_req > ctx->cfg.max_requests) return fail(ctx, SPIN_ERR_INVALID, "bad batch arguments");
@@ -871,34 +863,34 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     if (with_append && cluster && !L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req_ids[i]);
     if (with_append && L.n_tokens % kPageTokens == 0) completes_page = true;     // a new page starts
   }
+  const __nv_bfloat16 *kk = nullptr, *vv = nullptr;
+  bool in_grid = false;
   if (with_append) {
-    const bool parallel = !completes_page && !ctx->prof.on && ctx->side != nullptr;
-    cudaStream_t as = parallel ? ctx->side : st;
-    if (parallel) {
-      CK(cudaEventRecord(ctx->ev_fork, st));
-      CK(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
-    }
-    AppendEdgeArgs a{};
-    a.n_req = n_req;
-    a.layer = layer;
     for (int i = 0; i < n_req; ++i) {
-      a.req[i] = req_ids[i];
       LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
-      int rc = cluster ? grow_cluster_tail(ctx, req_ids[i], layer, 1, as) : grow_paged(ctx, req_ids[i], layer, L.n_tokens + 1, as);
+      int rc = cluster ? grow_cluster_tail(ctx, req_ids[i], layer, 1, st) : grow_paged(ctx, req_ids[i], layer, L.n_tokens + 1, st);
       if (rc) return rc;
     }
-    const __nv_bfloat16 *kk = reinterpret_cast<const __nv_bfloat16 *>(k), *vv = reinterpret_cast<const __nv_bfloat16 *>(v);
+    kk = reinterpret_cast<const __nv_bfloat16 *>(k);
+    vv = reinterpret_cast<const __nv_bfloat16 *>(v);
     if (!is_device_ptr(k)) {
       const size_t bytes = (size_t)n_req * ctx->cfg.num_kv_heads * kRowBytes;
-      CK(cudaMemcpyAsync(ctx->stage_k, k, bytes, cudaMemcpyHostToDevice, as));
-      CK(cudaMemcpyAsync(ctx->stage_v, v, bytes, cudaMemcpyHostToDevice, as));
+      CK(cudaMemcpyAsync(ctx->stage_k, k, bytes, cudaMemcpyHostToDevice, st));
+      CK(cudaMemcpyAsync(ctx->stage_v, v, bytes, cudaMemcpyHostToDevice, st));
       kk = ctx->stage_k;
       vv = ctx->stage_v;
     }
-    prof_mark(&ctx->prof, as, -1);
-    ctx->launches += launch_append_edge(ctx->d, a, kk, vv, 1, as, &ctx->prof);
-    if (parallel) CK(cudaEventRecord(ctx->ev_join, ctx->side));
-    ctx->join_pending = parallel;
+    // An append that completes no page cannot change what Select sees: it then runs inside
+    // the scoring kernel (one extra CTA per set).  Otherwise it runs first, on its own.
+    in_grid = !completes_page;
+    if (!in_grid) {
+      AppendEdgeArgs a{};
+      a.n_req = n_req;
+      a.layer = layer;
+      for (int i = 0; i < n_req; ++i) a.req[i] = req_ids[i];
+      prof_mark(&ctx->prof, st, -1);
+      ctx->launches += launch_append_edge(ctx->d, a, kk, vv, 1, st, &ctx->prof);
+    }
   }
   int64_t max_cand = 0, max_pages = 0;
   bool may_be_empty = false;
@@ -910,6 +902,8 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     max_pages = std::max(max_pages, pages + L.tail_pages);
     may_be_empty = may_be_empty || L.n_tokens == 0;
     L.last_batch_pos = i;
+    b.tail_pages[i] = (int16_t)L.tail_pages;
+    b.tail_len[i] = (int16_t)L.tail_len;
   }
   const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
   const __nv_bfloat16 *qd = reinterpret_cast<const __nv_bfloat16 *>(q);
@@ -918,12 +912,10 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   if (!q_dev) { CK(cudaMemcpyAsync(ctx->stage_q, q, qbytes, cudaMemcpyHostToDevice, st)); qd = ctx->stage_q; }
   if (!out_dev) od = ctx->stage_out;
   prof_mark(&ctx->prof, st, -1);
-  ctx->launches += launch_select(ctx->d, b, qd, (int)max_cand, st, &ctx->prof);
-  if (ctx->join_pending) {
-    CK(cudaStreamWaitEvent(st, ctx->ev_join, 0));
-    ctx->join_pending = false;
-  }
-  ctx->launches += launch_cache(ctx->d, b, st, ctx->sm_count, &ctx->prof);
+  b.epoch = ++ctx->epoch;
+  b.append_in_grid = in_grid ? 1 : 0;
+  ctx->launches += launch_select(ctx->d, b, qd, kk, vv, (int)max_cand, st, &ctx->prof);
+  ctx->launches += launch_fetch(ctx->d, st, ctx->sm_count, &ctx->prof);
   ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, may_be_empty, st, &ctx->prof);
   if (!out_dev) CK(cudaMemcpyAsync(out, ctx->stage_out, qbytes, cudaMemcpyDeviceToHost, st));
   CK(cudaGetLastError());

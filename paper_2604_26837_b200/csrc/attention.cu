@@ -153,7 +153,15 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   __shared__ int sh_last;
   const int b = blockIdx.x, chunk = blockIdx.y;       // chunk-major launch order: chunk 0 of every set first
   pdl_launch_next();
-  pdl_wait_prev();
+  if (c.ready) {
+    // start as soon as this set's page list and tail page are complete (see flag_wait)
+    __shared__ int sh_ok;
+    if (threadIdx.x == 0) sh_ok = flag_wait(c, c.ready + b, bt.epoch) && flag_wait(c, c.tail_ready + b, bt.epoch);
+    __syncthreads();
+    if (!sh_ok) return;
+  } else {
+    pdl_wait_prev();
+  }
   const int np = c.n_pages[b];
   const int first = chunk * kChunkPages;
   if (first >= np) return;
@@ -431,6 +439,8 @@ extern "C" int spin_paged_attention_static(const void *q, const void *page_pool,
   c.n_pages = const_cast<int32_t *>(n_pages);
   c.page_fill = nullptr;                                    // every listed page is already in the pool
   c.page_desc = nullptr;                                    // the lists are attended in the order given
+  c.ready = nullptr;                                        // plain stream order: no per-set flags
+  c.tail_ready = nullptr;
   c.att_count = reinterpret_cast<int32_t *>(g_static_partials_addr[dev]);
   c.att_part = g_static_partials_addr[dev] + counter_floats;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);

@@ -8,19 +8,19 @@
 // balanced tree over adjacent blocks; the group's query heads are added in ascending order.
 // Products of two bf16 values are exact in fp32, so fused or separate multiply-add agree.
 //
-// k_topk keeps, per set, the k best candidates (ties -> lower index) with a 4-pass radix
-// select on order-preserving keys followed by one ordered compaction, and emits them in
-// ascending index order.  For token-granular selection it also folds the chosen tokens into
-// their pages with a 16-bit token mask per page.
-#include <cooperative_groups.h>
-
-#include "spin_dev.cuh"
-
-namespace cg = cooperative_groups;
+// In its fused form the last scoring CTA of a set (an arrival counter per set) carries on
+// with that set's top-k and cache management (stages.cuh) while other sets are still being
+// scored, so the step needs no top-k or cache-manager launch.  k_topk is the stand-alone
+// top-k for candidate counts beyond one CTA's shared memory: a thread-block cluster per set.
+#include "append_body.cuh"
+#include "stages.cuh"
 
 namespace spin {
 
 namespace {
+
+constexpr int kScoreThreads = 256;
+constexpr int kTopkThreads = 512;
 
 __device__ __forceinline__ void unpack8(uint4 raw, float *f) {
   const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -70,20 +70,35 @@ __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, con
 }
 
 template <int G, bool MINMAX>
-__global__ void __launch_bounds__(256)
-k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
+__global__ void __launch_bounds__(kScoreThreads)
+k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
+        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap) {
+  extern __shared__ __align__(16) uint8_t dyn_smem[];      // used by the fused continuation only
   const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
   pdl_launch_next();
   pdl_wait_prev();
   if (blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *c.fetch_count = 0;   // new step, new miss queue
+  if (blockIdx.x == gridDim.x - 1) {
+    // the set's tail CTA: appends this step's token (unless a stand-alone append already ran)
+    // and tells the attention kernel that the tail page is complete
+    __shared__ __align__(16) __nv_bfloat16 krows[kPageTokens][kHeadDim];
+    if (bt.append_in_grid) append_edge_body(c, set, i_req, head, k_new, v_new, 1, krows);
+    __syncthreads();
+    if (threadIdx.x == 0) flag_publish(c.tail_ready + b, bt.epoch);
+    return;
+  }
   const SetState st = c.state[set];
   const int n_cand = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
   const int seg_entries = 1 << c.sum_shift;
   const int e0 = blockIdx.x * seg_entries;
-  if (e0 >= n_cand) return;
-  const int seg = c.dir_sumseg[(size_t)set * c.dir_sum + blockIdx.x];
-  if (seg < 0) { if (threadIdx.x == 0) dev_error(c, kErrBounds); return; }
+  // the CTAs that count towards the set's arrival counter: one per non-empty segment, and
+  // segment 0 even when the set has no candidate yet
+  const int segs_here = max(1, (n_cand + seg_entries - 1) >> c.sum_shift);
+  if ((int)blockIdx.x >= segs_here) return;
+  const int seg = e0 < n_cand ? c.dir_sumseg[(size_t)set * c.dir_sum + blockIdx.x] : 0;
+  if (seg < 0 && threadIdx.x == 0) dev_error(c, kErrBounds);
+  if (e0 < n_cand && seg >= 0) {
   const int lane16 = threadIdx.x & 15, grp = threadIdx.x >> 4;
   // the two 16-lane rows of a warp may leave the loop at different times: each shuffles
   // only among its own lanes
@@ -120,241 +135,89 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q) {
       if (lane16 == 0) out[e + 16] = s1;
     }
   }
-}
-
-__device__ __forceinline__ uint32_t order_key(float s) {
-  const uint32_t u = __float_as_uint(s);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-constexpr int kTopkThreads = 512;
-
-// Exclusive prefix of v over the block (thread order) and the block total.
-__device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t *wsum, uint32_t *total) {
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  uint32_t inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
   }
-  if (lane == 31) wsum[w] = inc;
+  if (!fuse) return;
+
+  // ---- fused continuation: the last CTA of the set to arrive selects and manages the cache ----
+  __shared__ TopkShared tsh;
+  __shared__ CacheShared csh;
+  __shared__ int s_last;
+  __threadfence();
   __syncthreads();
-  if (w == 0) {
-    uint32_t x = lane < kTopkThreads / 32 ? wsum[lane] : 0, xi = x;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      uint32_t t = __shfl_up_sync(0xffffffffu, xi, o);
-      if (lane >= o) xi += t;
-    }
-    wsum[lane] = xi - x;                         // exclusive warp offsets
-    if (lane == 31) wsum[32] = xi;               // total
-  }
+  if (threadIdx.x == 0) s_last = atomicAdd(&c.sel_count[b], 1) == segs_here - 1;
   __syncthreads();
-  const uint32_t res = wsum[w] + inc - v;
-  *total = wsum[32];
-  __syncthreads();                               // wsum is reused by the next call
-  return res;
+  if (!s_last) return;
+  __threadfence();
+  if (threadIdx.x == 0) c.sel_count[b] = 0;                 // ready for the next step
+  topk_stage<kScoreThreads, false>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh);
+  cache_stage<kScoreThreads>(c, b, set, __ldcg(c.n_parts + b), bt.tail_pages[i_req], bt.tail_len[i_req],
+                             bt.epoch, reinterpret_cast<int32_t *>(dyn_smem), csh);
 }
 
-// One thread-block cluster per set: the candidates are cut into one contiguous slice per CTA
-// (keys kept in shared memory), every radix pass builds per-CTA histograms that all CTAs sum
-// through distributed shared memory, and the ordered compaction uses the lower-ranked CTAs'
-// counts as its offset.  A cluster of one CTA is the small-set case (a few thousand pages);
-// token-granular selection over 64K+ keys uses 8 CTAs.  Cluster barriers are hardware
-// barriers (no flag spinning); every CTA of a cluster executes the same number of them.
+// Stand-alone top-k: one thread-block cluster per set (slices of the keys in shared memory).
 __global__ void __launch_bounds__(kTopkThreads)
 k_topk(DevCtx c, Batch bt, int keys_cap) {
-  extern __shared__ uint32_t s_keys[];                 // [keys_cap] order-preserving keys of this slice
-  __shared__ uint32_t hist[256];                       // this CTA's histogram (read remotely)
-  __shared__ uint32_t ghist[256];                      // cluster-wide histogram
-  __shared__ uint32_t wsum[33];
-  __shared__ uint32_t cnt[2];                          // this CTA's (above threshold, equal) counts
-  __shared__ uint32_t sh_prefix, sh_remaining;
-  cg::cluster_group cluster = cg::this_cluster();
-  const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
-  const int b = blockIdx.x / C, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
+  extern __shared__ __align__(16) uint8_t dyn_smem[];
+  __shared__ TopkShared tsh;
+  const int C = (int)cg::this_cluster().num_blocks();
+  const int b = blockIdx.x / C, i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
   pdl_launch_next();
   pdl_wait_prev();
   const SetState st = c.state[set];
-  const int n = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
-  const int k = min(c.topk, n);
-  const float *scores = c.scores + (size_t)b * c.max_cand;
-  int32_t *sel = c.sel_ids + (size_t)b * c.max_sel;
-  const int per = (n + C - 1) / C;
-  const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
-  const bool cached = m <= keys_cap;
-
-  if (tid == 0 && rank == 0) {
-    c.n_sel[b] = k;
-    atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
-  }
-  if (cached)
-    for (int i = tid; i < m; i += kTopkThreads) s_keys[i] = order_key(scores[lo + i]);
-  __syncthreads();
-  auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(scores[lo + i]); };
-
-  if (k == n) {
-    for (int i = tid; i < m; i += kTopkThreads) sel[lo + i] = lo + i;
-  } else {
-    // ---- radix select: key of the k-th best candidate --------------------------------
-    uint32_t prefix = 0, mask = 0, remaining = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      if (tid < 256) hist[tid] = 0;
-      __syncthreads();
-      for (int i = tid; i < m; i += kTopkThreads) {
-        const uint32_t key = key_at(i);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-      }
-      cluster.sync();                                   // every CTA's histogram is complete
-      if (tid < 256) {
-        uint32_t tot = 0;
-        for (int r = 0; r < C; ++r) tot += cluster.map_shared_rank(hist, r)[tid];
-        ghist[tid] = tot;
-      }
-      cluster.sync();                                   // remote reads done before hist is reused
-      if (tid < 32) {
-        // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the
-        // top reaches `remaining`
-        uint32_t loc[8], sum = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { loc[j] = ghist[255 - 8 * tid - j]; sum += loc[j]; }
-        uint32_t inc = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-          if (tid >= o) inc += t;
-        }
-        const uint32_t before = inc - sum;
-        if (before < remaining && inc >= remaining) {
-          uint32_t cum = before;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (cum < remaining && cum + loc[j] >= remaining) {
-              sh_prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
-              sh_remaining = remaining - cum;
-            }
-            cum += loc[j];
-          }
-        }
-      }
-      __syncthreads();
-      prefix = sh_prefix;
-      remaining = sh_remaining;
-      mask |= 255u << shift;
-    }
-    const uint32_t thr = prefix, need_eq = remaining;
-    // ---- counts of this slice, offsets from the lower-ranked slices ---------------------
-    if (tid < 2) cnt[tid] = 0;
-    __syncthreads();
-    {
-      uint32_t gt = 0, eq = 0;
-      for (int i = tid; i < m; i += kTopkThreads) {
-        const uint32_t key = key_at(i);
-        gt += key > thr;
-        eq += key == thr;
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        gt += __shfl_xor_sync(0xffffffffu, gt, o);
-        eq += __shfl_xor_sync(0xffffffffu, eq, o);
-      }
-      if ((tid & 31) == 0) { atomicAdd(&cnt[0], gt); atomicAdd(&cnt[1], eq); }
-    }
-    cluster.sync();
-    uint32_t run_gt = 0, run_eq = 0;
-    for (int r = 0; r < rank; ++r) {
-      const uint32_t *rc = cluster.map_shared_rank(cnt, r);
-      run_gt += rc[0];
-      run_eq += rc[1];
-    }
-    // ---- ordered compaction: everything above thr, plus the first need_eq equal to it --
-    for (int base = 0; base < m; base += kTopkThreads) {
-      const int i = base + tid;
-      uint32_t gt = 0, eq = 0;
-      if (i < m) {
-        const uint32_t key = key_at(i);
-        gt = key > thr;
-        eq = key == thr;
-      }
-      uint32_t total;
-      const uint32_t ex = block_scan(gt | (eq << 16), wsum, &total);
-      const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
-      if (gt || (eq && eq_before < need_eq))
-        sel[gt_before + min(eq_before, need_eq)] = lo + i;
-      run_gt += total & 0xffffu;
-      run_eq += total >> 16;
-    }
-  }
-  cluster.sync();            // selections of all slices are written; nobody reads remote smem after this
-  if (rank != 0) return;
-
-  // ---- candidates -> partitions of the cache manager (first CTA of the cluster) ----------
-  int32_t *parts = c.parts + (size_t)b * c.max_parts;
-  if (c.kind != kKindToken) {
-    for (int i = tid; i < k; i += kTopkThreads) parts[i] = __ldcg(sel + i);
-    if (tid == 0) c.n_parts[b] = k;
-    return;
-  }
-  uint32_t *pmask = c.part_mask + (size_t)b * c.max_parts;
-  for (int i = tid; i < k; i += kTopkThreads) pmask[i] = 0;
-  __syncthreads();
-  uint32_t run = 0;
-  for (int base = 0; base < k; base += kTopkThreads) {
-    const int i = base + tid;
-    uint32_t first = 0;
-    int tok = 0;
-    if (i < k) {
-      tok = __ldcg(sel + i);
-      first = (i == 0) || ((__ldcg(sel + i - 1) >> 4) != (tok >> 4));
-    }
-    uint32_t total;
-    const uint32_t ex = block_scan(first, wsum, &total);
-    if (i < k) {
-      const uint32_t rank_ = run + ex + first - 1;
-      if (first) parts[rank_] = tok >> 4;
-      atomicOr(&pmask[rank_], 1u << (tok & 15));
-    }
-    run += total;
-  }
-  if (tid == 0) c.n_parts[b] = (int)run;
+  topk_stage<kTopkThreads, true>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh);
 }
 
+
 template <int G>
-void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, dim3 grid, cudaStream_t st) {
-  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(256), 0, st, 1, c, b, q);
-  else launch_pdl(k_score<G, false>, grid, dim3(256), 0, st, 1, c, b, q);
+void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
+                    const __nv_bfloat16 *v_new, dim3 grid, size_t smem, int fuse, int keys_cap, cudaStream_t st) {
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaFuncSetAttribute(k_score<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(k_score<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    configured = smem;
+  }
+  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap);
+  else launch_pdl(k_score<G, false>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap);
 }
 
 }  // namespace
 
-int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int max_cand,
-                  cudaStream_t st, Prof *prof) {
+// Select + (fused or separate) cache management.  Returns the kernels launched.
+int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
+                  const __nv_bfloat16 *v_new, int max_cand, cudaStream_t st, Prof *prof) {
   const int n_sets = b.n_req * c.Hkv;
   int segs = (max_cand + (1 << c.sum_shift) - 1) >> c.sum_shift;
-  if (segs < 1) segs = 1;                         // the first block also resets the miss queue
-  dim3 grid(segs, n_sets);
+  if (segs < 1) segs = 1;                         // segment 0 always runs (arrival counter, miss-queue reset)
+  dim3 grid(segs + 1, n_sets);                    // + one tail CTA per set (in-grid append, tail flag)
+  // fused: one CTA can hold a set's keys and the cache manager's tables in shared memory
+  const size_t cache_smem = cache_stage_smem_bytes(c.max_parts, c.max_pages, c.max_slots);
+  const bool fuse = max_cand <= 16384 && cache_smem <= 96 * 1024;
+  const int keys_cap = fuse ? max_cand : 0;
+  size_t smem = 0;
+  if (fuse) smem = cache_smem > (size_t)keys_cap * 4 ? cache_smem : (size_t)keys_cap * 4;
   switch (c.G) {
-    case 1: launch_score_g<1>(c, b, q, grid, st); break;
-    case 2: launch_score_g<2>(c, b, q, grid, st); break;
-    case 4: launch_score_g<4>(c, b, q, grid, st); break;
-    default: launch_score_g<8>(c, b, q, grid, st); break;
+    case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
+    case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
+    case 4: launch_score_g<4>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
+    default: launch_score_g<8>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
   }
   prof_mark(prof, st, kProfScore);
+  if (fuse) return 1;
   {
     // cluster size from the largest candidate count: slices of at most 8192 keys stay in smem
     int C = 1;
     while (C < 8 && (max_cand + C - 1) / C > 8192) C *= 2;
-    int keys_cap = (max_cand + C - 1) / C;
-    if (keys_cap > 16384) keys_cap = 0;                  // too many for shared memory: re-read from L2
+    int kc = (max_cand + C - 1) / C;
+    if (kc > 16384) kc = 0;                              // too many for shared memory: re-read from L2
     static int smem_set = 0;
-    const int smem = keys_cap * 4;
-    if (smem > smem_set) { cudaFuncSetAttribute(k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); smem_set = smem; }
-    launch_pdl(k_topk, dim3(n_sets * C), dim3(kTopkThreads), (size_t)smem, st, C, c, b, keys_cap);
+    const int ksmem = kc * 4;
+    if (ksmem > smem_set) { cudaFuncSetAttribute(k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, ksmem); smem_set = ksmem; }
+    launch_pdl(k_topk, dim3(n_sets * C), dim3(kTopkThreads), (size_t)ksmem, st, C, c, b, kc);
   }
   prof_mark(prof, st, kProfTopk);
-  return 2;
+  return 2 + launch_cache(c, b, st, prof);
 }
 
 }  // namespace spin

@@ -98,6 +98,9 @@ struct DevCtx {
   int32_t fetch_cap;
   float *att_part;              // split-K partials [b][max_chunks][G][kHeadDim + 2]
   int32_t *att_count;           // [b] chunks of the set that have finished (zero before attention)
+  int32_t *sel_count;           // [b] scoring CTAs of the set that have finished (zero between steps)
+  int32_t *ready;               // [b] epoch of the last step whose page list is complete
+  int32_t *tail_ready;          // [b] epoch of the last step whose appended rows are in the tail page
   int32_t max_chunks;
   int32_t fetch_mode;           // 0: misses are fetched by the attention kernel; 1: by k_fetch
   Counters *counters;
@@ -107,6 +110,12 @@ struct Batch {
   int32_t n_req;
   int32_t layer;
   int32_t req[kMaxBatch];
+  // local tail of each request after this step's append, as the host has counted it: lets
+  // the cache manager lay out the page list without waiting for the append kernel
+  int16_t tail_pages[kMaxBatch];
+  int16_t tail_len[kMaxBatch];
+  int32_t epoch;            // number of this decode call: value of the ready flags it sets
+  int32_t append_in_grid;   // the scoring kernel's tail CTAs append this step's tokens
 };
 
 __host__ __device__ inline int set_index(const DevCtx &c, int req, int layer, int head) {
@@ -149,6 +158,27 @@ __device__ __forceinline__ uint8_t *summary_at(const DevCtx &c, int set, int e) 
 // another kernel touches.
 __device__ __forceinline__ void pdl_launch_next() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_prev() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Per-set flags that let the attention kernel start on a set as soon as that set's page list
+// is complete, while the scoring kernel is still working on other sets.  The producer is
+// always resident before a consumer can exist (the consumer kernel is launched with
+// programmatic stream serialization after every producer CTA has started), so a consumer only
+// ever waits for work that is already running.  The wait is bounded all the same: it gives up
+// after ~0.1 s, reports SPIN_DEV_ERR_TIMEOUT and the CTA returns without touching the set.
+__device__ __forceinline__ void flag_publish(int32_t *flag, int32_t value) {
+  __threadfence();
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
+}
+__device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, int32_t value) {
+  for (int spin = 0; spin < (1 << 20); ++spin) {
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v == value) return true;
+    __nanosleep(100);
+  }
+  dev_error(c, kErrTimeout);
+  return false;
+}
 
 __device__ __forceinline__ const uint8_t *page_ptr(const DevCtx &c, int src) {
   return src >= 0 ? c.gpu_pages + (size_t)src * kPageBytes : c.host_pages + (size_t)(~src) * kPageBytes;
@@ -209,9 +239,10 @@ int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloa
                            cudaStream_t st);
 int launch_copy_centroids(const DevCtx &c, int req, int layer, const __nv_bfloat16 *cen,
                           int n_clusters, cudaStream_t st);
-int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, int max_cand,
-                  cudaStream_t st, Prof *prof);
-int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, int sm_count, Prof *prof);
+int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
+                  const __nv_bfloat16 *v_new, int max_cand, cudaStream_t st, Prof *prof);
+int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
+int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
 size_t cache_smem_bytes(const DevCtx &c);
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
                      __nv_bfloat16 *out, int max_pages_hint, bool may_be_empty, cudaStream_t st, Prof *prof);

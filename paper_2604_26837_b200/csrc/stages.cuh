@@ -1,0 +1,539 @@
+// The two per-set stages between scoring and attention, written as device functions so that
+// they can run either as kernels of their own (token-granular selection over 64K+ keys uses a
+// thread-block cluster per set for top-k) or as the continuation of the scoring kernel: the
+// last scoring CTA of a set to finish goes straight on with that set's top-k and cache
+// management while the other sets are still being scored.
+//
+//   topk_stage  -- Select's "-> topk" (Table 1): k best candidates, ties to the lower index,
+//                  emitted ascending; token-granular selections are folded into pages + masks.
+//   cache_stage -- Retrieve steps 1-3 (Section 5.2) and bucketed LRU steps 1-4 (Section 5.3):
+//                  metadata only; the page bytes move in the attention kernel (or k_fetch).
+#pragma once
+#include <cooperative_groups.h>
+
+#include "spin_dev.cuh"
+
+namespace spin {
+
+namespace cg = cooperative_groups;
+
+enum : int { kHit = 0, kAdmit = 1, kBypass = 2 };
+
+__device__ __forceinline__ uint32_t order_key(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive prefix of v over the block (thread order) and the block total.  wsum: 33 words.
+template <int T>
+__device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t *wsum, uint32_t *total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    uint32_t x = lane < T / 32 ? wsum[lane] : 0, xi = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t t = __shfl_up_sync(0xffffffffu, xi, o);
+      if (lane >= o) xi += t;
+    }
+    wsum[lane] = xi - x;                         // exclusive warp offsets
+    if (lane == 31) wsum[32] = xi;               // total
+  }
+  __syncthreads();
+  const uint32_t res = wsum[w] + inc - v;
+  *total = wsum[32];
+  __syncthreads();                               // wsum is reused by the next call
+  return res;
+}
+
+// index of `p` in the ascending array a[0..n), or -1
+__device__ __forceinline__ int find_sorted(const int32_t *a, int n, int p) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    int mid = (lo + hi) >> 1;
+    if (a[mid] < p) lo = mid + 1; else hi = mid;
+  }
+  return (lo < n && a[lo] == p) ? lo : -1;
+}
+// largest r with off[r] <= idx (off ascending, off[0] == 0)
+__device__ __forceinline__ int owner_of(const int32_t *off, int n, int idx) {
+  int lo = 0, hi = n;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (off[mid] <= idx) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+struct TopkShared {
+  uint32_t hist[256];          // this CTA's histogram (read remotely inside a cluster)
+  uint32_t ghist[256];         // histogram over the whole set
+  uint32_t wsum[33];
+  uint32_t cnt[2];             // this CTA's (above threshold, equal) counts
+  uint32_t prefix, remaining;
+};
+
+template <bool CLUSTER> __device__ __forceinline__ void stage_sync() {
+  if constexpr (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
+}
+
+// Top-k of one set.  With CLUSTER the set's candidates are cut into one contiguous slice per
+// CTA of the cluster (keys kept in shared memory), every radix pass builds per-CTA histograms
+// that all CTAs sum through distributed shared memory, and the ordered compaction starts at
+// the lower-ranked CTAs' counts.  Cluster barriers are hardware barriers (nothing spins on a
+// flag) and every CTA of a cluster executes the same number of them.  Without CLUSTER the
+// calling CTA owns the whole set.  On return (all threads of rank 0) the partitions handed to
+// the cache manager are in c.parts / c.n_parts; other ranks return false and must exit.
+template <int T, bool CLUSTER>
+__device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partitions, uint32_t *s_keys,
+                                           int keys_cap, TopkShared &sh) {
+  int C = 1, rank = 0;
+  if constexpr (CLUSTER) {
+    cg::cluster_group cluster = cg::this_cluster();
+    C = (int)cluster.num_blocks();
+    rank = (int)cluster.block_rank();
+  }
+  const int tid = threadIdx.x;
+  const int n = c.kind == kKindToken ? n_partitions * kPageTokens : n_partitions;
+  const int k = min(c.topk, n);
+  const float *scores = c.scores + (size_t)b * c.max_cand;
+  int32_t *sel = c.sel_ids + (size_t)b * c.max_sel;
+  const int per = (n + C - 1) / C;
+  const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
+  const bool cached = m <= keys_cap;
+
+  if (tid == 0 && rank == 0) {
+    c.n_sel[b] = k;
+    atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
+  }
+  if (cached)
+    for (int i = tid; i < m; i += T) s_keys[i] = order_key(__ldcg(scores + lo + i));
+  __syncthreads();
+  auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(__ldcg(scores + lo + i)); };
+
+  if (k == n) {
+    for (int i = tid; i < m; i += T) sel[lo + i] = lo + i;
+  } else {
+    // ---- radix select: key of the k-th best candidate --------------------------------
+    uint32_t prefix = 0, mask = 0, remaining = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      if (tid < 256) sh.hist[tid] = 0;
+      __syncthreads();
+      for (int i = tid; i < m; i += T) {
+        const uint32_t key = key_at(i);
+        if ((key & mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
+      }
+      stage_sync<CLUSTER>();                          // every CTA's histogram is complete
+      for (int bin = tid; bin < 256; bin += T) {
+        uint32_t tot = 0;
+        if constexpr (CLUSTER) {
+          cg::cluster_group cluster = cg::this_cluster();
+          for (int r = 0; r < C; ++r) tot += cluster.map_shared_rank(sh.hist, r)[bin];
+        } else {
+          tot = sh.hist[bin];
+        }
+        sh.ghist[bin] = tot;
+      }
+      stage_sync<CLUSTER>();                          // remote reads done before hist is reused
+      if (tid < 32) {
+        // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the
+        // top reaches `remaining`
+        uint32_t loc[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { loc[j] = sh.ghist[255 - 8 * tid - j]; sum += loc[j]; }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += t;
+        }
+        const uint32_t before = inc - sum;
+        if (before < remaining && inc >= remaining) {
+          uint32_t cum = before;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (cum < remaining && cum + loc[j] >= remaining) {
+              sh.prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
+              sh.remaining = remaining - cum;
+            }
+            cum += loc[j];
+          }
+        }
+      }
+      __syncthreads();
+      prefix = sh.prefix;
+      remaining = sh.remaining;
+      mask |= 255u << shift;
+    }
+    const uint32_t thr = prefix, need_eq = remaining;
+    // ---- counts of this slice, offsets from the lower-ranked slices ---------------------
+    uint32_t run_gt = 0, run_eq = 0;
+    if constexpr (CLUSTER) {
+      if (tid < 2) sh.cnt[tid] = 0;
+      __syncthreads();
+      uint32_t gt = 0, eq = 0;
+      for (int i = tid; i < m; i += T) {
+        const uint32_t key = key_at(i);
+        gt += key > thr;
+        eq += key == thr;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        gt += __shfl_xor_sync(0xffffffffu, gt, o);
+        eq += __shfl_xor_sync(0xffffffffu, eq, o);
+      }
+      if ((tid & 31) == 0) { atomicAdd(&sh.cnt[0], gt); atomicAdd(&sh.cnt[1], eq); }
+      cg::cluster_group cluster = cg::this_cluster();
+      cluster.sync();
+      for (int r = 0; r < rank; ++r) {
+        const uint32_t *rc = cluster.map_shared_rank(sh.cnt, r);
+        run_gt += rc[0];
+        run_eq += rc[1];
+      }
+    }
+    // ---- ordered compaction: everything above thr, plus the first need_eq equal to it --
+    for (int base = 0; base < m; base += T) {
+      const int i = base + tid;
+      uint32_t gt = 0, eq = 0;
+      if (i < m) {
+        const uint32_t key = key_at(i);
+        gt = key > thr;
+        eq = key == thr;
+      }
+      uint32_t total;
+      const uint32_t ex = block_scan<T>(gt | (eq << 16), sh.wsum, &total);
+      const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
+      if (gt || (eq && eq_before < need_eq))
+        sel[gt_before + min(eq_before, need_eq)] = lo + i;
+      run_gt += total & 0xffffu;
+      run_eq += total >> 16;
+    }
+  }
+  stage_sync<CLUSTER>();     // selections of all slices are written; no remote smem is read after this
+  if (rank != 0) return false;
+
+  // ---- candidates -> partitions of the cache manager (first CTA of the cluster) ----------
+  int32_t *parts = c.parts + (size_t)b * c.max_parts;
+  if (c.kind != kKindToken) {
+    for (int i = tid; i < k; i += T) parts[i] = __ldcg(sel + i);
+    if (tid == 0) c.n_parts[b] = k;
+    __syncthreads();
+    return true;
+  }
+  uint32_t *pmask = c.part_mask + (size_t)b * c.max_parts;
+  for (int i = tid; i < k; i += T) pmask[i] = 0;
+  __syncthreads();
+  uint32_t run = 0;
+  for (int base = 0; base < k; base += T) {
+    const int i = base + tid;
+    uint32_t first = 0;
+    int tok = 0;
+    if (i < k) {
+      tok = __ldcg(sel + i);
+      first = (i == 0) || ((__ldcg(sel + i - 1) >> 4) != (tok >> 4));
+    }
+    uint32_t total;
+    const uint32_t ex = block_scan<T>(first, sh.wsum, &total);
+    if (i < k) {
+      const uint32_t rank_ = run + ex + first - 1;
+      if (first) parts[rank_] = tok >> 4;
+      atomicOr(&pmask[rank_], 1u << (tok & 15));
+    }
+    run += total;
+  }
+  if (tid == 0) c.n_parts[b] = (int)run;
+  __syncthreads();
+  return true;
+}
+
+struct CacheShared {
+  uint32_t hist[kMaxBuckets + 2];
+  uint32_t wsum[33];
+  int32_t hostpage[512];       // CPU page ids of the first missed pages (looked up early)
+  int x, demand, evicted, qbase, admit_pages, bypass_pages;
+};
+
+__host__ __device__ inline size_t cache_stage_smem_bytes(int max_parts, int max_pages, int max_slots) {
+  return (size_t)(6 * max_parts + 1 + max_pages) * 4 + (size_t)((max_slots + 31) / 32) * 4 + 16;
+}
+
+// Cache manager of one set, run by all T threads of one CTA.  `np_in` partitions are read
+// from c.parts (ascending).  smem: cache_stage_smem_bytes() of dynamic shared memory.
+template <int T>
+__device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int np_in, int tail_pages,
+                                            int tail_len, int epoch, int32_t *smem, CacheShared &sh) {
+  int32_t *s_parts = smem;                          // [max_parts]
+  int32_t *s_tokens = s_parts + c.max_parts;        // [max_parts]
+  int32_t *s_pageoff = s_tokens + c.max_parts;      // [max_parts + 1]
+  int32_t *s_missoff = s_pageoff + c.max_parts + 1; // [max_parts] offset into the free list
+  int32_t *s_missbefore = s_missoff + c.max_parts;  // [max_parts] missed pages of earlier partitions
+  int32_t *s_state = s_missbefore + c.max_parts;    // [max_parts]
+  int32_t *s_free = s_state + c.max_parts;          // [max_pages]
+  uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_free + c.max_pages);   // [max_slots/32]
+  const int tid = threadIdx.x;
+  const SetState st = c.state[set];
+  const int S = st.slots, n = c.n_buckets, t = st.step;
+  const int top = min(t, n - 1);
+  int np = np_in;
+  const int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
+  const size_t pl = (size_t)b * (c.max_pages + c.tail_cap);
+  int32_t *page_src = c.page_src + pl, *page_slot = c.page_slot + pl;
+  int32_t *page_part = c.page_part + pl, *page_pidx = c.page_pidx + pl;
+  uint32_t *page_mask = c.page_mask + pl;
+  int32_t *page_fill = c.page_fill + pl;
+  int4 *page_desc = c.page_desc + pl;
+  if (tid == 0) c.att_count[b] = 0;
+
+  // ---- step 1: hit/miss classification, page demand ------------------------------------
+  uint32_t run_all = 0, run_miss = 0;
+  for (int base = 0; base < np; base += T) {
+    const int r = base + tid;
+    uint32_t npg = 0, miss = 0;
+    if (r < np) {
+      const int p = __ldcg(g_parts + r);
+      const MetaEntry *m = meta_at(c, set, p);
+      int tokens = 0, res = 1;
+      if (m) { tokens = m->tokens; res = m->resident; } else dev_error(c, kErrBounds);
+      npg = (tokens + kPageTokens - 1) / kPageTokens;
+      miss = res ? 0 : 1;
+      s_parts[r] = p;
+      s_tokens[r] = tokens;
+      s_state[r] = res ? kHit : kAdmit;
+    }
+    uint32_t tot_a, tot_m;
+    const uint32_t ex_a = block_scan<T>(npg, sh.wsum, &tot_a);
+    const uint32_t ex_m = block_scan<T>(miss ? npg : 0, sh.wsum, &tot_m);
+    if (r < np) {
+      s_pageoff[r] = run_all + ex_a;
+      s_missoff[r] = run_miss + ex_m;
+      s_missbefore[r] = run_miss + ex_m;
+    }
+    run_all += tot_a;
+    run_miss += tot_m;
+  }
+  if (tid == 0) {
+    s_pageoff[np] = run_all;
+    sh.evicted = 0;
+    sh.admit_pages = 0;
+    sh.bypass_pages = 0;
+  }
+  int total_pages = (int)run_all;
+  const int demand = (int)run_miss;
+  if (total_pages > c.max_pages) {
+    // more pages than the scratch holds: drop the partitions that do not fit, report it
+    if (tid == 0) dev_error(c, kErrPageList);
+    __syncthreads();
+    while (np > 0 && s_pageoff[np] > c.max_pages) --np;
+    total_pages = s_pageoff[np];
+  }
+  for (int i = tid; i < (S + 31) / 32; i += T) s_hit[i] = 0;
+  for (int i = tid; i < kMaxBuckets + 2; i += T) sh.hist[i] = 0;
+  __syncthreads();
+
+  // Retrieve step 3, started early: the Partition Offset / CPU page table entries of the
+  // missed pages live in pinned host memory, two dependent reads over the host link.  They
+  // are issued here and consumed after the table scans below, which hides their latency.
+  int early_i = 0, early_off = -1, early_host = -1;
+  if (tid < demand && np > 0) {
+    const int r = owner_of(s_missbefore, np, tid);
+    early_i = tid - s_missbefore[r];
+    const int32_t *off = off_at(c, set, s_parts[r]);
+    if (off) early_off = *off;
+  }
+
+  // ---- step 2: one scan of the GPU page table: promote, demote, histogram ---------------
+  for (int s = tid; s < S; s += T) {
+    GptEntry *e = gpt_at(c, set, s);
+    if (!e) { dev_error(c, kErrBounds); continue; }
+    const int4 raw = *reinterpret_cast<const int4 *>(e);
+    const int part = raw.x, phys = raw.y, pidx = raw.z;
+    int ts = raw.w;
+    if (c.trace) {
+      c.evict_trace[((size_t)set * c.max_slots + s) * 2] = -1;
+      c.evict_trace[((size_t)set * c.max_slots + s) * 2 + 1] = -1;
+    }
+    if (part < 0) { atomicAdd(&sh.hist[0], 1u); continue; }
+    const int r = find_sorted(s_parts, np, part);
+    if (r >= 0) {
+      atomicOr(&s_hit[s >> 5], 1u << (s & 31));
+      if (ts != top) e->ts = top;
+      const int idx = s_pageoff[r] + pidx;
+      page_src[idx] = phys;
+      page_slot[idx] = s;
+    } else {
+      if (t > n - 1 && ts > 0) { --ts; e->ts = ts; }
+      atomicAdd(&sh.hist[ts + 1], 1u);
+    }
+  }
+  __syncthreads();
+
+  if (early_off >= 0) {
+    const int32_t *hp = cpt_at(c, set, early_off + early_i);
+    if (hp) early_host = *hp;
+  }
+
+  // ---- step 3: threshold and eviction; free slots in ascending order --------------------
+  if (tid == 0) {
+    int x = -2;                                   // nothing is <= -2: no eviction
+    if (demand > 0) {
+      x = n - 1;
+      uint32_t cum = 0;
+      for (int bk = -1; bk < n; ++bk) {
+        cum += sh.hist[bk + 1];
+        if ((int)cum >= demand) { x = bk; break; }
+      }
+    }
+    sh.x = x;
+  }
+  __syncthreads();
+  const int x = sh.x;
+  uint32_t run_free = 0;
+  if (demand > 0) {
+    for (int base = 0; base < S; base += T) {
+      const int s = base + tid;
+      uint32_t fr = 0;
+      if (s < S) {
+        GptEntry *e = gpt_at(c, set, s);
+        if (e) {
+          const int part = e->partition;
+          if (part < 0) fr = 1;
+          else if (!((s_hit[s >> 5] >> (s & 31)) & 1u) && e->ts <= x) {
+            MetaEntry *m = meta_at(c, set, part);
+            if (m) m->resident = 0;
+            if (c.trace) {
+              c.evict_trace[((size_t)set * c.max_slots + s) * 2] = part;
+              c.evict_trace[((size_t)set * c.max_slots + s) * 2 + 1] = e->page_idx;
+            }
+            e->partition = -1;
+            e->page_idx = 0;
+            e->ts = -1;
+            atomicAdd(&sh.evicted, 1);
+            fr = 1;
+          }
+        }
+      }
+      uint32_t tot;
+      const uint32_t ex = block_scan<T>(fr, sh.wsum, &tot);
+      if (fr && run_free + ex < (uint32_t)c.max_pages) s_free[run_free + ex] = s;
+      run_free += tot;
+    }
+  }
+  __syncthreads();
+
+  sh.hostpage[tid] = early_host;
+
+  // ---- step 4: admission (whole partitions; what does not fit is bypassed) --------------
+  if (demand > (int)run_free) {
+    if (tid == 0) {
+      int used = 0;
+      for (int r = 0; r < np; ++r) {
+        if (s_state[r] == kHit) continue;
+        const int npg = (s_tokens[r] + kPageTokens - 1) / kPageTokens;
+        if (npg <= (int)run_free - used) { s_missoff[r] = used; used += npg; }
+        else s_state[r] = kBypass;
+      }
+      sh.demand = used;
+    }
+  } else if (tid == 0) sh.demand = demand;
+  __syncthreads();
+  if (tid == 0) sh.qbase = (sh.demand > 0 && c.fetch_mode != 0) ? atomicAdd(c.fetch_count, sh.demand) : 0;
+  __syncthreads();
+  const int qbase = sh.qbase;
+
+  for (int r = tid; r < np; r += T) {
+    c.part_state[(size_t)b * c.max_parts + r] = s_state[r];
+    if (s_state[r] == kAdmit) {
+      MetaEntry *m = meta_at(c, set, s_parts[r]);
+      if (m) m->resident = 1;
+    }
+  }
+  int my_admit = 0, my_bypass = 0;
+  for (int idx = tid; idx < total_pages; idx += T) {
+    const int r = owner_of(s_pageoff, np, idx);
+    const int i = idx - s_pageoff[r], p = s_parts[r], state = s_state[r];
+    const int valid = min(kPageTokens, s_tokens[r] - i * kPageTokens);
+    page_mask[idx] = c.kind == kKindToken ? c.part_mask[(size_t)b * c.max_parts + r]
+                                           : ((1u << valid) - 1u);
+    page_part[idx] = p;
+    page_pidx[idx] = i;
+    page_fill[idx] = -1;
+    // work order of the attention kernel: pages that cross the host link first, so that all
+    // of them are requested by the first CTAs and overlap the hits' HBM traffic
+    const int pos = state == kHit ? demand + (s_pageoff[r] - s_missbefore[r]) + i : s_missbefore[r] + i;
+    if (state == kHit) { page_desc[pos] = make_int4(page_src[idx], -1, (int)page_mask[idx], idx); continue; }
+    // lookup step 3: Partition Offset -> slice of the CPU page table (pinned host memory)
+    const int mi = s_missbefore[r] + i;
+    int host_page = mi < T ? sh.hostpage[mi] : -1;
+    const int32_t *hp = &host_page;
+    if (host_page < 0) {                       // beyond the early batch (or it failed): look up now
+      const int32_t *off = off_at(c, set, p);
+      hp = off ? cpt_at(c, set, *off + i) : nullptr;
+      if (hp) host_page = *hp;
+    }
+    if (!hp) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
+    if (state == kAdmit) {
+      const int slot = s_free[s_missoff[r] + i];
+      GptEntry *e = gpt_at(c, set, slot);
+      const int phys = e->phys;
+      e->partition = p;
+      e->page_idx = i;
+      e->ts = top;
+      page_src[idx] = phys;
+      page_slot[idx] = slot;
+      if (c.fetch_mode == 0) {
+        page_fill[idx] = host_page;               // the attention kernel brings it in
+      } else {
+        const int qi = qbase + s_missoff[r] + i;
+        if (qi < c.fetch_cap) c.fetch_queue[qi] = FetchItem{host_page, phys};
+        else dev_error(c, kErrBounds);
+      }
+      page_desc[pos] = make_int4(phys, page_fill[idx], (int)page_mask[idx], idx);
+      ++my_admit;
+    } else {
+      page_src[idx] = ~host_page;
+      page_slot[idx] = -1;
+      page_desc[pos] = make_int4(~host_page, -1, (int)page_mask[idx], idx);
+      ++my_bypass;
+    }
+  }
+  if (my_admit) atomicAdd(&sh.admit_pages, my_admit);
+  if (my_bypass) atomicAdd(&sh.bypass_pages, my_bypass);
+
+  // ---- local tail: always attended -------------------------------------------------------
+  for (int j = tid; j < tail_pages; j += T) {
+    const int idx = total_pages + j;
+    page_src[idx] = c.tail_phys[(size_t)set * c.tail_cap + j];
+    page_mask[idx] = j == tail_pages - 1 ? ((1u << tail_len) - 1u) : 0xffffu;
+    page_slot[idx] = -2;
+    page_fill[idx] = -1;
+    page_desc[idx] = make_int4(page_src[idx], -1, (int)page_mask[idx], idx);
+    page_part[idx] = -1;
+    page_pidx[idx] = j;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    c.n_pages[b] = total_pages + tail_pages;
+    c.n_parts[b] = np;
+    c.state[set].step = t + 1;
+    Counters *k = c.counters;
+    const int miss_pages = sh.admit_pages + sh.bypass_pages;
+    atomicAdd(&k->set_steps, 1ull);
+    atomicAdd(&k->selected_partitions, (unsigned long long)np);
+    atomicAdd(&k->selected_pages, (unsigned long long)total_pages);
+    atomicAdd(&k->tail_pages, (unsigned long long)tail_pages);
+    atomicAdd(&k->hit_pages, (unsigned long long)(total_pages - miss_pages));
+    atomicAdd(&k->miss_pages, (unsigned long long)miss_pages);
+    atomicAdd(&k->evicted_pages, (unsigned long long)sh.evicted);
+    atomicAdd(&k->bypass_pages, (unsigned long long)sh.bypass_pages);
+    flag_publish(c.ready + b, epoch);            // attention may start on this set
+  }
+}
+
+}  // namespace spin
