@@ -96,6 +96,11 @@ typedef struct spin_config {
   int32_t fetch_mode;           /* 0: missed pages are fetched inside the attention kernel (they
                                    cross the host link while the hits are attended from HBM);
                                    1: by a separate persistent warp-per-page copy kernel */
+  int32_t host_tables_only;     /* 0: the decode kernels read the Partition Offset and CPU page
+                                   tables through an HBM mirror (4 B per entry) that the append
+                                   kernels keep up to date; 1: they read the pinned host tables
+                                   over the host link, as in Section 5.2 (saves the mirror's HBM,
+                                   but those small reads queue behind the page traffic) */
   int64_t gpu_cache_pages;      /* HBM pages (8 KiB each) shared by all sets' cache slots */
   int64_t host_pages;           /* pinned host pages (8 KiB each) for the complete KV */
   void *hbm_pool;               /* device pointer, 256-byte aligned, caller-owned */

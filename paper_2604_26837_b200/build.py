@@ -39,7 +39,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src in SOURCES:
         s, o = os.path.join(CSRC, src), os.path.join(OBJ, src[:-3] + ".o")
         if force or _stale(o, [s] + headers):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            extra = ["-DSPIN_TIMING"] if os.environ.get("SPIN_TIMING") else []
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):

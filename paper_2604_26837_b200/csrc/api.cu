@@ -54,6 +54,7 @@ struct SetHost {                     // host mirror of one (request, layer, kv h
 
 struct LayerHost {                   // counts shared by the kv-head sets of (request, layer)
   int64_t n_tokens = 0;
+  int32_t steps = 0;                 // decode steps done
   int32_t n_partitions = 0, n_host_pages = 0, tail_first = 0, tail_pages = 0, tail_len = 0;
   bool clustered = false;
   int32_t last_batch_pos = -1;
@@ -197,6 +198,10 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.summaries = a.take<uint8_t>((size_t)g.n_sum_segs * g.sum_entries * g.sum_entry_bytes);
   d.meta_pool = a.take<MetaEntry>((size_t)g.n_meta_segs * g.seg);
   d.gpt_pool = a.take<GptEntry>((size_t)g.n_gpt_segs * g.seg);
+  if (!cfg.host_tables_only) {
+    d.off_mirror = a.take<int32_t>((size_t)g.n_off_segs * g.seg);
+    d.cpt_mirror = a.take<int32_t>((size_t)g.n_cpt_segs * g.seg);
+  }
   d.state = a.take<SetState>((size_t)g.n_sets);
   d.dir_meta = a.take<int32_t>((size_t)g.n_sets * g.dir_part);
   d.dir_off = a.take<int32_t>((size_t)g.n_sets * g.dir_part);
@@ -452,6 +457,16 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
     s.tail_first = total_pages_max;
     s.n_host_pages = total_pages_max;
     CK(cudaMemcpy(d.state + set, &s, sizeof s, cudaMemcpyHostToDevice));
+  }
+  // the decode kernels read the two host tables through their HBM mirror
+  if (d.off_mirror) {
+    for (int h = 0; h < H; ++h) {
+      const SetHost &S = set_of(ctx, req, layer, h);
+      for (int32_t seg : S.dir_off)
+        if (seg >= 0) CK(cudaMemcpyAsync(d.off_mirror + ((size_t)seg << g.seg_shift), ctx->h_off_pool + ((size_t)seg << g.seg_shift), (size_t)g.seg * 4, cudaMemcpyHostToDevice, st));
+      for (int32_t seg : S.dir_cpt)
+        if (seg >= 0) CK(cudaMemcpyAsync(d.cpt_mirror + ((size_t)seg << g.seg_shift), ctx->h_cpt_pool + ((size_t)seg << g.seg_shift), (size_t)g.seg * 4, cudaMemcpyHostToDevice, st));
+    }
   }
   // destination row of every (token, head): clusters keep their tokens in arrival order
   std::vector<int32_t> filled((size_t)H * C, 0);
@@ -904,6 +919,9 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     L.last_batch_pos = i;
     b.tail_pages[i] = (int16_t)L.tail_pages;
     b.tail_len[i] = (int16_t)L.tail_len;
+    b.slots[i] = (int32_t)ctx->reqs[(size_t)req_ids[i]].slots;
+    b.step[i] = L.steps++;
+    b.n_partitions[i] = L.n_partitions;
   }
   const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
   const __nv_bfloat16 *qd = reinterpret_cast<const __nv_bfloat16 *>(q);
@@ -959,7 +977,8 @@ int spin_stats(spin_ctx *ctx, spin_stats_t *out) {
                    (c.miss_pages - c.bypass_pages) * (uint64_t)kPageBytes;
   out->kernel_launches = ctx->launches;
   out->gpu_meta_bytes = (uint64_t)ctx->gpt_segs.in_use * g.seg * sizeof(GptEntry) +
-                        (uint64_t)ctx->meta_segs.in_use * g.seg * sizeof(MetaEntry) + ctx->dir_bytes_in_use;
+                        (uint64_t)ctx->meta_segs.in_use * g.seg * sizeof(MetaEntry) + ctx->dir_bytes_in_use +
+                        (ctx->d.off_mirror ? (uint64_t)(ctx->off_segs.in_use + ctx->cpt_segs.in_use) * g.seg * 4 : 0);
   out->host_meta_bytes = (uint64_t)(ctx->off_segs.in_use + ctx->cpt_segs.in_use) * g.seg * 4;
   out->summary_bytes = (uint64_t)ctx->sum_segs.in_use * g.sum_entries * g.sum_entry_bytes;
   out->gpu_pages_in_use = (uint64_t)ctx->gpu_page_pool.in_use;

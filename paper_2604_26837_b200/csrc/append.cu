@@ -24,7 +24,9 @@ k_append_bulk(DevCtx c, int req, int layer, const __nv_bfloat16 *__restrict__ k,
   uint4 vv = ld16(reinterpret_cast<const uint8_t *>(v) + in_off);
   const int32_t *hp = cpt_at(c, set, page);
   if (!hp) { if (tid == 0) dev_error(c, 1u); return; }
-  uint8_t *dst = c.host_pages + (size_t)(*hp) * kPageBytes + r * kRowBytes + piece * 16;
+  const int32_t host_page = *hp;
+  if (tid == 0) cpt_mirror_set(c, set, page, host_page);
+  uint8_t *dst = c.host_pages + (size_t)host_page * kPageBytes + r * kRowBytes + piece * 16;
   st16(dst, kk);
   st16(dst + kHalfPageBytes, vv);
   st16(reinterpret_cast<uint8_t *>(krows[r]) + piece * 16, kk);

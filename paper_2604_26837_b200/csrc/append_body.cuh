@@ -44,6 +44,7 @@ __device__ __forceinline__ void index_page(const DevCtx &c, int set, int part,
   if (tid == 0) {
     MetaEntry *m = meta_at(c, set, part);
     if (m) { m->tokens = kPageTokens; m->resident = 0; } else dev_error(c, 1u);
+    off_mirror_set(c, set, part, part);          // page-sized kinds: partition p starts at page p
   }
 }
 
@@ -128,9 +129,11 @@ __device__ __forceinline__ void append_edge_body(const DevCtx &c, int set, int i
       uint4 kk = ld16(kin + in_off(tok)), vv = ld16(vin + in_off(tok));
       const int32_t *hp = cpt_at(c, set, j_end);
       if (hp) {
-        uint8_t *dst = c.host_pages + (size_t)(*hp) * kPageBytes + r * kRowBytes + piece * 16;
+        const int32_t host_page = *hp;
+        uint8_t *dst = c.host_pages + (size_t)host_page * kPageBytes + r * kRowBytes + piece * 16;
         st16(dst, kk);
         st16(dst + kHalfPageBytes, vv);
+        if (piece == 0 && r == lo) cpt_mirror_set(c, set, j_end, host_page);
       } else if (piece == 0) dev_error(c, 1u);
       st16(tail + r * kRowBytes + piece * 16, kk);
       st16(tail + kHalfPageBytes + r * kRowBytes + piece * 16, vv);

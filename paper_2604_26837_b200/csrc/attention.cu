@@ -21,6 +21,13 @@
 
 namespace spin {
 
+#ifdef SPIN_TIMING
+__device__ unsigned long long g_dbg_ta[256][16];
+__device__ __forceinline__ void dbg_ta(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ta[b & 255][slot] = t; } }
+#else
+__device__ __forceinline__ void dbg_ta(int, int) {}
+#endif
+
 namespace {
 
 constexpr int kAttnWarps = 4;
@@ -162,6 +169,7 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   } else {
     pdl_wait_prev();
   }
+  if (chunk == 0) dbg_ta(b, 10);
   const int np = c.n_pages[b];
   const int first = chunk * kChunkPages;
   if (first >= np) return;
@@ -179,6 +187,17 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
     if (c.page_desc) {                      // work-ordered descriptors written by the cache manager
       const int4 dsc = c.page_desc[pl + pg[i]];
       src[i] = dsc.x; fill[i] = dsc.y; mask[i] = (uint32_t)dsc.z;
+      if (fill[i] == -2) {
+        // Retrieve step 3 for a missed page: Partition Offset -> CPU page table, both in pinned
+        // host memory (two dependent reads over the host link, all lanes read the same words)
+        const int set = set_index(c, bt.req[i_req], bt.layer, head);
+        const int32_t *off = off_lookup(c, set, c.page_part[pl + dsc.w]);
+        const int32_t *hp = off ? cpt_lookup(c, set, *off + c.page_pidx[pl + dsc.w]) : nullptr;
+        const int host_page = hp ? *hp : -1;
+        if (host_page < 0) { src[i] = -1; fill[i] = c.n_host_pages; }       // fails the range check below
+        else if (src[i] >= 0) fill[i] = host_page;                          // admitted: fetch into slot src
+        else { src[i] = ~host_page; fill[i] = -1; }                         // bypassed: attend from host
+      }
     } else {                                // plain lists, attended in the order given
       src[i] = c.page_src[pl + pg[i]];
       mask[i] = c.page_mask[pl + pg[i]];
@@ -192,6 +211,7 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
     t = fill[0]; fill[0] = fill[1]; fill[1] = t;
     uint32_t u = mask[0]; mask[0] = mask[1]; mask[1] = u;
   }
+  if (chunk == 0) dbg_ta(b, 11);
   uint8_t *spage[2] = {smem_pages + (size_t)(2 * warp) * kPageBytes, smem_pages + (size_t)(2 * warp + 1) * kPageBytes};
   for (int i = 0; i < 2; ++i) {
     if (i < n_mine) {
@@ -221,12 +241,14 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
 
   cp_async_wait<1>();
   __syncwarp();
+  if (chunk == 0) dbg_ta(b, 12);
   if (n_mine >= 1) {
     attend_page(smem_u32(spage[0]), qa, mask[0], scale2, acc, lane);
     if (fill[0] >= 0) store_page(spage[0], c.gpu_pages + (size_t)src[0] * kPageBytes, lane);
   }
   cp_async_wait<0>();
   __syncwarp();
+  if (chunk == 0) dbg_ta(b, 13);
   if (n_mine >= 2) {
     attend_page(smem_u32(spage[1]), qa, mask[1], scale2, acc, lane);
     if (fill[1] >= 0) store_page(spage[1], c.gpu_pages + (size_t)src[1] * kPageBytes, lane);
@@ -277,6 +299,7 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   if (threadIdx.x == 0) sh_last = atomicAdd(&c.att_count[b], 1) == n_chunks - 1;
   __syncthreads();
   if (!sh_last) return;
+  dbg_ta(b, 14);
   __threadfence();
   // merge: the per-chunk (max, sum) pairs first, then the outputs, with the loads of a batch
   // of chunks issued together
@@ -462,3 +485,10 @@ extern "C" int spin_paged_attention_static(const void *q, const void *page_pool,
   }
   return SPIN_OK;
 }
+
+#ifdef SPIN_TIMING
+extern "C" __attribute__((visibility("default"))) int spin_debug_timestamps_attn(unsigned long long *out) {
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpyFromSymbol(out, spin::g_dbg_ta, sizeof(unsigned long long) * 256 * 16);
+}
+#endif

@@ -70,9 +70,9 @@ __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, con
 }
 
 template <int G, bool MINMAX>
-__global__ void __launch_bounds__(kScoreThreads)
+__global__ void __launch_bounds__(kScoreThreads, 3)
 k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
-        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap) {
+        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap) {   // fuse: 0 none, 1 staged, 2 fast
   extern __shared__ __align__(16) uint8_t dyn_smem[];      // used by the fused continuation only
   const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
@@ -88,6 +88,7 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
     if (threadIdx.x == 0) flag_publish(c.tail_ready + b, bt.epoch);
     return;
   }
+  if (blockIdx.x == 0) dbg_ts(b, 0);
   const SetState st = c.state[set];
   const int n_cand = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
   const int seg_entries = 1 << c.sum_shift;
@@ -120,38 +121,64 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
   const uint8_t *base = c.summaries + ((size_t)seg << c.sum_shift) * kEntry + lane16 * 16;
   float *out = c.scores + (size_t)b * c.max_cand + e0;
 
-  // two entries per half-warp and iteration, all their loads issued before any arithmetic
-  for (int e = grp; e < n_here; e += 32) {
-    const bool two = e + 16 < n_here;
-    const uint4 z = make_uint4(0, 0, 0, 0);
-    const uint4 a0 = ld_stream16(base + (size_t)e * kEntry);
-    const uint4 m0 = MINMAX ? ld_stream16(base + (size_t)e * kEntry + kRowBytes) : z;
-    const uint4 a1 = two ? ld_stream16(base + (size_t)(e + 16) * kEntry) : z;
-    const uint4 m1 = (MINMAX && two) ? ld_stream16(base + (size_t)(e + 16) * kEntry + kRowBytes) : z;
-    const float s0 = score_entry<G, MINMAX>(a0, m0, qf, qsel, row_mask);
-    if (lane16 == 0) out[e] = s0;
-    if (two) {
-      const float s1 = score_entry<G, MINMAX>(a1, m1, qf, qsel, row_mask);
-      if (lane16 == 0) out[e + 16] = s1;
+  // Every lane requests, up front, the 16-byte pieces it will itself consume (cp.async into a
+  // per-CTA staging area, four groups per lane), then scores group by group as they land.
+  // A lane only ever reads what it copied, so waiting on its own groups is all the
+  // synchronisation there is, and a CTA keeps its whole 64 KiB segment in flight.
+  constexpr int kPerHalfWarp = MINMAX ? 8 : 16;          // entries of the segment per half-warp
+  constexpr int kPerGroup = kPerHalfWarp / 4;            // entries per cp.async group
+  uint8_t *stage = dyn_smem + (size_t)grp * kPerHalfWarp * kEntry + lane16 * 16;
+#pragma unroll
+  for (int gI = 0; gI < 4; ++gI) {
+#pragma unroll
+    for (int j = 0; j < kPerGroup; ++j) {
+      const int slot = gI * kPerGroup + j, e = grp + 16 * slot;
+      if (e < n_here) {
+        cp_async16_ca(stage + (size_t)slot * kEntry, base + (size_t)e * kEntry);
+        if (MINMAX) cp_async16_ca(stage + (size_t)slot * kEntry + kRowBytes, base + (size_t)e * kEntry + kRowBytes);
+      }
+    }
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+  }
+#pragma unroll
+  for (int gI = 0; gI < 4; ++gI) {
+    if (gI == 0) asm volatile("cp.async.wait_group 3;\n" ::: "memory");
+    else if (gI == 1) asm volatile("cp.async.wait_group 2;\n" ::: "memory");
+    else if (gI == 2) asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < kPerGroup; ++j) {
+      const int slot = gI * kPerGroup + j, e = grp + 16 * slot;
+      if (e < n_here) {
+        const uint4 a0 = *reinterpret_cast<const uint4 *>(stage + (size_t)slot * kEntry);
+        const uint4 m0 = MINMAX ? *reinterpret_cast<const uint4 *>(stage + (size_t)slot * kEntry + kRowBytes)
+                                : make_uint4(0, 0, 0, 0);
+        const float s0 = score_entry<G, MINMAX>(a0, m0, qf, qsel, row_mask);
+        if (lane16 == 0) out[e] = s0;
+      }
     }
   }
   }
   if (!fuse) return;
 
   // ---- fused continuation: the last CTA of the set to arrive selects and manages the cache ----
-  __shared__ TopkShared tsh;
-  __shared__ CacheShared csh;
+  __shared__ union { struct { TopkShared t; CacheShared c; } staged; FastShared fast; } shm;
   __shared__ int s_last;
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) s_last = atomicAdd(&c.sel_count[b], 1) == segs_here - 1;
   __syncthreads();
   if (!s_last) return;
+  dbg_ts(b, 9);
   __threadfence();
   if (threadIdx.x == 0) c.sel_count[b] = 0;                 // ready for the next step
-  topk_stage<kScoreThreads, false>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh);
+  if (fuse == 2) {
+    select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, shm.fast);
+    return;
+  }
+  topk_stage<kScoreThreads, false>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, shm.staged.t);
   cache_stage<kScoreThreads>(c, b, set, __ldcg(c.n_parts + b), bt.tail_pages[i_req], bt.tail_len[i_req],
-                             bt.epoch, reinterpret_cast<int32_t *>(dyn_smem), csh);
+                             bt.epoch, reinterpret_cast<int32_t *>(dyn_smem), shm.staged.c);
 }
 
 // Stand-alone top-k: one thread-block cluster per set (slices of the keys in shared memory).
@@ -193,10 +220,17 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
   dim3 grid(segs + 1, n_sets);                    // + one tail CTA per set (in-grid append, tail flag)
   // fused: one CTA can hold a set's keys and the cache manager's tables in shared memory
   const size_t cache_smem = cache_stage_smem_bytes(c.max_parts, c.max_pages, c.max_slots);
-  const bool fuse = max_cand <= 16384 && cache_smem <= 96 * 1024;
+  int fuse = (max_cand <= 16384 && cache_smem <= 96 * 1024) ? 1 : 0;
   const int keys_cap = fuse ? max_cand : 0;
   size_t smem = 0;
   if (fuse) smem = cache_smem > (size_t)keys_cap * 4 ? cache_smem : (size_t)keys_cap * 4;
+  if (fuse && c.kind != kKindToken) {
+    int max_slots_batch = 0;
+    for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
+    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
+    if (max_slots_batch <= kFastSlots && fs <= 64 * 1024) { fuse = 2; smem = fs > smem ? fs : smem; }
+  }
+  if (smem < 64 * 1024) smem = 64 * 1024;         // the scoring CTAs' staging area: one summary segment
   switch (c.G) {
     case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
     case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
@@ -221,3 +255,10 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
 }
 
 }  // namespace spin
+
+#ifdef SPIN_TIMING
+extern "C" __attribute__((visibility("default"))) int spin_debug_timestamps(unsigned long long *out) {
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpyFromSymbol(out, spin::g_dbg_ts, sizeof(unsigned long long) * 256 * 16);
+}
+#endif

@@ -71,6 +71,8 @@ struct DevCtx {
   GptEntry *gpt_pool;           // GPU
   int32_t *off_pool;            // pinned host: Partition Offset table segments
   int32_t *cpt_pool;            // pinned host: CPU page table segments
+  int32_t *off_mirror;          // HBM copies of the two host tables (same segment layout), or null:
+  int32_t *cpt_mirror;          //   what the decode kernels read, kept up to date by the append kernels
   // per set
   SetState *state;
   int32_t *dir_meta, *dir_gpt, *dir_off, *dir_cpt, *dir_sumseg;
@@ -114,6 +116,11 @@ struct Batch {
   // the cache manager lay out the page list without waiting for the append kernel
   int16_t tail_pages[kMaxBatch];
   int16_t tail_len[kMaxBatch];
+  // what the host knows of every request's sets without asking the device (all kv heads of a
+  // request and layer agree): GPU slots, decode steps done, indexed partitions
+  int32_t slots[kMaxBatch];
+  int32_t step[kMaxBatch];
+  int32_t n_partitions[kMaxBatch];
   int32_t epoch;            // number of this decode call: value of the ready flags it sets
   int32_t append_in_grid;   // the scoring kernel's tail CTAs append this step's tokens
 };
@@ -143,6 +150,28 @@ __device__ __forceinline__ int32_t *off_at(const DevCtx &c, int set, int p) {
 __device__ __forceinline__ int32_t *cpt_at(const DevCtx &c, int set, int i) {
   int seg = c.dir_cpt[(size_t)set * c.dir_page + (i >> c.seg_shift)];
   return seg < 0 ? nullptr : c.cpt_pool + ((size_t)seg << c.seg_shift) + (i & ((1 << c.seg_shift) - 1));
+}
+// Lookups for the decode path: the HBM mirror when there is one, else the pinned host table.
+__device__ __forceinline__ const int32_t *off_lookup(const DevCtx &c, int set, int p) {
+  int seg = c.dir_off[(size_t)set * c.dir_part + (p >> c.seg_shift)];
+  if (seg < 0) return nullptr;
+  return (c.off_mirror ? c.off_mirror : c.off_pool) + ((size_t)seg << c.seg_shift) + (p & ((1 << c.seg_shift) - 1));
+}
+__device__ __forceinline__ const int32_t *cpt_lookup(const DevCtx &c, int set, int i) {
+  int seg = c.dir_cpt[(size_t)set * c.dir_page + (i >> c.seg_shift)];
+  if (seg < 0) return nullptr;
+  return (c.cpt_mirror ? c.cpt_mirror : c.cpt_pool) + ((size_t)seg << c.seg_shift) + (i & ((1 << c.seg_shift) - 1));
+}
+// Append-side helpers: record an entry of a host table in its HBM mirror.
+__device__ __forceinline__ void off_mirror_set(const DevCtx &c, int set, int p, int32_t v) {
+  if (!c.off_mirror) return;
+  int seg = c.dir_off[(size_t)set * c.dir_part + (p >> c.seg_shift)];
+  if (seg >= 0) c.off_mirror[((size_t)seg << c.seg_shift) + (p & ((1 << c.seg_shift) - 1))] = v;
+}
+__device__ __forceinline__ void cpt_mirror_set(const DevCtx &c, int set, int i, int32_t v) {
+  if (!c.cpt_mirror) return;
+  int seg = c.dir_cpt[(size_t)set * c.dir_page + (i >> c.seg_shift)];
+  if (seg >= 0) c.cpt_mirror[((size_t)seg << c.seg_shift) + (i & ((1 << c.seg_shift) - 1))] = v;
 }
 __device__ __forceinline__ uint8_t *summary_at(const DevCtx &c, int set, int e) {
   int seg = c.dir_sumseg[(size_t)set * c.dir_sum + (e >> c.sum_shift)];

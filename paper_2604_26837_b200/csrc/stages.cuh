@@ -72,6 +72,12 @@ __device__ __forceinline__ int owner_of(const int32_t *off, int n, int idx) {
   return lo;
 }
 
+// The cache manager resolves the CPU page ids of missed pages itself when the copy kernel needs
+// them (fetch_mode 1) or when they are one HBM read away (mirror); when they are only in pinned
+// host memory and the fetch is fused into attention, the fetching warp looks them up instead,
+// so that a set's page list never waits on the host link.
+__device__ __forceinline__ bool resolve_in_manager(const DevCtx &c) { return c.fetch_mode != 0 || c.cpt_mirror != nullptr; }
+
 struct TopkShared {
   uint32_t hist[256];          // this CTA's histogram (read remotely inside a cluster)
   uint32_t ghist[256];         // histogram over the whole set
@@ -341,10 +347,10 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
   // missed pages live in pinned host memory, two dependent reads over the host link.  They
   // are issued here and consumed after the table scans below, which hides their latency.
   int early_i = 0, early_off = -1, early_host = -1;
-  if (tid < demand && np > 0) {
+  if (resolve_in_manager(c) && tid < demand && np > 0) {
     const int r = owner_of(s_missbefore, np, tid);
     early_i = tid - s_missbefore[r];
-    const int32_t *off = off_at(c, set, s_parts[r]);
+    const int32_t *off = off_lookup(c, set, s_parts[r]);
     if (off) early_off = *off;
   }
 
@@ -375,7 +381,7 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
   __syncthreads();
 
   if (early_off >= 0) {
-    const int32_t *hp = cpt_at(c, set, early_off + early_i);
+    const int32_t *hp = cpt_lookup(c, set, early_off + early_i);
     if (hp) early_host = *hp;
   }
 
@@ -470,14 +476,18 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
     if (state == kHit) { page_desc[pos] = make_int4(page_src[idx], -1, (int)page_mask[idx], idx); continue; }
     // lookup step 3: Partition Offset -> slice of the CPU page table (pinned host memory)
     const int mi = s_missbefore[r] + i;
-    int host_page = mi < T ? sh.hostpage[mi] : -1;
-    const int32_t *hp = &host_page;
-    if (host_page < 0) {                       // beyond the early batch (or it failed): look up now
-      const int32_t *off = off_at(c, set, p);
-      hp = off ? cpt_at(c, set, *off + i) : nullptr;
-      if (hp) host_page = *hp;
+    // with the fetch fused into attention the fetching warp resolves the CPU page id itself
+    // (fill = -2); otherwise it is resolved here, from the early batch where possible
+    int host_page = -2;
+    if (resolve_in_manager(c)) {
+      host_page = mi < T ? sh.hostpage[mi] : -1;
+      if (host_page < 0) {
+        const int32_t *off = off_lookup(c, set, p);
+        const int32_t *hp = off ? cpt_lookup(c, set, *off + i) : nullptr;
+        if (hp) host_page = *hp;
+      }
+      if (host_page < 0) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
     }
-    if (!hp) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
     if (state == kAdmit) {
       const int slot = s_free[s_missoff[r] + i];
       GptEntry *e = gpt_at(c, set, slot);
@@ -488,7 +498,7 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
       page_src[idx] = phys;
       page_slot[idx] = slot;
       if (c.fetch_mode == 0) {
-        page_fill[idx] = host_page;               // the attention kernel brings it in
+        page_fill[idx] = host_page;               // the attention kernel brings it in (-2: and looks it up)
       } else {
         const int qi = qbase + s_missoff[r] + i;
         if (qi < c.fetch_cap) c.fetch_queue[qi] = FetchItem{host_page, phys};
@@ -497,9 +507,10 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
       page_desc[pos] = make_int4(phys, page_fill[idx], (int)page_mask[idx], idx);
       ++my_admit;
     } else {
-      page_src[idx] = ~host_page;
+      page_src[idx] = host_page == -2 ? -1 : ~host_page;
       page_slot[idx] = -1;
-      page_desc[pos] = make_int4(~host_page, -1, (int)page_mask[idx], idx);
+      page_desc[pos] = host_page == -2 ? make_int4(-1, -2, (int)page_mask[idx], idx)
+                                       : make_int4(~host_page, -1, (int)page_mask[idx], idx);
       ++my_bypass;
     }
   }
@@ -534,6 +545,425 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
     atomicAdd(&k->bypass_pages, (unsigned long long)sh.bypass_pages);
     flag_publish(c.ready + b, epoch);            // attention may start on this set
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Fast path of the fused continuation: top-k + cache manager of one set by one CTA, for sets
+// whose candidate keys and GPU page table both fit in shared memory (partition and cluster
+// granularity, up to kFastSlots slots).  Same results as topk_stage + cache_stage; what differs
+// is latency: the directories and the whole GPU page table are brought into shared memory by
+// cp.async while the radix select runs, the compaction and the free-slot scan need one block
+// scan each, and the page table is written back once at the end.  The time this takes is the
+// time before the set's missed pages can start to cross the host link.
+constexpr int kFastSlots = 1024;
+
+#ifdef SPIN_TIMING
+__device__ unsigned long long g_dbg_ts[256][16];
+__device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; } }
+#else
+__device__ __forceinline__ void dbg_ts(int, int) {}
+#endif
+
+struct FastShared {
+  uint32_t hist[2][256];
+  uint32_t wsum[33];
+  uint32_t lhist[kMaxBuckets + 2];
+  uint32_t prefix, remaining;
+  int x, demand, evicted, qbase, admit_pages, bypass_pages;
+};
+
+__host__ __device__ inline size_t fast_smem_bytes(int n_keys, int slots, int dir_part, int dir_slot,
+                                                  int max_parts, int max_pages) {
+  size_t b = (size_t)((n_keys + 3) / 4 * 4) * 4;                 // keys
+  b += (size_t)slots * 16;                                       // GPU page table copy
+  b += (size_t)((dir_part + dir_slot + 3) / 4 * 4) * 4;          // directories
+  b += (size_t)(6 * max_parts + 4 + 2 * max_pages) * 4;          // cache manager tables, free list, host ids
+  b += (size_t)((slots + 31) / 32 + 4) * 4;                      // hit bitmask
+  return b + 64;
+}
+
+__device__ __forceinline__ void cp_async4(void *smem_dst, const void *gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async16_ca(void *smem_dst, const void *gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_wait_all() {
+  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+}
+
+template <int T>
+__device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
+                                            uint8_t *dyn, FastShared &sh) {
+  const int tid = threadIdx.x;
+  const int n = bt.n_partitions[i_req];
+  const int k = min(c.topk, n);
+  const int S = bt.slots[i_req], t = bt.step[i_req], nb = c.n_buckets, top = min(t, nb - 1);
+  const int tail_pages = bt.tail_pages[i_req], tail_len = bt.tail_len[i_req];
+  const int seg_mask = (1 << c.seg_shift) - 1;
+  const int n_gdir = (S + seg_mask) >> c.seg_shift;
+
+  // ---- shared memory layout -----------------------------------------------------------------
+  uint32_t *s_keys = reinterpret_cast<uint32_t *>(dyn);
+  int4 *s_gpt = reinterpret_cast<int4 *>(s_keys + (n + 3) / 4 * 4);
+  int32_t *s_mdir = reinterpret_cast<int32_t *>(s_gpt + S);
+  int32_t *s_gdir = s_mdir + c.dir_part;
+  int32_t *s_parts = s_mdir + (c.dir_part + c.dir_slot + 3) / 4 * 4;
+  int32_t *s_tokens = s_parts + c.max_parts;
+  int32_t *s_pageoff = s_tokens + c.max_parts;        // [max_parts + 1]
+  int32_t *s_missoff = s_pageoff + c.max_parts + 1;
+  int32_t *s_missbefore = s_missoff + c.max_parts;
+  int32_t *s_state = s_missbefore + c.max_parts;
+  int32_t *s_free = s_state + c.max_parts + 3;        // [max_pages]
+  int32_t *s_host = s_free + c.max_pages;             // [max_pages] CPU page ids of missed pages
+  uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_host + c.max_pages);
+
+  dbg_ts(b, 1);
+  // ---- directories on their way (consumed after the keys are loaded) ------------------------
+  for (int i = tid; i < c.dir_part; i += T) cp_async4(s_mdir + i, c.dir_meta + (size_t)set * c.dir_part + i);
+  for (int i = tid; i < n_gdir; i += T) cp_async4(s_gdir + i, c.dir_gpt + (size_t)set * c.dir_slot + i);
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+
+  const float *scores = c.scores + (size_t)b * c.max_cand;
+  for (int i = tid; i < n; i += T) s_keys[i] = order_key(__ldcg(scores + i));
+  for (int i = tid; i < 512; i += T) (&sh.hist[0][0])[i] = 0;
+  if (tid == 0) {
+    c.n_sel[b] = k;
+    c.att_count[b] = 0;
+    atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
+    sh.evicted = 0; sh.admit_pages = 0; sh.bypass_pages = 0;
+  }
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+  __syncthreads();
+
+  dbg_ts(b, 2);
+  // ---- the GPU page table on its way (consumed after top-k) ---------------------------------
+  for (int s_ = tid; s_ < S; s_ += T) {
+    const int seg = s_gdir[s_ >> c.seg_shift];
+    if (seg >= 0) cp_async16_ca(s_gpt + s_, c.gpt_pool + ((size_t)seg << c.seg_shift) + (s_ & seg_mask));
+    else { dev_error(c, kErrBounds); s_gpt[s_] = make_int4(-1, 0, 0, -1); }
+  }
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+
+  // ---- top-k: radix select (two barriers per pass), one-scan ordered compaction -------------
+  int32_t *g_sel = c.sel_ids + (size_t)b * c.max_sel;
+  int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
+  if (k == n) {
+    for (int i = tid; i < n; i += T) { s_parts[i] = i; g_sel[i] = i; g_parts[i] = i; }
+  } else {
+    uint32_t prefix = 0, mask = 0, remaining = k;
+    int buf = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, buf ^= 1) {
+      for (int i = tid; i < n; i += T) {
+        const uint32_t key = s_keys[i];
+        if ((key & mask) == prefix) atomicAdd(&sh.hist[buf][(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid < 32) {
+        uint32_t loc[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { loc[j] = sh.hist[buf][255 - 8 * tid - j]; sum += loc[j]; }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += v;
+        }
+        const uint32_t before = inc - sum;
+        if (before < remaining && inc >= remaining) {
+          uint32_t cum = before;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (cum < remaining && cum + loc[j] >= remaining) {
+              sh.prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
+              sh.remaining = remaining - cum;
+            }
+            cum += loc[j];
+          }
+        }
+      } else {
+        for (int i = tid - 32; i < 256; i += T - 32) sh.hist[buf ^ 1][i] = 0;   // for the pass after next
+      }
+      __syncthreads();
+      prefix = sh.prefix;
+      remaining = sh.remaining;
+      mask |= 255u << shift;
+      // the buffer just searched is cleared by the next pass's idle warps (it is used again two passes on)
+    }
+    const uint32_t thr = prefix, need_eq = remaining;
+    const int E = (n + T - 1) / T, lo = min(n, tid * E), hi = min(n, lo + E);
+    uint32_t gt = 0, eq = 0;
+    for (int i = lo; i < hi; ++i) { const uint32_t key = s_keys[i]; gt += key > thr; eq += key == thr; }
+    uint32_t total;
+    const uint32_t ex = block_scan<T>(gt | (eq << 16), sh.wsum, &total);
+    uint32_t gt_before = ex & 0xffffu, eq_before = ex >> 16;
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t key = s_keys[i];
+      if (key > thr || (key == thr && eq_before < need_eq)) {
+        const uint32_t pos = gt_before + min(eq_before, need_eq);
+        s_parts[pos] = i; g_sel[pos] = i; g_parts[pos] = i;
+      }
+      gt_before += key > thr;
+      eq_before += key == thr;
+    }
+  }
+  dbg_ts(b, 3);
+  const int np_sel = k;
+  __syncthreads();
+
+  // ---- cache manager step 1: Meta-partition lookups, classification, page demand ------------
+  int np = np_sel;
+  uint32_t run_all = 0, run_miss = 0;
+  for (int base = 0; base < np; base += T) {
+    const int r = base + tid;
+    uint32_t npg = 0, miss = 0;
+    if (r < np) {
+      const int p = s_parts[r];
+      const int seg = s_mdir[p >> c.seg_shift];
+      int tokens = 0, res = 1;
+      if (seg >= 0) {
+        const int2 m = *reinterpret_cast<const int2 *>(c.meta_pool + ((size_t)seg << c.seg_shift) + (p & seg_mask));
+        tokens = m.x; res = m.y;
+      } else dev_error(c, kErrBounds);
+      npg = (tokens + kPageTokens - 1) / kPageTokens;
+      miss = res ? 0 : 1;
+      s_tokens[r] = tokens;
+      s_state[r] = res ? kHit : kAdmit;
+    }
+    uint32_t tot_a, tot_m;
+    const uint32_t ex_a = block_scan<T>(npg, sh.wsum, &tot_a);
+    const uint32_t ex_m = block_scan<T>(miss ? npg : 0, sh.wsum, &tot_m);
+    if (r < np) {
+      s_pageoff[r] = run_all + ex_a;
+      s_missoff[r] = run_miss + ex_m;
+      s_missbefore[r] = run_miss + ex_m;
+    }
+    run_all += tot_a;
+    run_miss += tot_m;
+  }
+  if (tid == 0) s_pageoff[np] = run_all;
+  int total_pages = (int)run_all;
+  const int demand = (int)run_miss;
+  if (total_pages > c.max_pages) {
+    if (tid == 0) dev_error(c, kErrPageList);
+    __syncthreads();
+    while (np > 0 && s_pageoff[np] > c.max_pages) --np;
+    total_pages = s_pageoff[np];
+  }
+  for (int i = tid; i < (S + 31) / 32; i += T) s_hit[i] = 0;
+  for (int i = tid; i < kMaxBuckets + 2; i += T) sh.lhist[i] = 0;
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");     // the GPU page table copy has landed
+  __syncthreads();
+
+  dbg_ts(b, 4);
+  // Retrieve step 3 started early (pinned host tables, two dependent reads over the host link)
+  int early_off[2] = {-1, -1}, early_i[2] = {0, 0};
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int mi = tid + j * T;
+    if (resolve_in_manager(c) && mi < demand && mi < c.max_pages && np > 0) {
+      const int r = owner_of(s_missbefore, np, mi);
+      early_i[j] = mi - s_missbefore[r];
+      const int32_t *off = off_lookup(c, set, s_parts[r]);
+      if (off) early_off[j] = *off;
+    }
+  }
+
+  // ---- step 2: one pass over the page table copy: promote, demote, histogram ----------------
+  const size_t pl = (size_t)b * (c.max_pages + c.tail_cap);
+  int32_t *page_src = c.page_src + pl, *page_slot = c.page_slot + pl;
+  int32_t *page_part = c.page_part + pl, *page_pidx = c.page_pidx + pl;
+  uint32_t *page_mask = c.page_mask + pl;
+  int32_t *page_fill = c.page_fill + pl;
+  int4 *page_desc = c.page_desc + pl;
+  for (int s_ = tid; s_ < S; s_ += T) {
+    int4 e = s_gpt[s_];
+    if (c.trace) {
+      c.evict_trace[((size_t)set * c.max_slots + s_) * 2] = -1;
+      c.evict_trace[((size_t)set * c.max_slots + s_) * 2 + 1] = -1;
+    }
+    if (e.x < 0) { atomicAdd(&sh.lhist[0], 1u); continue; }
+    const int r = find_sorted(s_parts, np, e.x);
+    if (r >= 0) {
+      atomicOr(&s_hit[s_ >> 5], 1u << (s_ & 31));
+      e.w = top;
+      const int idx = s_pageoff[r] + e.z;
+      page_src[idx] = e.y;
+      page_slot[idx] = s_;
+    } else {
+      if (t > nb - 1 && e.w > 0) --e.w;
+      atomicAdd(&sh.lhist[e.w + 1], 1u);
+    }
+    s_gpt[s_] = e;
+  }
+  __syncthreads();
+
+  dbg_ts(b, 5);
+  int early_host[2] = {-1, -1};
+#pragma unroll
+  for (int j = 0; j < 2; ++j)
+    if (early_off[j] >= 0) {
+      const int32_t *hp = cpt_lookup(c, set, early_off[j] + early_i[j]);
+      if (hp) early_host[j] = *hp;
+    }
+
+  // ---- step 3: threshold, eviction, free slots in ascending order (one scan) ----------------
+  if (tid == 0) {
+    int x = -2;
+    if (demand > 0) {
+      x = nb - 1;
+      uint32_t cum = 0;
+      for (int bk = -1; bk < nb; ++bk) {
+        cum += sh.lhist[bk + 1];
+        if ((int)cum >= demand) { x = bk; break; }
+      }
+    }
+    sh.x = x;
+  }
+  __syncthreads();
+  const int x = sh.x;
+  uint32_t run_free = 0;
+  if (demand > 0) {
+    const int E = (S + T - 1) / T, lo = min(S, tid * E), hi = min(S, lo + E);
+    uint32_t nfree = 0;
+    for (int s_ = lo; s_ < hi; ++s_) {
+      int4 e = s_gpt[s_];
+      if (e.x < 0) { ++nfree; continue; }
+      if (!((s_hit[s_ >> 5] >> (s_ & 31)) & 1u) && e.w <= x) {
+        const int seg = s_mdir[e.x >> c.seg_shift];
+        if (seg >= 0) c.meta_pool[((size_t)seg << c.seg_shift) + (e.x & seg_mask)].resident = 0;
+        if (c.trace) {
+          c.evict_trace[((size_t)set * c.max_slots + s_) * 2] = e.x;
+          c.evict_trace[((size_t)set * c.max_slots + s_) * 2 + 1] = e.z;
+        }
+        s_gpt[s_] = make_int4(-1, e.y, 0, -1);
+        atomicAdd(&sh.evicted, 1);
+        ++nfree;
+      }
+    }
+    uint32_t tot;
+    uint32_t pos = block_scan<T>(nfree, sh.wsum, &tot);
+    for (int s_ = lo; s_ < hi; ++s_)
+      if (s_gpt[s_].x < 0) { if (pos < (uint32_t)c.max_pages) s_free[pos] = s_; ++pos; }
+    run_free = tot;
+  }
+#pragma unroll
+  for (int j = 0; j < 2; ++j) { const int mi = tid + j * T; if (mi < c.max_pages) s_host[mi] = early_host[j]; }
+  __syncthreads();
+
+  dbg_ts(b, 6);
+  // ---- step 4: admission --------------------------------------------------------------------
+  if (demand > (int)run_free) {
+    if (tid == 0) {
+      int used = 0;
+      for (int r = 0; r < np; ++r) {
+        if (s_state[r] == kHit) continue;
+        const int npg = (s_tokens[r] + kPageTokens - 1) / kPageTokens;
+        if (npg <= (int)run_free - used) { s_missoff[r] = used; used += npg; }
+        else s_state[r] = kBypass;
+      }
+      sh.demand = used;
+    }
+  } else if (tid == 0) sh.demand = demand;
+  __syncthreads();
+  if (tid == 0) sh.qbase = (sh.demand > 0 && c.fetch_mode != 0) ? atomicAdd(c.fetch_count, sh.demand) : 0;
+  __syncthreads();
+  const int qbase = sh.qbase;
+  for (int r = tid; r < np; r += T) {
+    c.part_state[(size_t)b * c.max_parts + r] = s_state[r];
+    if (s_state[r] == kAdmit) {
+      const int p = s_parts[r], seg = s_mdir[p >> c.seg_shift];
+      if (seg >= 0) c.meta_pool[((size_t)seg << c.seg_shift) + (p & seg_mask)].resident = 1;
+    }
+  }
+  int my_admit = 0, my_bypass = 0;
+  for (int idx = tid; idx < total_pages; idx += T) {
+    const int r = owner_of(s_pageoff, np, idx);
+    const int i = idx - s_pageoff[r], p = s_parts[r], state = s_state[r];
+    const int valid = min(kPageTokens, s_tokens[r] - i * kPageTokens);
+    const uint32_t pmask = (1u << valid) - 1u;
+    page_mask[idx] = pmask;
+    page_part[idx] = p;
+    page_pidx[idx] = i;
+    page_fill[idx] = -1;
+    const int pos = state == kHit ? demand + (s_pageoff[r] - s_missbefore[r]) + i : s_missbefore[r] + i;
+    if (state == kHit) { page_desc[pos] = make_int4(page_src[idx], -1, (int)pmask, idx); continue; }
+    const int mi = s_missbefore[r] + i;
+    // Retrieve step 3 (Partition Offset -> CPU page table, both in pinned host memory): with
+    // the fetch fused into attention, the warp that brings the page in looks its CPU page id up
+    // itself (fill = -2), so this set's page list does not wait on the host link; with the
+    // stand-alone copy kernel the ids are resolved here
+    int host_page = -2;
+    if (resolve_in_manager(c)) {
+      host_page = mi < 2 * T && mi < c.max_pages ? s_host[mi] : -1;
+      if (host_page < 0) {
+        const int32_t *off = off_lookup(c, set, p);
+        const int32_t *hp = off ? cpt_lookup(c, set, *off + i) : nullptr;
+        if (hp) host_page = *hp;
+      }
+      if (host_page < 0) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
+    }
+    if (state == kAdmit) {
+      const int slot = s_free[s_missoff[r] + i];
+      const int phys = s_gpt[slot].y;
+      s_gpt[slot] = make_int4(p, phys, i, top);
+      page_src[idx] = phys;
+      page_slot[idx] = slot;
+      int fill = -1;
+      if (c.fetch_mode == 0) { fill = host_page; page_fill[idx] = host_page; }    // host_page is -2 if unresolved
+      else {
+        const int qi = qbase + s_missoff[r] + i;
+        if (qi < c.fetch_cap) c.fetch_queue[qi] = FetchItem{host_page, phys};
+        else dev_error(c, kErrBounds);
+      }
+      page_desc[pos] = make_int4(phys, fill, (int)pmask, idx);
+      ++my_admit;
+    } else {
+      // bypassed: attended from host memory, never cached (x = -1: no slot)
+      page_src[idx] = host_page == -2 ? -1 : ~host_page;
+      page_slot[idx] = -1;
+      page_desc[pos] = host_page == -2 ? make_int4(-1, -2, (int)pmask, idx) : make_int4(~host_page, -1, (int)pmask, idx);
+      ++my_bypass;
+    }
+  }
+  if (my_admit) atomicAdd(&sh.admit_pages, my_admit);
+  if (my_bypass) atomicAdd(&sh.bypass_pages, my_bypass);
+  for (int j = tid; j < tail_pages; j += T) {
+    const int idx = total_pages + j;
+    const int src = c.tail_phys[(size_t)set * c.tail_cap + j];
+    const uint32_t m = j == tail_pages - 1 ? ((1u << tail_len) - 1u) : 0xffffu;
+    page_src[idx] = src;
+    page_mask[idx] = m;
+    page_slot[idx] = -2;
+    page_fill[idx] = -1;
+    page_desc[idx] = make_int4(src, -1, (int)m, idx);
+    page_part[idx] = -1;
+    page_pidx[idx] = j;
+  }
+  __syncthreads();
+  dbg_ts(b, 7);
+  if (tid == 0) {
+    c.n_pages[b] = total_pages + tail_pages;
+    c.n_parts[b] = np;
+    c.state[set].step = t + 1;
+    Counters *kc = c.counters;
+    const int miss_pages = sh.admit_pages + sh.bypass_pages;
+    atomicAdd(&kc->set_steps, 1ull);
+    atomicAdd(&kc->selected_partitions, (unsigned long long)np);
+    atomicAdd(&kc->selected_pages, (unsigned long long)total_pages);
+    atomicAdd(&kc->tail_pages, (unsigned long long)tail_pages);
+    atomicAdd(&kc->hit_pages, (unsigned long long)(total_pages - miss_pages));
+    atomicAdd(&kc->miss_pages, (unsigned long long)miss_pages);
+    atomicAdd(&kc->evicted_pages, (unsigned long long)sh.evicted);
+    atomicAdd(&kc->bypass_pages, (unsigned long long)sh.bypass_pages);
+    flag_publish(c.ready + b, bt.epoch);
+  }
+  // ---- the page table goes back in one sweep; attention does not wait for it -----------------
+  for (int s_ = tid; s_ < S; s_ += T) {
+    const int seg = s_gdir[s_ >> c.seg_shift];
+    if (seg >= 0) *reinterpret_cast<int4 *>(c.gpt_pool + ((size_t)seg << c.seg_shift) + (s_ & seg_mask)) = s_gpt[s_];
+  }
+  dbg_ts(b, 8);
 }
 
 }  // namespace spin

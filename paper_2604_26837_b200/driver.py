@@ -21,15 +21,15 @@ def context_sizes(w: W.Workload):
 
 def make_spin(w: W.Workload, device="cuda:0", trace: bool = False, sm_scale: float = 0.0,
               slots_per_set: Optional[int] = None, segment_entries: int = 0,
-              fetch_mode: int = 0) -> "SpinRun":
-    return SpinRun(w, device, trace, sm_scale, slots_per_set, segment_entries, fetch_mode)
+              fetch_mode: int = 0, host_tables_only: int = 0) -> "SpinRun":
+    return SpinRun(w, device, trace, sm_scale, slots_per_set, segment_entries, fetch_mode, host_tables_only)
 
 
 class SpinRun:
     """A library context sized for one workload, plus the per-step call sequence."""
 
     def __init__(self, w: W.Workload, device="cuda:0", trace=False, sm_scale=0.0,
-                 slots_per_set=None, segment_entries=0, fetch_mode=0):
+                 slots_per_set=None, segment_entries=0, fetch_mode=0, host_tables_only=0):
         self.w = w
         self.device = torch.device(device)
         T = w.page_tokens
@@ -48,7 +48,7 @@ class SpinRun:
             topk=w.topk, num_clusters=w.num_clusters if cluster else 0,
             max_selected_pages=(w.topk * w.max_partition_pages if cluster else 0),
             max_tail_tokens=(w.steps + T if cluster else 0), lru_buckets=w.lru_buckets,
-            segment_entries=segment_entries, sm_scale=sm_scale, trace=1 if trace else 0, fetch_mode=fetch_mode,
+            segment_entries=segment_entries, sm_scale=sm_scale, trace=1 if trace else 0, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
             gpu_cache_pages=self.slots * sets_per_req * w.batch, host_pages=host_pages)
         self.spin = B.Spin(cfg, self.device)
         self.reqs: List[int] = [self.spin.request_open(self.slots) for _ in range(w.batch)]

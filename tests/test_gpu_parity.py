@@ -27,11 +27,11 @@ def _wl(kind, **kw):
 
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
-               one_call=False, fetch_mode=0):
+               one_call=False, fetch_mode=0, host_tables_only=0):
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
-                  segment_entries=segment_entries, fetch_mode=fetch_mode)
+                  segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
@@ -133,6 +133,15 @@ def test_append_and_decode_in_one_call(kind):
     run_parity(_wl(kind, steps=40, topk=12 if kind == W.PART_TOKEN_DOT else 6, **extra), one_call=True)
 
 
+@pytest.mark.parametrize("fetch_mode", [0, 1])
+def test_host_tables_read_over_the_link_as_in_the_paper(fetch_mode):
+    # no HBM mirror: Partition Offset / CPU page table are read from pinned host memory
+    run_parity(_wl(W.PART_PAGE_MINMAX, steps=30, topk=10, slots_per_set=7), host_tables_only=1,
+               fetch_mode=fetch_mode, one_call=True)
+    run_parity(_wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=23, max_partition_pages=8,
+                   steps=20), host_tables_only=1, fetch_mode=fetch_mode)
+
+
 def test_separate_fetch_kernel_mode():
     run_parity(_wl(W.PART_PAGE_MINMAX, steps=30), fetch_mode=1)
     run_parity(_wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=23, max_partition_pages=8,
@@ -161,6 +170,13 @@ def test_page_minmax_overflowing_budget_bypasses():
 def test_page_minmax_single_bucket_and_gqa1_gqa8():
     run_parity(_wl(W.PART_PAGE_MINMAX, lru_buckets=1, steps=10, num_q_heads=2, num_kv_heads=2))
     run_parity(_wl(W.PART_PAGE_MINMAX, steps=6, num_q_heads=16, num_kv_heads=2))
+
+
+def test_more_slots_than_the_shared_memory_path_holds():
+    # > 1024 slots per set: the cache manager works on the page table in global memory
+    w = _wl(W.PART_PAGE_MINMAX, context=16 * 1300 + 3, slots_per_set=1100, topk=40, steps=36, batch=1,
+            num_layers=1, lru_buckets=8, drift=0.4)
+    run_parity(w, check_bytes=False, one_call=True)
 
 
 def test_empty_and_short_contexts():
