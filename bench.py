@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 PAGE_BYTES = 8192
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
 # (profiles/), keyed by workload then kernel; None = not captured for this workload.
-NCU_TRAFFIC = {"c2": {"fetch": None, "score": None, "attn_split": None}}
+NCU_TRAFFIC = {"c2": {"fetch": None, "score": 69.5e6, "attn_split": 66.1e6}}
 
 
 def load_peaks():
@@ -162,6 +162,29 @@ def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests:
                                 f"(all {w.num_kv_heads} kv heads, {w.num_layers} layer(s)), numpy, 1 thread")
 
 
+def rank_workload(base, rank: int, total_steps: int):
+    """The replica a rank runs: same shapes, its own seed (sets are independent, so N ranks are N
+    independent replicas with no collective on the data path)."""
+    import workloads as W
+    return W.scaled(base, seed=base.seed + 1000 * rank, steps=total_steps)
+
+
+def allreduce_max(values, device="cpu"):
+    """Max over ranks of a list of floats (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_value(units_per_rank: int, world: int, max_elapsed_ms: float) -> float:
+    """Whole-job throughput: the units all ranks processed over the slowest rank's time."""
+    return units_per_rank * world / (max_elapsed_ms * 1e-3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -223,7 +246,7 @@ def main():
     prof_steps = min(K, 64)
     e2e_steps = 0 if args.no_e2e else K
     total_steps = P + Wm + K + K + prof_steps + (Wm + e2e_steps)
-    w = W.scaled(base, seed=base.seed + 1000 * rank, steps=total_steps)
+    w = rank_workload(base, rank, total_steps)
     run = SpinRun(w, device, fetch_mode=args.fetch_mode)
     stream = torch.cuda.Stream(device)
     B, L = w.batch, w.num_layers
@@ -338,9 +361,7 @@ def main():
     final = run.spin.stats()
 
     if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_ms if e2e_steps else 0.0, noflush_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_max, noflush_ms = (float(x) for x in t)
+        elapsed_ms, e2e_max, noflush_ms = allreduce_max([elapsed_ms, e2e_ms if e2e_steps else 0.0, noflush_ms], device)
         if e2e_steps:
             e2e_ms = e2e_max
     if rank != 0:
@@ -350,8 +371,7 @@ def main():
         return
 
     peaks = load_peaks()
-    tokens = B * K * world
-    value = tokens / (elapsed_ms * 1e-3)
+    value = aggregate_value(B * K, world, elapsed_ms)
     d = {k: st1[k] - st0[k] for k in st0 if k != "error_bits"}
     hbm_step = d["hbm_bytes"] / K
     pcie_step = d["pcie_bytes"] / K

@@ -1,0 +1,45 @@
+"""The N > 1 plumbing of bench.py on CPU: two gloo ranks, max-over-ranks timing, whole-job value,
+independent replicas (different seeds, no data-path collective)."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    import workloads as W
+    w = bench.rank_workload(W.CONFIGS["c1"], rank, 40)
+    k, _ = W.kv_tokens(w, 0, 0, 0, 8)
+    # each rank "measures" a different time; everyone must end up with the slowest one
+    elapsed, other = bench.allreduce_max([10.0 + 5.0 * rank, 3.0 - rank])
+    dist.barrier()
+    out[rank] = (w.seed, w.steps, float(k.float().sum()), elapsed, other,
+                 bench.aggregate_value(8 * 128, world, elapsed))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_max_timing_and_replica_seeds():
+    world, port = 2, 29500 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+        r0, r1 = out[0], out[1]
+    assert r0[0] != r1[0] and r0[1] == r1[1] == 40          # own seed per replica, same shape
+    assert r0[2] != r1[2]                                    # so the replicas hold different data
+    assert r0[3] == r1[3] == 15.0 and r0[4] == r1[4] == 3.0  # max over ranks, on every rank
+    assert r0[5] == r1[5] == 8 * 128 * 2 / 15e-3             # units of all ranks / slowest time
+
+
+def test_single_process_is_identity():
+    import bench
+    assert bench.allreduce_max([1.5, 2.5]) == [1.5, 2.5]
+    assert bench.aggregate_value(100, 1, 1000.0) == 100.0
