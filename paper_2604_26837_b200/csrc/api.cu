@@ -250,6 +250,16 @@ size_t host_bytes_needed(const Geometry &g, const spin_config &cfg) {
   return b;
 }
 
+// 0: device memory; 1: pinned (or registered) host memory, *alias = the address kernels can use;
+// 2: ordinary host memory
+int classify_ptr(const void *p, const void **alias) {
+  cudaPointerAttributes at{};
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return 2; }
+  if (at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged) { if (alias) *alias = p; return 0; }
+  if (at.type == cudaMemoryTypeHost && at.devicePointer) { if (alias) *alias = at.devicePointer; return 1; }
+  return 2;
+}
+
 bool is_device_ptr(const void *p) {
   cudaPointerAttributes at{};
   if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
@@ -879,7 +889,12 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     if (with_append && L.n_tokens % kPageTokens == 0) completes_page = true;     // a new page starts
   }
   const __nv_bfloat16 *kk = nullptr, *vv = nullptr;
-  bool in_grid = false;
+  const void *k_alias = nullptr, *v_alias = nullptr, *q_alias = nullptr, *out_alias = nullptr;
+  const size_t kv_bytes = (size_t)n_req * ctx->cfg.num_kv_heads * kRowBytes;
+  const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
+  bool in_grid = false, kv_pinned = false;
+  // q and new k/v in pinned host memory: one zero-copy staging kernel brings them in
+  const int qc = classify_ptr(q, &q_alias), oc = classify_ptr(out, &out_alias);
   if (with_append) {
     for (int i = 0; i < n_req; ++i) {
       LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
@@ -888,16 +903,20 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     }
     kk = reinterpret_cast<const __nv_bfloat16 *>(k);
     vv = reinterpret_cast<const __nv_bfloat16 *>(v);
-    if (!is_device_ptr(k)) {
-      const size_t bytes = (size_t)n_req * ctx->cfg.num_kv_heads * kRowBytes;
-      CK(cudaMemcpyAsync(ctx->stage_k, k, bytes, cudaMemcpyHostToDevice, st));
-      CK(cudaMemcpyAsync(ctx->stage_v, v, bytes, cudaMemcpyHostToDevice, st));
-      kk = ctx->stage_k;
-      vv = ctx->stage_v;
+    const int kc = classify_ptr(k, &k_alias), vc = classify_ptr(v, &v_alias);
+    if (kc != vc) return fail(ctx, SPIN_ERR_INVALID, "k_new and v_new must live in the same kind of memory");
+    if (kc == 2) {
+      CK(cudaMemcpyAsync(ctx->stage_k, k, kv_bytes, cudaMemcpyHostToDevice, st));
+      CK(cudaMemcpyAsync(ctx->stage_v, v, kv_bytes, cudaMemcpyHostToDevice, st));
     }
+    if (kc != 0) { kk = ctx->stage_k; vv = ctx->stage_v; }
+    kv_pinned = kc == 1;
     // An append that completes no page cannot change what Select sees: it then runs inside
     // the scoring kernel (one extra CTA per set).  Otherwise it runs first, on its own.
     in_grid = !completes_page;
+    if (kv_pinned || qc == 1)
+      ctx->launches += launch_stage_in(ctx->stage_q, qc == 1 ? q_alias : nullptr, qc == 1 ? qbytes : 0, ctx->stage_k,
+                                       k_alias, ctx->stage_v, v_alias, kv_pinned ? kv_bytes : 0, st);
     if (!in_grid) {
       AppendEdgeArgs a{};
       a.n_req = n_req;
@@ -923,19 +942,22 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     b.step[i] = L.steps++;
     b.n_partitions[i] = L.n_partitions;
   }
-  const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
   const __nv_bfloat16 *qd = reinterpret_cast<const __nv_bfloat16 *>(q);
   __nv_bfloat16 *od = reinterpret_cast<__nv_bfloat16 *>(out);
-  const bool q_dev = is_device_ptr(q), out_dev = is_device_ptr(out);
-  if (!q_dev) { CK(cudaMemcpyAsync(ctx->stage_q, q, qbytes, cudaMemcpyHostToDevice, st)); qd = ctx->stage_q; }
-  if (!out_dev) od = ctx->stage_out;
+  if (qc == 2) CK(cudaMemcpyAsync(ctx->stage_q, q, qbytes, cudaMemcpyHostToDevice, st));
+  if (qc == 1 && !with_append)
+    ctx->launches += launch_stage_in(ctx->stage_q, q_alias, qbytes, nullptr, nullptr, nullptr, nullptr, 0, st);
+  if (qc != 0) qd = ctx->stage_q;
+  // pinned host output: the attention kernel writes it directly (visible once the stream is synchronised)
+  if (oc == 1) od = reinterpret_cast<__nv_bfloat16 *>(const_cast<void *>(out_alias));
+  else if (oc == 2) od = ctx->stage_out;
   prof_mark(&ctx->prof, st, -1);
   b.epoch = ++ctx->epoch;
   b.append_in_grid = in_grid ? 1 : 0;
   ctx->launches += launch_select(ctx->d, b, qd, kk, vv, (int)max_cand, st, &ctx->prof);
   ctx->launches += launch_fetch(ctx->d, st, ctx->sm_count, &ctx->prof);
   ctx->launches += launch_attention(ctx->d, b, qd, od, (int)max_pages, may_be_empty, st, &ctx->prof);
-  if (!out_dev) CK(cudaMemcpyAsync(out, ctx->stage_out, qbytes, cudaMemcpyDeviceToHost, st));
+  if (oc == 2) CK(cudaMemcpyAsync(out, ctx->stage_out, qbytes, cudaMemcpyDeviceToHost, st));
   CK(cudaGetLastError());
   return SPIN_OK;
 }

@@ -73,7 +73,33 @@ k_copy_centroids(DevCtx c, int req, int layer, const __nv_bfloat16 *__restrict__
   }
 }
 
+// Step inputs that live in pinned host memory (q, new k/v) are brought into the staging
+// buffers by one small kernel of zero-copy reads instead of one copy-engine transfer each.
+__global__ void __launch_bounds__(256)
+k_stage_in(uint4 *dq, const uint4 *sq, int nq, uint4 *dk, const uint4 *sk, uint4 *dv, const uint4 *sv, int nkv) {
+  pdl_launch_next();
+  pdl_wait_prev();
+  const int total = nq + 2 * nkv;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    if (i < nq) dq[i] = sq[i];
+    else if (i < nq + nkv) dk[i - nq] = sk[i - nq];
+    else dv[i - nq - nkv] = sv[i - nq - nkv];
+  }
+}
+
 }  // namespace
+
+int launch_stage_in(void *dq, const void *sq, size_t q_bytes, void *dk, const void *sk, void *dv, const void *sv,
+                    size_t kv_bytes, cudaStream_t st) {
+  const int nq = (int)(q_bytes / 16), nkv = (int)(kv_bytes / 16);
+  if (nq + nkv == 0) return 0;
+  int grid = (nq + 2 * nkv + 255) / 256;
+  if (grid > 64) grid = 64;
+  launch_pdl(k_stage_in, dim3(grid), dim3(256), 0, st, 1, reinterpret_cast<uint4 *>(dq), reinterpret_cast<const uint4 *>(sq), nq,
+             reinterpret_cast<uint4 *>(dk), reinterpret_cast<const uint4 *>(sk), reinterpret_cast<uint4 *>(dv),
+             reinterpret_cast<const uint4 *>(sv), nkv);
+  return 1;
+}
 
 int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,

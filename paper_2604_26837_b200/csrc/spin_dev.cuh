@@ -266,6 +266,8 @@ int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bflo
 int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                            const __nv_bfloat16 *v, const int64_t *dest_row, int n_tokens,
                            cudaStream_t st);
+int launch_stage_in(void *dq, const void *sq, size_t q_bytes, void *dk, const void *sk, void *dv, const void *sv,
+                    size_t kv_bytes, cudaStream_t st);
 int launch_copy_centroids(const DevCtx &c, int req, int layer, const __nv_bfloat16 *cen,
                           int n_clusters, cudaStream_t st);
 int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,

@@ -27,7 +27,7 @@ def _wl(kind, **kw):
 
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
-               one_call=False, fetch_mode=0, host_tables_only=0):
+               one_call=False, fetch_mode=0, host_tables_only=0, host_io=None):
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
@@ -46,6 +46,15 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
                 orc.append_kv(oreq[r], l, W.to_bits(k), W.to_bits(v))
     qs = {(r, l): W.QueryStream(w, r, l, dev) for r in range(w.batch) for l in range(w.num_layers)}
     out = torch.zeros(w.batch, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    if host_io:                          # q / k / v / out handed over as HOST buffers
+        out = torch.zeros(w.batch, w.num_q_heads, w.head_dim, dtype=torch.bfloat16)
+        out = out.pin_memory() if host_io == "pinned" else out
+
+    def to_io(x):
+        if not host_io:
+            return x
+        x = x.cpu()
+        return x.pin_memory() if host_io == "pinned" else x
     cap_sel = w.topk
     cap_pages = w.topk * max(1, w.max_partition_pages) + (w.steps + 16) // 16 + 2
     worst_abs, worst_mean, rel_num, rel_den = 0.0, 0.0, 0.0, 0.0
@@ -56,11 +65,12 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
             for r in range(w.batch):
                 orc.append_kv(oreq[r], l, kb[r:r + 1], vb[r:r + 1])
             q = torch.stack([qs[(r, l)].next() for r in range(w.batch)]).contiguous()
+            kio, vio, qio = to_io(kn), to_io(vn), to_io(q)
             if one_call:                      # spin_decode_step_append: append + decode in one call
-                run.step(l, kn, vn, q, out)
+                run.step(l, kio, vio, qio, out)
             else:
-                run.append(l, kn, vn)
-                run.decode(l, q, out)
+                run.append(l, kio, vio)
+                run.decode(l, qio, out)
             ref = orc.decode_step(l, oreq, W.to_bits(q))
             torch.cuda.synchronize()
             got = out.float().cpu().numpy().astype(np.float64)
@@ -140,6 +150,12 @@ def test_host_tables_read_over_the_link_as_in_the_paper(fetch_mode):
                fetch_mode=fetch_mode, one_call=True)
     run_parity(_wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=23, max_partition_pages=8,
                    steps=20), host_tables_only=1, fetch_mode=fetch_mode)
+
+
+@pytest.mark.parametrize("host_io", ["pinned", "pageable"])
+@pytest.mark.parametrize("one_call", [True, False])
+def test_host_buffers_in_and_out(host_io, one_call):
+    run_parity(_wl(W.PART_PAGE_MINMAX, steps=20), host_io=host_io, one_call=one_call, check_bytes=False)
 
 
 def test_separate_fetch_kernel_mode():
