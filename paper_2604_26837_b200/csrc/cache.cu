@@ -24,15 +24,32 @@ namespace {
 constexpr int kCacheThreads = 512;
 
 // Stand-alone cache manager: one CTA per set (used when top-k ran as its own cluster kernel).
+// fast != 0: every set of the batch has at most kFastSlots slots and the shared-memory layout
+// fits, so the page table is staged in shared memory (cache_fast); else it is worked on in
+// global memory (cache_stage).
 __global__ void __launch_bounds__(kCacheThreads)
-k_cache(DevCtx c, Batch bt) {
-  extern __shared__ __align__(16) int32_t smem[];
-  __shared__ CacheShared sh;
-  const int b = blockIdx.x, i_req = b / c.Hkv, head = b % c.Hkv;
+k_cache(DevCtx c, Batch bt, int fast) {
+  extern __shared__ __align__(16) uint8_t dyn_smem[];
+  __shared__ union { CacheShared staged; FastShared fast; } shm;
+  const int b = blockIdx.x, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
   pdl_launch_next();
   pdl_wait_prev();
-  cache_stage<kCacheThreads>(c, b, set, c.n_parts[b], bt.tail_pages[i_req], bt.tail_len[i_req], bt.epoch, smem, sh);
+  const int np = c.n_parts[b];
+  if (!fast) {
+    cache_stage<kCacheThreads>(c, b, set, np, bt.tail_pages[i_req], bt.tail_len[i_req], bt.epoch,
+                               reinterpret_cast<int32_t *>(dyn_smem), shm.staged);
+    return;
+  }
+  const int S = bt.slots[i_req];
+  const FastLayout L = fast_layout(c, dyn_smem, 0, S);
+  fast_prefetch_dirs<kCacheThreads>(c, L, set, S);
+  const int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
+  for (int r = tid; r < np; r += kCacheThreads) L.s_parts[r] = g_parts[r];
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+  __syncthreads();
+  fast_prefetch_gpt<kCacheThreads>(c, L, S);
+  cache_fast<kCacheThreads>(c, bt, b, i_req, set, L, np, shm.fast);
 }
 
 // One warp per missed page: 8 KiB = 16 x (32 lanes x 16 B), all loads issued before the
@@ -60,12 +77,16 @@ size_t cache_smem_bytes(const DevCtx &c) { return cache_stage_smem_bytes(c.max_p
 
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
   static size_t configured = 0;
-  const size_t smem = cache_smem_bytes(c);
+  int max_slots_batch = 0;
+  for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
+  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
+  const int fast = (max_slots_batch <= kFastSlots && fs <= 96 * 1024) ? 1 : 0;
+  const size_t smem = fast ? fs : cache_smem_bytes(c);
   if (smem > configured) {
     cudaFuncSetAttribute(k_cache, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b);
+  launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b, fast);
   prof_mark(prof, st, kProfCache);
   return 1;
 }

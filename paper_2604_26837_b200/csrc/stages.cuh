@@ -205,21 +205,37 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
       }
     }
     // ---- ordered compaction: everything above thr, plus the first need_eq equal to it --
-    for (int base = 0; base < m; base += T) {
-      const int i = base + tid;
+    if (m <= 60000) {
+      // every thread owns a contiguous run of the slice: one block scan in all
+      const int E = (m + T - 1) / T, r0 = min(m, tid * E), r1 = min(m, r0 + E);
       uint32_t gt = 0, eq = 0;
-      if (i < m) {
-        const uint32_t key = key_at(i);
-        gt = key > thr;
-        eq = key == thr;
-      }
+      for (int i = r0; i < r1; ++i) { const uint32_t key = key_at(i); gt += key > thr; eq += key == thr; }
       uint32_t total;
       const uint32_t ex = block_scan<T>(gt | (eq << 16), sh.wsum, &total);
-      const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
-      if (gt || (eq && eq_before < need_eq))
-        sel[gt_before + min(eq_before, need_eq)] = lo + i;
-      run_gt += total & 0xffffu;
-      run_eq += total >> 16;
+      uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
+      for (int i = r0; i < r1; ++i) {
+        const uint32_t key = key_at(i);
+        if (key > thr || (key == thr && eq_before < need_eq)) sel[gt_before + min(eq_before, need_eq)] = lo + i;
+        gt_before += key > thr;
+        eq_before += key == thr;
+      }
+    } else {
+      for (int base = 0; base < m; base += T) {
+        const int i = base + tid;
+        uint32_t gt = 0, eq = 0;
+        if (i < m) {
+          const uint32_t key = key_at(i);
+          gt = key > thr;
+          eq = key == thr;
+        }
+        uint32_t total;
+        const uint32_t ex = block_scan<T>(gt | (eq << 16), sh.wsum, &total);
+        const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
+        if (gt || (eq && eq_before < need_eq))
+          sel[gt_before + min(eq_before, need_eq)] = lo + i;
+        run_gt += total & 0xffffu;
+        run_eq += total >> 16;
+      }
     }
   }
   stage_sync<CLUSTER>();     // selections of all slices are written; no remote smem is read after this
@@ -592,58 +608,87 @@ __device__ __forceinline__ void cp_async_commit_wait_all() {
   asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
 }
 
+struct FastLayout {
+  uint32_t *s_keys;
+  int4 *s_gpt;
+  int32_t *s_mdir, *s_gdir, *s_parts, *s_tokens, *s_pageoff, *s_missoff, *s_missbefore, *s_state, *s_free, *s_host;
+  uint32_t *s_hit;
+};
+
+__device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn, int n_keys, int S) {
+  FastLayout L;
+  L.s_keys = reinterpret_cast<uint32_t *>(dyn);
+  L.s_gpt = reinterpret_cast<int4 *>(L.s_keys + (n_keys + 3) / 4 * 4);
+  L.s_mdir = reinterpret_cast<int32_t *>(L.s_gpt + S);
+  L.s_gdir = L.s_mdir + c.dir_part;
+  L.s_parts = L.s_mdir + (c.dir_part + c.dir_slot + 3) / 4 * 4;
+  L.s_tokens = L.s_parts + c.max_parts;
+  L.s_pageoff = L.s_tokens + c.max_parts;        // [max_parts + 1]
+  L.s_missoff = L.s_pageoff + c.max_parts + 1;
+  L.s_missbefore = L.s_missoff + c.max_parts;
+  L.s_state = L.s_missbefore + c.max_parts;
+  L.s_free = L.s_state + c.max_parts + 3;        // [max_pages]
+  L.s_host = L.s_free + c.max_pages;             // [max_pages] CPU page ids of missed pages
+  L.s_hit = reinterpret_cast<uint32_t *>(L.s_host + c.max_pages);
+  return L;
+}
+
+// Directories of the Meta-partition table and of the GPU page table -> shared memory (one
+// cp.async group; the caller waits for it and barriers before fast_prefetch_gpt).
+template <int T>
+__device__ __forceinline__ void fast_prefetch_dirs(const DevCtx &c, const FastLayout &L, int set, int S) {
+  const int tid = threadIdx.x, n_gdir = (S + (1 << c.seg_shift) - 1) >> c.seg_shift;
+  for (int i = tid; i < c.dir_part; i += T) cp_async4(L.s_mdir + i, c.dir_meta + (size_t)set * c.dir_part + i);
+  for (int i = tid; i < n_gdir; i += T) cp_async4(L.s_gdir + i, c.dir_gpt + (size_t)set * c.dir_slot + i);
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+}
+// The set's whole GPU page table -> shared memory (one cp.async group).
+template <int T>
+__device__ __forceinline__ void fast_prefetch_gpt(const DevCtx &c, const FastLayout &L, int S) {
+  const int tid = threadIdx.x, seg_mask = (1 << c.seg_shift) - 1;
+  for (int s_ = tid; s_ < S; s_ += T) {
+    const int seg = L.s_gdir[s_ >> c.seg_shift];
+    if (seg >= 0) cp_async16_ca(L.s_gpt + s_, c.gpt_pool + ((size_t)seg << c.seg_shift) + (s_ & seg_mask));
+    else { dev_error(c, kErrBounds); L.s_gpt[s_] = make_int4(-1, 0, 0, -1); }
+  }
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+}
+
+template <int T>
+__device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
+                                           const FastLayout &L, int np_sel, FastShared &sh);
+
 template <int T>
 __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
                                             uint8_t *dyn, FastShared &sh) {
   const int tid = threadIdx.x;
   const int n = bt.n_partitions[i_req];
   const int k = min(c.topk, n);
-  const int S = bt.slots[i_req], t = bt.step[i_req], nb = c.n_buckets, top = min(t, nb - 1);
-  const int tail_pages = bt.tail_pages[i_req], tail_len = bt.tail_len[i_req];
-  const int seg_mask = (1 << c.seg_shift) - 1;
-  const int n_gdir = (S + seg_mask) >> c.seg_shift;
+  const int S = bt.slots[i_req];
 
-  // ---- shared memory layout -----------------------------------------------------------------
-  uint32_t *s_keys = reinterpret_cast<uint32_t *>(dyn);
-  int4 *s_gpt = reinterpret_cast<int4 *>(s_keys + (n + 3) / 4 * 4);
-  int32_t *s_mdir = reinterpret_cast<int32_t *>(s_gpt + S);
-  int32_t *s_gdir = s_mdir + c.dir_part;
-  int32_t *s_parts = s_mdir + (c.dir_part + c.dir_slot + 3) / 4 * 4;
-  int32_t *s_tokens = s_parts + c.max_parts;
-  int32_t *s_pageoff = s_tokens + c.max_parts;        // [max_parts + 1]
-  int32_t *s_missoff = s_pageoff + c.max_parts + 1;
-  int32_t *s_missbefore = s_missoff + c.max_parts;
-  int32_t *s_state = s_missbefore + c.max_parts;
-  int32_t *s_free = s_state + c.max_parts + 3;        // [max_pages]
-  int32_t *s_host = s_free + c.max_pages;             // [max_pages] CPU page ids of missed pages
-  uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_host + c.max_pages);
+  const FastLayout L = fast_layout(c, dyn, n, S);
+  uint32_t *s_keys = L.s_keys;
+  int32_t *s_parts = L.s_parts;
 
   dbg_ts(b, 1);
   // ---- directories on their way (consumed after the keys are loaded) ------------------------
-  for (int i = tid; i < c.dir_part; i += T) cp_async4(s_mdir + i, c.dir_meta + (size_t)set * c.dir_part + i);
-  for (int i = tid; i < n_gdir; i += T) cp_async4(s_gdir + i, c.dir_gpt + (size_t)set * c.dir_slot + i);
-  asm volatile("cp.async.commit_group;\n" ::: "memory");
+  fast_prefetch_dirs<T>(c, L, set, S);
 
   const float *scores = c.scores + (size_t)b * c.max_cand;
   for (int i = tid; i < n; i += T) s_keys[i] = order_key(__ldcg(scores + i));
   for (int i = tid; i < 512; i += T) (&sh.hist[0][0])[i] = 0;
   if (tid == 0) {
+    sh.lhist[0] = 0u;                        // OR / AND of the keys (reused as the timestamp histogram later)
+    sh.lhist[1] = 0xffffffffu;
     c.n_sel[b] = k;
-    c.att_count[b] = 0;
     atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
-    sh.evicted = 0; sh.admit_pages = 0; sh.bypass_pages = 0;
   }
   asm volatile("cp.async.wait_group 0;\n" ::: "memory");
   __syncthreads();
 
   dbg_ts(b, 2);
   // ---- the GPU page table on its way (consumed after top-k) ---------------------------------
-  for (int s_ = tid; s_ < S; s_ += T) {
-    const int seg = s_gdir[s_ >> c.seg_shift];
-    if (seg >= 0) cp_async16_ca(s_gpt + s_, c.gpt_pool + ((size_t)seg << c.seg_shift) + (s_ & seg_mask));
-    else { dev_error(c, kErrBounds); s_gpt[s_] = make_int4(-1, 0, 0, -1); }
-  }
-  asm volatile("cp.async.commit_group;\n" ::: "memory");
+  fast_prefetch_gpt<T>(c, L, S);
 
   // ---- top-k: radix select (two barriers per pass), one-scan ordered compaction -------------
   int32_t *g_sel = c.sel_ids + (size_t)b * c.max_sel;
@@ -651,9 +696,25 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   if (k == n) {
     for (int i = tid; i < n; i += T) { s_parts[i] = i; g_sel[i] = i; g_parts[i] = i; }
   } else {
+    // The scores of one set share their sign, exponent and often a few mantissa bits, so the
+    // leading radix passes would put every key into one bin (and serialise on its counter).
+    // Bytes on which all keys agree (OR == AND over the set) are skipped outright.
+    uint32_t k_or = 0, k_and = 0xffffffffu;
+    for (int i = tid; i < n; i += T) { const uint32_t key = s_keys[i]; k_or |= key; k_and &= key; }
+    k_or = __reduce_or_sync(0xffffffffu, k_or);
+    k_and = __reduce_and_sync(0xffffffffu, k_and);
+    if ((tid & 31) == 0) { atomicOr(&sh.lhist[0], k_or); atomicAnd(&sh.lhist[1], k_and); }
+    __syncthreads();
+    const uint32_t differ = sh.lhist[0] ^ sh.lhist[1];           // bits on which some keys differ
     uint32_t prefix = 0, mask = 0, remaining = k;
+    int first_shift = 24;
+    while (first_shift >= 0 && ((differ >> first_shift) & 255u) == 0) {
+      prefix |= sh.lhist[1] & (255u << first_shift);
+      mask |= 255u << first_shift;
+      first_shift -= 8;
+    }
     int buf = 0;
-    for (int shift = 24; shift >= 0; shift -= 8, buf ^= 1) {
+    for (int shift = first_shift; shift >= 0; shift -= 8, buf ^= 1) {
       for (int i = tid; i < n; i += T) {
         const uint32_t key = s_keys[i];
         if ((key & mask) == prefix) atomicAdd(&sh.hist[buf][(key >> shift) & 255u], 1u);
@@ -708,9 +769,27 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
     }
   }
   dbg_ts(b, 3);
-  const int np_sel = k;
   __syncthreads();
+  cache_fast<T>(c, bt, b, i_req, set, L, k, sh);
+}
 
+
+// Cache manager on the shared-memory copy of the page table.  Before the call: L.s_parts holds
+// the np_sel selected partitions (ascending), fast_prefetch_dirs has completed, and
+// fast_prefetch_gpt has been issued (its group may still be in flight).
+template <int T>
+__device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
+                                           const FastLayout &L, int np_sel, FastShared &sh) {
+  const int tid = threadIdx.x;
+  const int S = bt.slots[i_req], t = bt.step[i_req], nb = c.n_buckets, top = min(t, nb - 1);
+  const int tail_pages = bt.tail_pages[i_req], tail_len = bt.tail_len[i_req];
+  const int seg_mask = (1 << c.seg_shift) - 1;
+  int4 *s_gpt = L.s_gpt;
+  int32_t *s_mdir = L.s_mdir, *s_gdir = L.s_gdir, *s_parts = L.s_parts, *s_tokens = L.s_tokens;
+  int32_t *s_pageoff = L.s_pageoff, *s_missoff = L.s_missoff, *s_missbefore = L.s_missbefore;
+  int32_t *s_state = L.s_state, *s_free = L.s_free, *s_host = L.s_host;
+  uint32_t *s_hit = L.s_hit;
+  if (tid == 0) { c.att_count[b] = 0; sh.evicted = 0; sh.admit_pages = 0; sh.bypass_pages = 0; }
   // ---- cache manager step 1: Meta-partition lookups, classification, page demand ------------
   int np = np_sel;
   uint32_t run_all = 0, run_miss = 0;
@@ -881,7 +960,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
     const int r = owner_of(s_pageoff, np, idx);
     const int i = idx - s_pageoff[r], p = s_parts[r], state = s_state[r];
     const int valid = min(kPageTokens, s_tokens[r] - i * kPageTokens);
-    const uint32_t pmask = (1u << valid) - 1u;
+    const uint32_t pmask = c.kind == kKindToken ? c.part_mask[(size_t)b * c.max_parts + r] : ((1u << valid) - 1u);
     page_mask[idx] = pmask;
     page_part[idx] = p;
     page_pidx[idx] = i;
