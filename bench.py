@@ -123,7 +123,7 @@ def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests:
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets))
     reqs = []
     for r in range(sample_requests):
-        req = orc.request_open(w.slots_per_set)
+        req = orc.request_open(w.slots_per_set if w.slots_per_set else min(w.topk * 2, 512))
         reqs.append(req)
         for l in range(w.num_layers):
             k, v = W.kv_tokens(w, r, l, 0, w.request_context(r))
@@ -197,6 +197,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--context", type=int, default=0, help="override the context length (smaller captures)")
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (scaled runs of the 32-layer config)")
     ap.add_argument("--fetch-mode", type=int, default=0, help="0 fused into attention, 1 separate copy kernel")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -211,10 +212,18 @@ def main():
         base = W.scaled(base, context=args.context)
     if args.batch:
         base = W.scaled(base, batch=args.batch)
+    if args.layers:
+        base = W.scaled(base, num_layers=args.layers)
+    # a workload without a fixed budget states a total: 60 GB of KV over its 32 layers and 64
+    # requests; a scaled run keeps the per-layer, per-request share
+    cache_pages_per_layer = None
+    if base.slots_per_set == 0:
+        cache_pages_per_layer = int(60e9 / 32 / PAGE_BYTES * base.batch / 64)
     metric, unit = "decode_tokens_per_s", "tokens/s"
     cfg_desc = dict(workload=f"{base.name}: batch {base.batch} x {base.num_layers} layer(s), "
                              f"{base.num_q_heads}q/{base.num_kv_heads}kv heads, context {base.context}, "
-                             f"kind {base.partition_kind}, top-k {base.topk}, {base.slots_per_set} slots/set, "
+                             f"kind {base.partition_kind}, top-k {base.topk}, "
+                             f"{base.slots_per_set if base.slots_per_set else 'dynamic'} slots/set, "
                              f"{base.lru_buckets} buckets, drift {base.drift}",
                     global_batch=base.batch * world, context=base.context, parallelism=f"replicas x{world}")
 
@@ -247,7 +256,7 @@ def main():
     e2e_steps = 0 if args.no_e2e else K
     total_steps = P + Wm + K + K + prof_steps + (Wm + e2e_steps)
     w = rank_workload(base, rank, total_steps)
-    run = SpinRun(w, device, fetch_mode=args.fetch_mode)
+    run = SpinRun(w, device, fetch_mode=args.fetch_mode, cache_pages_per_layer=cache_pages_per_layer)
     stream = torch.cuda.Stream(device)
     B, L = w.batch, w.num_layers
 
@@ -402,7 +411,7 @@ def main():
     bound = kern[top]["bound"]
     peak = pcie_gbs if bound == "pcie" else peaks["hbm_gbs"]
     achieved = kern[top]["pcie_gbs"] if bound == "pcie" else kern[top]["hbm_gbs"]
-    traffic = (NCU_TRAFFIC.get(args.workload) or {}).get(top) if not (args.context or args.batch) else None
+    traffic = (NCU_TRAFFIC.get(args.workload) or {}).get(top) if not (args.context or args.batch or args.layers) else None
     names = dict(fetch="k_fetch", score="k_score", attn_split="k_attn (attention + page fetch)" if fused else "k_attn")
     roofline = dict(kernel=names[top], bound=bound, achieved=achieved, peak=peak, unit="GB/s",
                     frac=kern[top]["roof_frac"], traffic=traffic,

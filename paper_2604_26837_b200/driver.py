@@ -19,6 +19,24 @@ def context_sizes(w: W.Workload):
     return ctx
 
 
+def request_budgets(w: W.Workload, cache_pages_per_layer: int) -> List[int]:
+    """Per-request slots per set when the workload gives a total instead of a fixed budget:
+    every set first gets its mandatory pages min(top-k, its pages); what is left of the layer's
+    cache is shared in proportion to sequence length and capped at the set's page count
+    (Section 5.3, buffer elasticity: reclaim / grant in proportion to sequence length)."""
+    T = w.page_tokens
+    ctx = context_sizes(w)
+    pages = [(c + w.steps + T - 1) // T for c in ctx]
+    mandatory = [min(w.topk, p) for p in pages]
+    left = cache_pages_per_layer // w.num_kv_heads - sum(mandatory)
+    total = sum(pages)
+    out = []
+    for m, p in zip(mandatory, pages):
+        extra = max(0, left) * p // max(total, 1)
+        out.append(min(p, m + extra))
+    return out
+
+
 def make_spin(w: W.Workload, device="cuda:0", trace: bool = False, sm_scale: float = 0.0,
               slots_per_set: Optional[int] = None, segment_entries: int = 0,
               fetch_mode: int = 0, host_tables_only: int = 0) -> "SpinRun":
@@ -29,13 +47,17 @@ class SpinRun:
     """A library context sized for one workload, plus the per-step call sequence."""
 
     def __init__(self, w: W.Workload, device="cuda:0", trace=False, sm_scale=0.0,
-                 slots_per_set=None, segment_entries=0, fetch_mode=0, host_tables_only=0):
+                 slots_per_set=None, segment_entries=0, fetch_mode=0, host_tables_only=0,
+                 cache_pages_per_layer=None):
         self.w = w
         self.device = torch.device(device)
         T = w.page_tokens
         ctx = context_sizes(w)
         sets_per_req = w.num_layers * w.num_kv_heads
         self.slots = w.slots_per_set if slots_per_set is None else slots_per_set
+        # one budget per request (all its sets get it); a per-layer total switches to the dynamic split
+        self.budgets = ([self.slots] * w.batch if cache_pages_per_layer is None
+                        else request_budgets(w, cache_pages_per_layer))
         cluster = w.partition_kind == W.PART_CLUSTER_CENTROID
         pages_per_set = [(c + w.steps + T - 1) // T + 2 for c in ctx]
         if cluster:
@@ -49,9 +71,9 @@ class SpinRun:
             max_selected_pages=(w.topk * w.max_partition_pages if cluster else 0),
             max_tail_tokens=(w.steps + T if cluster else 0), lru_buckets=w.lru_buckets,
             segment_entries=segment_entries, sm_scale=sm_scale, trace=1 if trace else 0, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
-            gpu_cache_pages=self.slots * sets_per_req * w.batch, host_pages=host_pages)
+            gpu_cache_pages=sum(self.budgets) * sets_per_req, host_pages=host_pages)
         self.spin = B.Spin(cfg, self.device)
-        self.reqs: List[int] = [self.spin.request_open(self.slots) for _ in range(w.batch)]
+        self.reqs: List[int] = [self.spin.request_open(bud) for bud in self.budgets]
         self.ctx = ctx
         self.step_no = 0
 

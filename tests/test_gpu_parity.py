@@ -27,15 +27,16 @@ def _wl(kind, **kw):
 
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
-               one_call=False, fetch_mode=0, host_tables_only=0, host_io=None):
+               one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None):
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
-                  segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only)
+                  segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
+                  cache_pages_per_layer=cache_pages_per_layer)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
-    oreq = [orc.request_open(S) for _ in range(w.batch)]
+    oreq = [orc.request_open(bud) for bud in run.budgets]
     for r in range(w.batch):
         for l in range(w.num_layers):
             k, v, tp, cen = run.gen_prefill(r, l)
@@ -83,6 +84,7 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
                     tr = orc.last_trace[(oreq[r], l, h)]
                     st = orc.set(oreq[r], l, h)
                     ncand = len(tr.scores)
+                    S = run.budgets[r]
                     d = run.spin.debug_dump(run.reqs[r], l, h, cap_sel, cap_pages, S,
                                             st.n_partitions() + 1, ncand + 1)
                     where = f"step {step} layer {l} req {r} head {h}"
@@ -193,6 +195,15 @@ def test_more_slots_than_the_shared_memory_path_holds():
     w = _wl(W.PART_PAGE_MINMAX, context=16 * 1300 + 3, slots_per_set=1100, topk=40, steps=36, batch=1,
             num_layers=1, lru_buckets=8, drift=0.4)
     run_parity(w, check_bytes=False, one_call=True)
+
+
+def test_mixed_context_lengths_and_per_request_budgets():
+    # the mixed-batch configuration in small: contexts drawn per request, query drift drawn per
+    # request, budgets split from a per-layer total in proportion to sequence length
+    w = _wl(W.PART_PAGE_MINMAX, batch=5, num_layers=1, context=16 * 90, ctx_range=(40, 16 * 90),
+            drift_choices=(0.01, 0.1, 0.5), topk=10, steps=30, lru_buckets=8)
+    r = run_parity(w, cache_pages_per_layer=2 * 5 * 12, one_call=True)
+    assert r["stats"]["evicted_pages"] > 0
 
 
 def test_empty_and_short_contexts():
