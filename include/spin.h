@@ -128,6 +128,8 @@ typedef struct spin_stats_t {
   uint64_t summary_bytes;         /* summary segments in HBM, in use */
   uint64_t gpu_pages_in_use;
   uint64_t host_pages_in_use;
+  uint64_t first_error_site;      /* where the first device-side check tripped: source file id x
+                                     100000 + line (1 append, 2 select, 3 cache, 4 attention); 0 = none */
 } spin_stats_t;
 
 /* Logical view of one set after its last decode step (what the parity tests compare).

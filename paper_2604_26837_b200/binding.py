@@ -54,7 +54,7 @@ class spin_stats_t(C.Structure):
                                   "hit_pages", "miss_pages", "evicted_pages", "bypass_pages",
                                   "candidates_scored", "pcie_bytes", "hbm_bytes", "kernel_launches",
                                   "gpu_meta_bytes", "host_meta_bytes", "summary_bytes",
-                                  "gpu_pages_in_use", "host_pages_in_use")]
+                                  "gpu_pages_in_use", "host_pages_in_use", "first_error_site")]
 
 
 class spin_profile_t(C.Structure):

@@ -3,6 +3,7 @@
 // Index/Offload (which pages and segments an append touches) and the per-step launch sequence.
 // All decisions that need the tables' contents are taken on the GPU; the host only tracks
 // counts it can derive from the calls it has seen, so no call in the decode loop synchronises.
+#define SPIN_FILE_ID 5
 #include <algorithm>
 #include <cmath>
 #include <cstdarg>
@@ -984,6 +985,7 @@ int spin_stats(spin_ctx *ctx, spin_stats_t *out) {
   CK(cudaMemcpy(&c, ctx->d.counters, sizeof c, cudaMemcpyDeviceToHost));
   const Geometry &g = ctx->g;
   out->error_bits = c.error_bits;
+  out->first_error_site = c.first_site;
   out->set_steps = c.set_steps;
   out->selected_partitions = c.selected_partitions;
   out->selected_pages = c.selected_pages;

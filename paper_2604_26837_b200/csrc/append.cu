@@ -3,6 +3,7 @@
 // partition with its summary (per-channel min/max of the keys, or the key rows themselves
 // for token-granular selection).  The host runtime has already mapped the segments and
 // filled the host-side tables (Partition Offset, CPU page table) for the pages touched here.
+#define SPIN_FILE_ID 1
 #include "append_body.cuh"
 
 namespace spin {

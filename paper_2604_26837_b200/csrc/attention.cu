@@ -14,6 +14,7 @@
 // tiles are used to take instruction issue off the critical path, which is also why the
 // 64..128-row tcgen05 tiles (>90% padding at GQA 4) are not.  The last CTA of a set to finish
 // (a counter cleared by the cache-manager kernel) merges the set's partials and writes bf16.
+#define SPIN_FILE_ID 4
 #include <cstdio>
 
 #include "../../include/spin.h"

@@ -15,6 +15,7 @@
 // k_fetch: persistent warp-per-page copy from pinned host memory into HBM (Section 5.5: one
 // warp per page, vectorised 16-byte transactions, pages spread over all warps regardless of
 // owner).
+#define SPIN_FILE_ID 3
 #include "stages.cuh"
 
 namespace spin {

@@ -12,6 +12,7 @@
 // with that set's top-k and cache management (stages.cuh) while other sets are still being
 // scored, so the step needs no top-k or cache-manager launch.  k_topk is the stand-alone
 // top-k for candidate counts beyond one CTA's shared memory: a thread-block cluster per set.
+#define SPIN_FILE_ID 2
 #include "append_body.cuh"
 #include "stages.cuh"
 

@@ -45,7 +45,7 @@ struct Counters {
   unsigned long long set_steps, selected_partitions, selected_pages, tail_pages, hit_pages,
       miss_pages, evicted_pages, bypass_pages, candidates_scored;
   unsigned int error_bits;
-  unsigned int pad;
+  unsigned int first_site;   // where the first device-side error was raised (file id * 100000 + line)
 };
 
 struct FetchItem { int32_t host_page; int32_t gpu_page; };
@@ -130,9 +130,16 @@ __host__ __device__ inline int set_index(const DevCtx &c, int req, int layer, in
 }
 
 #ifdef __CUDACC__
-__device__ __forceinline__ void dev_error(const DevCtx &c, unsigned bits) {
+// Records the error bits and, for the first error only, where it was raised (source file id *
+// 100000 + line), so that a sticky bit can be traced to its check.
+__device__ __forceinline__ void dev_error_site(const DevCtx &c, unsigned bits, unsigned site) {
   atomicOr(&c.counters->error_bits, bits);
+  atomicCAS(&c.counters->first_site, 0u, site);
 }
+#ifndef SPIN_FILE_ID
+#define SPIN_FILE_ID 0
+#endif
+#define dev_error(c, bits) dev_error_site((c), (bits), (unsigned)(SPIN_FILE_ID * 100000 + __LINE__))
 // Two-level lookups.  A negative directory entry means "not mapped": the caller gets nullptr
 // and records a bounds error instead of touching memory.
 __device__ __forceinline__ MetaEntry *meta_at(const DevCtx &c, int set, int p) {

@@ -27,7 +27,10 @@ def _wl(kind, **kw):
 
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
-               one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None):
+               one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None,
+               oracle_reqs=None):
+    """oracle_reqs: the requests mirrored in the oracle (default all).  Sets are independent, so the
+    oracle run on a sample of the batch's requests must agree with those requests of the full batch."""
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
@@ -36,11 +39,14 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
-    oreq = [orc.request_open(bud) for bud in run.budgets]
+    sample = list(range(w.batch)) if oracle_reqs is None else list(oracle_reqs)
+    oreq = {r: orc.request_open(run.budgets[r]) for r in sample}
     for r in range(w.batch):
         for l in range(w.num_layers):
             k, v, tp, cen = run.gen_prefill(r, l)
             run.prefill(r, l, k, v, tp, cen)
+            if r not in oreq:
+                continue
             if tp is not None:
                 orc.append_kv(oreq[r], l, W.to_bits(k), W.to_bits(v), tp.cpu().numpy(), W.to_bits(cen))
             else:
@@ -63,7 +69,7 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
         for l in range(w.num_layers):
             kn, vn = run.gen_step_tokens(l, step)
             kb, vb = W.to_bits(kn), W.to_bits(vn)
-            for r in range(w.batch):
+            for r in sample:
                 orc.append_kv(oreq[r], l, kb[r:r + 1], vb[r:r + 1])
             q = torch.stack([qs[(r, l)].next() for r in range(w.batch)]).contiguous()
             kio, vio, qio = to_io(kn), to_io(vn), to_io(q)
@@ -72,14 +78,14 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
             else:
                 run.append(l, kio, vio)
                 run.decode(l, qio, out)
-            ref = orc.decode_step(l, oreq, W.to_bits(q))
+            ref = orc.decode_step(l, [oreq[r] for r in sample], W.to_bits(q)[sample])
             torch.cuda.synchronize()
-            got = out.float().cpu().numpy().astype(np.float64)
+            got = out.float().cpu().numpy().astype(np.float64)[sample]
             err = np.abs(got - ref)
             worst_abs, worst_mean = max(worst_abs, err.max()), max(worst_mean, err.mean())
             rel_num += float((err ** 2).sum())
             rel_den += float((ref ** 2).sum())
-            for r in range(w.batch):
+            for r in sample:
                 for h in range(w.num_kv_heads):
                     tr = orc.last_trace[(oreq[r], l, h)]
                     st = orc.set(oreq[r], l, h)
@@ -120,12 +126,23 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
                             assert np.array_equal(gpu[0][:valid], st.page_k[page][:valid]), where
                             assert np.array_equal(gpu[1][:valid], st.page_v[page][:valid]), where
     stats = run.spin.stats()
-    assert stats["error_bits"] == 0
-    for key in ("selected_partitions", "selected_pages", "tail_pages", "hit_pages", "miss_pages",
-                "evicted_pages", "bypass_pages"):
-        assert stats[key] == orc.counters[key], key
-    assert stats["set_steps"] == orc.counters["steps"]
-    assert stats["pcie_bytes"] == orc.step_bytes()["pcie"]
+    assert stats["error_bits"] == 0, (stats["error_bits"], stats["first_error_site"])
+    # every set of the batch (not only the mirrored requests) must have counted its appends and steps
+    for r in range(w.batch):
+        for l in range(w.num_layers):
+            for h in range(w.num_kv_heads):
+                dd = run.spin.debug_dump(run.reqs[r], l, h, cap_sel, cap_pages, run.budgets[r], 1 << 15)
+                assert dd["n_tokens"] == run.ctx[r] + w.steps and dd["step"] == w.steps, (r, l, h, dd["n_tokens"], dd["step"])
+    if len(sample) == w.batch:
+        for key in ("selected_partitions", "selected_pages", "tail_pages", "hit_pages", "miss_pages",
+                    "evicted_pages", "bypass_pages"):
+            assert stats[key] == orc.counters[key], key
+        assert stats["set_steps"] == orc.counters["steps"]
+        assert stats["pcie_bytes"] == orc.step_bytes()["pcie"]
+    # properties that hold at any size
+    assert stats["set_steps"] == w.batch * w.num_layers * w.num_kv_heads * w.steps
+    assert stats["selected_pages"] == stats["hit_pages"] + stats["miss_pages"]
+    assert stats["bypass_pages"] <= stats["miss_pages"] and stats["pcie_bytes"] == stats["miss_pages"] * 8192
     assert worst_abs <= MAX_ABS * tol_scale and worst_mean <= MEAN_ABS * tol_scale, (worst_abs, worst_mean)
     run.close()
     return dict(max_abs=worst_abs, mean_abs=worst_mean, rel_l2=math.sqrt(rel_num / max(rel_den, 1e-30)),
