@@ -173,6 +173,15 @@ SPIN_API int spin_destroy(spin_ctx *ctx);
  * slots (Section 5.3: per-request GPU buffer, per-head replacement), all empty (cold cache).
  * Synchronous. */
 SPIN_API int spin_request_open(spin_ctx *ctx, int64_t hbm_budget_pages_per_set, int32_t *out_req);
+/* Buffer elasticity (Section 5.3 "Buffer Elasticity"): change the GPU page slots of every set
+ * of an open request between decode steps.  Shrinking reclaims the tail of each set's GPU page
+ * table; a partition with a page in the reclaimed tail becomes non-resident as a whole (the
+ * paper does not say what happens to a straddling partition); its pages and the reclaimed
+ * slots' physical pages go back to the pool.  Growing appends empty slots (SPIN_ERR_BUDGET if
+ * the pool cannot cover them).  Timestamps of surviving pages are untouched.  Synchronous: it
+ * waits for the device before and after.  The policy -- when to resize whom -- is the caller's
+ * (the paper's scheduler); this is the mechanism. */
+SPIN_API int spin_set_budget(spin_ctx *ctx, int32_t req, int64_t hbm_budget_pages_per_set);
 /* Give back the request's pages and segments.  No work of this request may be in flight. */
 SPIN_API int spin_request_close(spin_ctx *ctx, int32_t req);
 

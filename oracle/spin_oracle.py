@@ -392,6 +392,37 @@ class OracleSet:
                 self.page_v[page, : rows.shape[0]] = v_bits[rows]
         self.n_tokens = int(k_bits.shape[0])
 
+    # ---- buffer elasticity (Section 5.3, "Buffer Elasticity") ------------------------------
+    def resize(self, new_slots: int) -> List[Tuple[int, int, int]]:
+        """Change the set's number of GPU page table slots between steps.
+
+        Shrinking reclaims from the TAIL of the table ("we reclaim pages from the tail of the
+        GPU page table to keep the table compact"): slots new_slots.. disappear.  Reading (the
+        paper does not say what happens to a partition that straddles the cut): a partition
+        with any page in the reclaimed tail becomes non-resident as a whole, so its pages below
+        the cut are cleared too.  Growing appends empty slots.  Timestamps of surviving pages
+        are untouched.  Returns the dropped pages as (slot, partition, page_idx) in slot order.
+        """
+        S = self.slot_part.shape[0]
+        dropped: List[Tuple[int, int, int]] = []
+        if new_slots < S:
+            gone = {int(p) for p in self.slot_part[new_slots:] if p >= 0}
+            for s in range(S):
+                p = int(self.slot_part[s])
+                if p >= 0 and (s >= new_slots or p in gone):
+                    dropped.append((s, p, int(self.slot_pidx[s])))
+                    self.part_resident[p] = 0
+                    self.slot_part[s], self.slot_pidx[s], self.slot_ts[s] = -1, 0, -1
+            self.slot_part = self.slot_part[:new_slots].copy()
+            self.slot_pidx = self.slot_pidx[:new_slots].copy()
+            self.slot_ts = self.slot_ts[:new_slots].copy()
+        elif new_slots > S:
+            grow = new_slots - S
+            self.slot_part = np.concatenate([self.slot_part, np.full(grow, -1, dtype=np.int64)])
+            self.slot_pidx = np.concatenate([self.slot_pidx, np.zeros(grow, dtype=np.int64)])
+            self.slot_ts = np.concatenate([self.slot_ts, np.full(grow, -1, dtype=np.int64)])
+        return dropped
+
     # ---- helpers ---------------------------------------------------------------------
     def n_partitions(self) -> int:
         return len(self.part_tokens)
@@ -503,6 +534,12 @@ class SpinOracle:
 
     def request_close(self, req: int):
         del self.requests[req]
+
+    def set_budget(self, req: int, slots_per_set: int):
+        """Resize every (layer, kv head) set of a request (see OracleSet.resize)."""
+        for layer in self.requests[req]:
+            for st in layer:
+                st.resize(slots_per_set)
 
     def set(self, req: int, layer: int, head: int) -> OracleSet:
         return self.requests[req][layer][head]

@@ -22,7 +22,7 @@ PART_PAGE_MINMAX, PART_TOKEN_DOT, PART_CLUSTER_CENTROID = 0, 1, 2
 PAGE_BYTES = 8192
 
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open",
-           "spin_request_close", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
+           "spin_request_close", "spin_set_budget", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
            "spin_decode_step_append", "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
            "spin_debug_read_page", "spin_paged_attention_static", "spin_last_error",
            "spin_version"]
@@ -101,6 +101,7 @@ def load() -> C.CDLL:
     lib.spin_destroy.argtypes = [vp]
     lib.spin_request_open.argtypes = [vp, i64, _I32P]
     lib.spin_request_close.argtypes = [vp, i32]
+    lib.spin_set_budget.argtypes = [vp, i32, i64]
     lib.spin_append_kv.argtypes = [vp, i32, i32, vp, vp, i64, vp, vp, vp]
     lib.spin_append_kv_batch.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
     lib.spin_decode_step.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
@@ -216,6 +217,9 @@ class Spin:
 
     def request_close(self, req: int):
         self._ck(self.lib.spin_request_close(self.h, req))
+
+    def set_budget(self, req: int, budget_pages_per_set: int):
+        self._ck(self.lib.spin_set_budget(self.h, req, budget_pages_per_set))
 
     def append_kv(self, req: int, layer: int, k, v, n_tokens: int, token_partition=None,
                   centroids=None, stream=None):

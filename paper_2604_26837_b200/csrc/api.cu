@@ -789,6 +789,68 @@ int spin_request_close(spin_ctx *ctx, int32_t req) {
   return SPIN_OK;
 }
 
+int spin_set_budget(spin_ctx *ctx, int32_t req, int64_t slots) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  if (req < 0 || req >= ctx->cfg.max_requests) return fail(ctx, SPIN_ERR_INVALID, "request id %d out of range", req);
+  RequestHost &R = ctx->reqs[(size_t)req];
+  if (!R.open) return fail(ctx, SPIN_ERR_STATE, "request %d is not open", req);
+  const Geometry &g = ctx->g;
+  const DevCtx &d = ctx->d;
+  if (slots < 0 || slots > g.max_slots) return fail(ctx, SPIN_ERR_INVALID, "budget %lld outside 0..%lld", (long long)slots, (long long)g.max_slots);
+  const int64_t old = R.slots;
+  if (slots == old) return SPIN_OK;
+  const int64_t sets_per_req = (int64_t)ctx->cfg.num_layers * ctx->cfg.num_kv_heads;
+  CK(cudaDeviceSynchronize());
+  if (slots < old) {
+    // reclaim the tail of every set's GPU page table on the device, then give the pages and
+    // the segments that lie wholly beyond the cut back to their pools
+    ctx->launches += launch_shrink(d, req, (int)old, (int)slots, nullptr);
+    CK(cudaDeviceSynchronize());
+    const int64_t keep_segs = (slots + g.seg - 1) / g.seg;
+    for (int l = 0; l < ctx->cfg.num_layers; ++l)
+      for (int h = 0; h < ctx->cfg.num_kv_heads; ++h) {
+        const int set = set_index(d, req, l, h);
+        SetHost &S = ctx->sets[(size_t)set];
+        for (int64_t s = slots; s < old; ++s) ctx->gpu_page_pool.release(S.gpu_pages[(size_t)s]);
+        S.gpu_pages.resize((size_t)slots);
+        for (int64_t di = keep_segs; di < (int64_t)S.dir_gpt.size(); ++di)
+          if (S.dir_gpt[(size_t)di] >= 0) {
+            ctx->gpt_segs.release(S.dir_gpt[(size_t)di]);
+            ctx->dir_bytes_in_use -= 4;
+            S.dir_gpt[(size_t)di] = -1;
+          }
+        CK(cudaMemcpy(d.dir_gpt + (size_t)set * g.dir_slot, S.dir_gpt.data(), (size_t)g.dir_slot * 4, cudaMemcpyHostToDevice));
+      }
+  } else {
+    const int64_t add = slots - old;
+    const int64_t new_segs = (slots + g.seg - 1) / g.seg - (old + g.seg - 1) / g.seg;
+    if (ctx->gpu_page_pool.available() < add * sets_per_req)
+      return fail(ctx, SPIN_ERR_BUDGET, "growing needs %lld GPU pages, %lld free", (long long)(add * sets_per_req), (long long)ctx->gpu_page_pool.available());
+    if (ctx->gpt_segs.available() < new_segs * sets_per_req) return fail(ctx, SPIN_ERR_OOM_DEVICE, "out of GPU page table segments");
+    for (int l = 0; l < ctx->cfg.num_layers; ++l)
+      for (int h = 0; h < ctx->cfg.num_kv_heads; ++h) {
+        const int set = set_index(d, req, l, h);
+        SetHost &S = ctx->sets[(size_t)set];
+        for (int64_t s = old; s < slots; ++s) {
+          const size_t di = (size_t)(s >> g.seg_shift);
+          if (S.dir_gpt[di] < 0) {
+            S.dir_gpt[di] = (int32_t)ctx->gpt_segs.alloc();
+            ctx->dir_bytes_in_use += 4;
+          }
+          const int32_t phys = (int32_t)ctx->gpu_page_pool.alloc();
+          S.gpu_pages.push_back(phys);
+          const GptEntry e{-1, phys, 0, -1};
+          CK(cudaMemcpy(d.gpt_pool + ((size_t)S.dir_gpt[di] << g.seg_shift) + (s & (g.seg - 1)), &e, sizeof e, cudaMemcpyHostToDevice));
+        }
+        CK(cudaMemcpy(d.dir_gpt + (size_t)set * g.dir_slot, S.dir_gpt.data(), (size_t)g.dir_slot * 4, cudaMemcpyHostToDevice));
+        const int32_t ns = (int32_t)slots;
+        CK(cudaMemcpy(&d.state[set].slots, &ns, 4, cudaMemcpyHostToDevice));
+      }
+  }
+  R.slots = slots;
+  return SPIN_OK;
+}
+
 int spin_append_kv(spin_ctx *ctx, int32_t req, int32_t layer, const void *k, const void *v,
                    int64_t n_tokens, const int32_t *token_partition, const void *centroids,
                    void *cuda_stream) {

@@ -53,6 +53,34 @@ k_cache(DevCtx c, Batch bt, int fast) {
   cache_fast<kCacheThreads>(c, bt, b, i_req, set, L, np, shm.fast);
 }
 
+// Buffer elasticity (Section 5.3): shrink a request's sets from old_S to new_S slots by
+// reclaiming the tail of the GPU page table.  A partition with a page in the reclaimed tail
+// becomes non-resident as a whole, so its pages below the cut are cleared as well.
+// One CTA per (layer, kv head) set of the request.
+__global__ void __launch_bounds__(256)
+k_shrink(DevCtx c, int req, int old_S, int new_S) {
+  const int set = req * c.num_layers * c.Hkv + blockIdx.x, tid = threadIdx.x;
+  for (int s = new_S + tid; s < old_S; s += 256) {
+    const GptEntry *e = gpt_at(c, set, s);
+    if (!e) { dev_error(c, kErrBounds); continue; }
+    if (e->partition >= 0) {
+      MetaEntry *m = meta_at(c, set, e->partition);
+      if (m) m->resident = 0;
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  for (int s = tid; s < old_S; s += 256) {
+    GptEntry *e = gpt_at(c, set, s);
+    if (!e) continue;
+    const int part = e->partition;
+    if (part < 0) continue;
+    const MetaEntry *m = meta_at(c, set, part);
+    if (s >= new_S || (m && m->resident == 0)) { e->partition = -1; e->page_idx = 0; e->ts = -1; }
+  }
+  if (tid == 0) c.state[set].slots = new_S;
+}
+
 // One warp per missed page: 8 KiB = 16 x (32 lanes x 16 B), all loads issued before the
 // stores so that a warp keeps a whole page in flight on the host link.
 __global__ void __launch_bounds__(256)
@@ -89,6 +117,11 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
   }
   launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b, fast);
   prof_mark(prof, st, kProfCache);
+  return 1;
+}
+
+int launch_shrink(const DevCtx &c, int req, int old_S, int new_S, cudaStream_t st) {
+  k_shrink<<<c.num_layers * c.Hkv, 256, 0, st>>>(c, req, old_S, new_S);
   return 1;
 }
 

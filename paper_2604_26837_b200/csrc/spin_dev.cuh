@@ -281,6 +281,7 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
                   const __nv_bfloat16 *v_new, int max_cand, cudaStream_t st, Prof *prof);
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
 int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
+int launch_shrink(const DevCtx &c, int req, int old_S, int new_S, cudaStream_t st);
 size_t cache_smem_bytes(const DevCtx &c);
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
                      __nv_bfloat16 *out, int max_pages_hint, bool may_be_empty, cudaStream_t st, Prof *prof);

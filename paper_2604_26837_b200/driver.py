@@ -48,7 +48,7 @@ class SpinRun:
 
     def __init__(self, w: W.Workload, device="cuda:0", trace=False, sm_scale=0.0,
                  slots_per_set=None, segment_entries=0, fetch_mode=0, host_tables_only=0,
-                 cache_pages_per_layer=None):
+                 cache_pages_per_layer=None, spare_cache_pages=0):
         self.w = w
         self.device = torch.device(device)
         T = w.page_tokens
@@ -71,7 +71,7 @@ class SpinRun:
             max_selected_pages=(w.topk * w.max_partition_pages if cluster else 0),
             max_tail_tokens=(w.steps + T if cluster else 0), lru_buckets=w.lru_buckets,
             segment_entries=segment_entries, sm_scale=sm_scale, trace=1 if trace else 0, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
-            gpu_cache_pages=sum(self.budgets) * sets_per_req, host_pages=host_pages)
+            gpu_cache_pages=sum(self.budgets) * sets_per_req + spare_cache_pages, host_pages=host_pages)
         self.spin = B.Spin(cfg, self.device)
         self.reqs: List[int] = [self.spin.request_open(bud) for bud in self.budgets]
         self.ctx = ctx
@@ -108,6 +108,11 @@ class SpinRun:
     def step(self, layer: int, k_new, v_new, q, out, stream=None):
         """Append one token per request and decode, in one library call."""
         self.spin.decode_step_append(layer, self.reqs, k_new, v_new, q, out, stream)
+
+    def set_budget(self, r: int, slots: int):
+        """Resize the GPU slots of every set of request r (buffer elasticity)."""
+        self.spin.set_budget(self.reqs[r], slots)
+        self.budgets[r] = slots
 
     def close(self):
         self.spin.close()

@@ -28,14 +28,14 @@ def _wl(kind, **kw):
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
                one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None,
-               oracle_reqs=None):
+               oracle_reqs=None, budget_schedule=None, spare_cache_pages=0):
     """oracle_reqs: the requests mirrored in the oracle (default all).  Sets are independent, so the
     oracle run on a sample of the batch's requests must agree with those requests of the full batch."""
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
                   segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
-                  cache_pages_per_layer=cache_pages_per_layer)
+                  cache_pages_per_layer=cache_pages_per_layer, spare_cache_pages=spare_cache_pages)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
@@ -66,6 +66,10 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     cap_pages = w.topk * max(1, w.max_partition_pages) + (w.steps + 16) // 16 + 2
     worst_abs, worst_mean, rel_num, rel_den = 0.0, 0.0, 0.0, 0.0
     for step in range(w.steps):
+        for r, new_slots in (budget_schedule or {}).get(step, {}).items():     # buffer elasticity between steps
+            run.set_budget(r, new_slots)
+            if r in oreq:
+                orc.set_budget(oreq[r], new_slots)
         for l in range(w.num_layers):
             kn, vn = run.gen_step_tokens(l, step)
             kb, vb = W.to_bits(kn), W.to_bits(vn)
@@ -221,6 +225,16 @@ def test_mixed_context_lengths_and_per_request_budgets():
             drift_choices=(0.01, 0.1, 0.5), topk=10, steps=30, lru_buckets=8)
     r = run_parity(w, cache_pages_per_layer=2 * 5 * 12, one_call=True)
     assert r["stats"]["evicted_pages"] > 0
+
+
+@pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_CLUSTER_CENTROID])
+def test_budget_shrinks_and_grows_between_steps(kind):
+    # request 0: 20 -> 9 slots (mid-segment cut with 16-entry segments) -> 33 -> 0 -> 12; request 1: 20 -> 26 -> 5
+    extra = dict(kv_recipe="mixture", num_clusters=29, max_partition_pages=8) if kind == W.PART_CLUSTER_CENTROID else {}
+    w = _wl(kind, steps=34, topk=7, slots_per_set=20, lru_buckets=4, **extra)
+    sched = {6: {0: 9}, 11: {0: 33, 1: 26}, 19: {0: 0}, 23: {0: 12, 1: 5}}
+    r = run_parity(w, segment_entries=16, budget_schedule=sched, spare_cache_pages=2 * 2 * 40, one_call=True)
+    assert r["stats"]["bypass_pages"] > 0 and r["stats"]["evicted_pages"] > 0
 
 
 def test_empty_and_short_contexts():

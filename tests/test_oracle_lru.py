@@ -180,3 +180,54 @@ def test_overflow_bypasses_whole_partitions_and_keeps_hits():
     r1 = O.bucketed_lru_step(part, pidx, ts, resident, npages, [0, 1, 2, 3, 4], 1, n)
     assert r1.hits == [0] and r1.bypass == [1, 3]
     assert list(part) == [0, 0, 2, 4] and list(resident) == [1, 0, 1, 0, 1]
+
+
+def _set_with(slots, parts):
+    """An oracle set whose slot array is `slots` = [(partition, page_idx, ts) or None, ...]."""
+    st = O.OracleSet(O.OracleConfig(1, 1, 1), len(slots))
+    st.part_tokens = [16 * n for n in parts]
+    st.part_resident = [0] * len(parts)
+    st.part_offset = list(np.cumsum([0] + parts[:-1]))
+    for s, e in enumerate(slots):
+        if e is not None:
+            st.slot_part[s], st.slot_pidx[s], st.slot_ts[s] = e
+            st.part_resident[e[0]] = 1
+    return st
+
+
+def test_shrink_reclaims_the_tail_and_whole_straddling_partitions():
+    # partition 0: 2 pages in slots 0,5; partition 1: slot 1; partition 2: 2 pages in slots 2,3
+    st = _set_with([(0, 0, 3), (1, 0, 2), (2, 0, 1), (2, 1, 1), None, (0, 1, 3)], [2, 1, 2])
+    dropped = st.resize(4)
+    # slot 5 is cut: partition 0 straddles the cut, so its page in slot 0 goes as well
+    assert dropped == [(0, 0, 0), (5, 0, 1)]
+    assert list(st.slot_part) == [-1, 1, 2, 2] and list(st.slot_ts) == [-1, 2, 1, 1]
+    assert st.part_resident == [0, 1, 1]
+
+
+def test_grow_appends_empty_slots_and_keeps_timestamps():
+    st = _set_with([(1, 0, 2), None, (0, 0, 0)], [1, 1])
+    assert st.resize(5) == []
+    assert list(st.slot_part) == [1, -1, 0, -1, -1] and list(st.slot_ts) == [2, -1, 0, -1, -1]
+    assert st.part_resident == [1, 1]
+    assert st.resize(5) == []                                   # no-op
+
+
+def test_resize_then_lru_equals_fresh_simulation_of_survivors():
+    # after a shrink the set behaves exactly like one that only ever held the surviving pages
+    rng = np.random.default_rng(11)
+    P, n = 40, 6
+    npages = np.ones(P, dtype=np.int64)
+    a = O.OracleSet(O.OracleConfig(1, 1, 1, lru_buckets=n), 12)
+    a.part_tokens, a.part_resident, a.part_offset = [16] * P, [0] * P, list(range(P))
+    for t in range(10):
+        sel = sorted(set(int(x) for x in rng.integers(0, P, size=4)))
+        res = np.asarray(a.part_resident, dtype=np.int64)
+        O.bucketed_lru_step(a.slot_part, a.slot_pidx, a.slot_ts, res, npages, sel, t, n)
+        a.part_resident = [int(x) for x in res]
+    before = [(int(p), int(ts)) for p, ts in zip(a.slot_part[:7], a.slot_ts[:7])]
+    a.resize(7)
+    assert [(int(p), int(ts)) for p, ts in zip(a.slot_part, a.slot_ts)] == before   # single-page partitions
+    assert sum(a.part_resident) == int((a.slot_part >= 0).sum())
+    occ = {int(p) for p in a.slot_part if p >= 0}
+    assert occ == {p for p in range(P) if a.part_resident[p]}
