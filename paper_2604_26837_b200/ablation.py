@@ -1,0 +1,90 @@
+"""Synthetic re-creation of the paper's buffer-management ablations (Section 6.5): decode
+throughput and GPU hit ratio of one workload as the per-set HBM budget goes from nothing
+("Base": every selected page crosses the host link), to the mandatory pages only
+("+Mandatory": room for one step's selection, i.e. only last step's pages can hit), to
+multiples of it ("+Buffering": the bucketed LRU keeps older pages).
+
+    python -m paper_2604_26837_b200.ablation [--workload c2] [--batch 2] [--steps 96]
+
+Prints one line per budget.  Marshalling and timing only; every stage runs in the library.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+import workloads as W
+
+from .driver import SpinRun
+
+
+def run_budget(w: W.Workload, slots: int, steps: int, prime: int, device="cuda:0") -> dict:
+    run = SpinRun(W.scaled(w, steps=steps + prime + 2), device, slots_per_set=slots)
+    stream = torch.cuda.Stream(device)
+    B, L = w.batch, w.num_layers
+    with torch.cuda.stream(stream):
+        for r in range(B):
+            for l in range(L):
+                k, v, tp, cen = run.gen_prefill(r, l)
+                run.prefill(r, l, k, v, tp, cen, stream)
+        qs = {(r, l): W.QueryStream(w, r, l, device) for r in range(B) for l in range(L)}
+        out = torch.zeros(B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=device)
+        ins = []
+        for s in range(prime + steps):
+            for l in range(L):
+                kn, vn = run.gen_step_tokens(l, s)
+                q = torch.stack([qs[(r, l)].next() for r in range(B)]).contiguous()
+                ins.append((l, kn, vn, q))
+        per_step = L
+        for i in range(prime * per_step):
+            run.step(*ins[i], out, stream)
+        torch.cuda.synchronize(device)
+        st0 = run.spin.stats()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(prime * per_step, (prime + steps) * per_step):
+            run.step(*ins[i], out, stream)
+        e1.record(stream)
+    torch.cuda.synchronize(device)
+    st1 = run.spin.stats()
+    ms = e0.elapsed_time(e1)
+    sel = st1["selected_pages"] - st0["selected_pages"]
+    hit = st1["hit_pages"] - st0["hit_pages"]
+    res = dict(slots=slots, tokens_per_s=B * steps / (ms * 1e-3), ms_per_step=ms / steps,
+               hit_ratio=hit / max(sel, 1), bypass_pages=st1["bypass_pages"] - st0["bypass_pages"],
+               pcie_mb_per_step=(st1["pcie_bytes"] - st0["pcie_bytes"]) / steps / 1e6,
+               error_bits=st1["error_bits"])
+    run.close()
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--batch", type=int, default=2)
+    ap.add_argument("--steps", type=int, default=96)
+    ap.add_argument("--prime", type=int, default=32)
+    args = ap.parse_args()
+    w = W.scaled(W.CONFIGS[args.workload], batch=args.batch)
+    mandatory = w.topk * max(1, w.max_partition_pages // 2 if w.partition_kind == W.PART_CLUSTER_CENTROID else 1)
+    if w.partition_kind == W.PART_TOKEN_DOT:
+        mandatory = 512
+    rows = []
+    for mult, label in ((0, "Base (no GPU buffer)"), (1, "+Mandatory (1x)"), (2, "+Buffering 2x"), (3, "+Buffering 3x"),
+                        (4, "+Buffering 4x"), (5, "+Buffering 5x"), (6, "+Buffering 6x"), (8, "+Buffering 8x")):
+        r = run_budget(w, mandatory * mult, args.steps, args.prime)
+        r["label"], r["x_mandatory"] = label, mult
+        rows.append(r)
+        print(json.dumps(r), flush=True)
+    base = rows[1]["tokens_per_s"]
+    print("\n| budget | slots/set | hit ratio | host-link MB/step | ms/step | tokens/s | vs +Mandatory |")
+    print("|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['label']} | {r['slots']} | {r['hit_ratio']:.3f} | {r['pcie_mb_per_step']:.2f} | "
+              f"{r['ms_per_step']:.3f} | {r['tokens_per_s']:.0f} | {r['tokens_per_s'] / base:.2f}x |")
+
+
+if __name__ == "__main__":
+    main()
