@@ -63,8 +63,11 @@ typedef enum spin_partition_kind {
   SPIN_PART_TOKEN_DOT = 1,        /* partition = one token scored by q.k; the selected tokens
                                      are cached and fetched as their containing pages and
                                      attended through a per-page token mask */
-  SPIN_PART_CLUSTER_CENTROID = 2  /* partition = caller-given cluster of tokens packed into
+  SPIN_PART_CLUSTER_CENTROID = 2, /* partition = caller-given cluster of tokens packed into
                                      1..n pages; summary = centroid; score = q.centroid */
+  SPIN_PART_PAGE_MEAN = 3         /* partition = one page; summary = mean of its keys (Table 1,
+                                     ShadowKV's Index: landmarks), keys added in token order in
+                                     fp32, x 1/16, rounded to bf16; score = q.mean */
 } spin_partition_kind;
 
 /* Bits of spin_stats_t.error_bits (set on the device, sticky). */

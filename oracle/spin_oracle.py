@@ -39,8 +39,16 @@ import numpy as np
 PART_PAGE_MINMAX = 0
 PART_TOKEN_DOT = 1
 PART_CLUSTER_CENTROID = 2
+PART_PAGE_MEAN = 3
 
 F32 = np.float32
+
+
+def f32_to_bf16_f32(x: np.ndarray) -> np.ndarray:
+    """Round fp32 to the nearest bf16 (ties to even) and widen back to fp32 (finite inputs)."""
+    b = np.asarray(x, dtype=np.float32).view(np.uint32)
+    r = (b + np.uint32(0x7FFF) + ((b >> 16) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32)
 
 
 def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
@@ -348,6 +356,14 @@ class OracleSet:
             self._grow_rows("sum_max", p + 1)
             self.sum_min[p] = keys.min(axis=0)
             self.sum_max[p] = keys.max(axis=0)
+        elif self.kind == PART_PAGE_MEAN:
+            # landmark = mean of the page's keys (Table 1, ShadowKV's Index).  Reading (the paper
+            # gives no precision): keys added in token order in fp32, times 1/T, rounded to bf16
+            self._grow_rows("sum_vec", p + 1)
+            acc = keys[0].astype(F32)
+            for r in range(1, self.T):
+                acc = (acc + keys[r]).astype(F32)
+            self.sum_vec[p] = f32_to_bf16_f32((acc * F32(1.0 / self.T)).astype(F32))
         else:                                                     # token granularity
             self._grow_rows("sum_vec", (p + 1) * self.T)
             self.sum_vec[p * self.T:(p + 1) * self.T] = keys

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libspin.so")
 SPIN_OK = 0
 STATUS_NAMES = {0: "SPIN_OK", 1: "SPIN_ERR_INVALID", 2: "SPIN_ERR_STATE", 3: "SPIN_ERR_OOM_DEVICE",
                 4: "SPIN_ERR_OOM_HOST", 5: "SPIN_ERR_BUDGET", 6: "SPIN_ERR_CUDA", 7: "SPIN_ERR_TIMEOUT"}
-PART_PAGE_MINMAX, PART_TOKEN_DOT, PART_CLUSTER_CENTROID = 0, 1, 2
+PART_PAGE_MINMAX, PART_TOKEN_DOT, PART_CLUSTER_CENTROID, PART_PAGE_MEAN = 0, 1, 2, 3
 PAGE_BYTES = 8192
 
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open",

@@ -90,7 +90,7 @@ int compute_geometry(const spin_config &cfg, Geometry &g, std::string &err) {
   if (G != 1 && G != 2 && G != 4 && G != 8) return bad("group size must be 1, 2, 4 or 8");
   if (cfg.max_requests < 1 || cfg.max_requests > kMaxBatch) return bad("max_requests must be 1..256");
   if (cfg.max_context_tokens < 1 || cfg.max_context_tokens > (1ll << 26)) return bad("bad max_context_tokens");
-  if (cfg.partition_kind < 0 || cfg.partition_kind > 2) return bad("bad partition_kind");
+  if (cfg.partition_kind < 0 || cfg.partition_kind > 3) return bad("bad partition_kind");
   if (cfg.topk < 1 || cfg.topk > 4096) return bad("topk must be 1..4096");
   if (cfg.lru_buckets < 1 || cfg.lru_buckets > kMaxBuckets) return bad("lru_buckets must be 1..64");
   if (cfg.gpu_cache_pages < 0 || cfg.host_pages < 1) return bad("bad page counts");

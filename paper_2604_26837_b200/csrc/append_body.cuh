@@ -29,6 +29,21 @@ __device__ __forceinline__ void write_minmax(const DevCtx &c, int set, int part,
   }
 }
 
+// Landmark summary (Table 1, ShadowKV's Index: mean(paged_key, dim=dim_page)): per channel the
+// 16 keys are added in token order in fp32, scaled by 1/16 (exact) and rounded to bf16
+// (nearest even) -- the order and rounding the CPU oracle uses.
+__device__ __forceinline__ void write_mean(const DevCtx &c, int set, int part,
+                                           const __nv_bfloat16 (*krows)[kHeadDim], int tid) {
+  if (tid < kHeadDim) {
+    float s = __bfloat162float(krows[0][tid]);
+#pragma unroll
+    for (int r = 1; r < kPageTokens; ++r) s = s + __bfloat162float(krows[r][tid]);
+    uint8_t *dst = summary_at(c, set, part);
+    if (!dst) { dev_error(c, 1u); return; }
+    reinterpret_cast<__nv_bfloat16 *>(dst)[tid] = __float2bfloat16_rn(s * 0.0625f);
+  }
+}
+
 __device__ __forceinline__ void write_token_summaries(const DevCtx &c, int set, int part,
                                                       const __nv_bfloat16 (*krows)[kHeadDim], int tid) {
   uint8_t *s = summary_at(c, set, part * kPageTokens);
@@ -40,6 +55,7 @@ __device__ __forceinline__ void write_token_summaries(const DevCtx &c, int set, 
 __device__ __forceinline__ void index_page(const DevCtx &c, int set, int part,
                                            const __nv_bfloat16 (*krows)[kHeadDim], int tid) {
   if (c.kind == kKindPage) write_minmax(c, set, part, krows, tid);
+  else if (c.kind == kKindPageMean) write_mean(c, set, part, krows, tid);
   else write_token_summaries(c, set, part, krows, tid);
   if (tid == 0) {
     MetaEntry *m = meta_at(c, set, part);

@@ -19,7 +19,7 @@ constexpr int kPageBytes = 2 * kHalfPageBytes;              // K rows then V row
 constexpr int kMaxBatch = 256;                              // requests per decode step
 constexpr int kMaxBuckets = 64;
 
-enum : int { kKindPage = 0, kKindToken = 1, kKindCluster = 2 };
+enum : int { kKindPage = 0, kKindToken = 1, kKindCluster = 2, kKindPageMean = 3 };
 // sticky device error bits (same values as SPIN_DEV_ERR_* of the public header)
 constexpr unsigned kErrBounds = 1u, kErrPageList = 2u, kErrTimeout = 4u;
 constexpr int kChunkPages = 8;                              // pages per attention split

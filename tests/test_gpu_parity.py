@@ -237,6 +237,13 @@ def test_budget_shrinks_and_grows_between_steps(kind):
     assert r["stats"]["bypass_pages"] > 0 and r["stats"]["evicted_pages"] > 0
 
 
+@pytest.mark.parametrize("sm_scale", [0.0, 1.0])
+def test_page_mean_landmarks(sm_scale):
+    # mean-pooled page summaries (Table 1, ShadowKV's Index) scored by q . mean
+    w = _wl(W.PART_PAGE_MEAN, steps=36, topk=7, slots_per_set=18, lru_buckets=8, kv_recipe="page_centre")
+    run_parity(w, sm_scale=sm_scale, one_call=True)
+
+
 def test_empty_and_short_contexts():
     # fewer candidates than top-k, and a context shorter than one page (no candidate at all)
     run_parity(_wl(W.PART_PAGE_MINMAX, context=16 * 3 + 2, topk=8, steps=20))

@@ -108,3 +108,36 @@ def test_topk_tie_goes_to_lower_index_and_zero_signs_tie():
     s = np.array([-0.0, 0.0, -1.0], dtype=F32)
     assert list(O.topk_select(s, 1)) == [0]
     assert list(O.topk_select(s, 10)) == [0, 1, 2]
+
+
+def _mean_set(keys_bits):
+    """An oracle set of the landmark kind holding one indexed page made of `keys_bits` (16 rows)."""
+    cfg = O.OracleConfig(1, 1, 1, partition_kind=O.PART_PAGE_MEAN)
+    st = O.OracleSet(cfg, 4)
+    st.append_tokens(keys_bits, keys_bits)
+    st.append_tokens(keys_bits[:1], keys_bits[:1])          # first token of the next page indexes it
+    return st
+
+
+def test_mean_summary_special_cases_and_rounding():
+    rng = np.random.default_rng(9)
+    one = _rand_bf16(rng, (1, 128))
+    st = _mean_set(np.repeat(one, 16, axis=0))              # 16 equal keys: the mean is the key
+    assert np.array_equal(st.sum_vec[0], O.bf16_to_f32(one[0]))
+    pair = np.concatenate([one, one ^ np.uint16(0x8000)] * 8)   # x, -x, x, -x ...: the mean is 0
+    assert np.array_equal(_mean_set(pair).sum_vec[0], np.zeros(128, dtype=F32))
+    keys = _rand_bf16(rng, (16, 128), scale=3.0)
+    got = _mean_set(keys).sum_vec[0]
+    exact = O.bf16_to_f32(keys).astype(np.float64).mean(axis=0)
+    assert np.array_equal(got, O.f32_to_bf16_f32(got))      # a bf16 value
+    # within half a bf16 ulp of the exact mean (plus the fp32 summation error, far smaller)
+    assert (np.abs(got - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30).all()
+    # small integers: exact arithmetic, so the value is fixed whatever the order
+    ints = rng.integers(-8, 8, size=(16, 128)).astype(np.float32)
+    ibits = (ints.view(np.uint32) >> 16).astype(np.uint16)
+    assert np.array_equal(_mean_set(ibits).sum_vec[0], O.f32_to_bf16_f32((ints.sum(axis=0) / 16).astype(F32)))
+
+
+def test_bf16_rounding_is_nearest_even():
+    x = np.array([1.0, 1.00390625, 1.01171875, 1.005859375 + 2 ** -20], dtype=F32)   # exact, tie->even, tie->even, above tie
+    assert list(O.f32_to_bf16_f32(x)) == [1.0, 1.0, 1.015625, 1.0078125]

@@ -25,6 +25,7 @@ import torch
 PART_PAGE_MINMAX = 0
 PART_TOKEN_DOT = 1
 PART_CLUSTER_CENTROID = 2
+PART_PAGE_MEAN = 3
 
 _M64 = (1 << 64) - 1
 
