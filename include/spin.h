@@ -74,6 +74,8 @@ typedef enum spin_partition_kind {
 #define SPIN_DEV_ERR_BOUNDS 1u      /* an index left its table; the access was skipped */
 #define SPIN_DEV_ERR_PAGE_LIST 2u   /* a set selected more pages than max_selected_pages */
 #define SPIN_DEV_ERR_TIMEOUT 4u     /* a bounded wait ran out */
+#define SPIN_DEV_ERR_STATE 8u       /* a per-set state word disagreed with the host's count (the host's
+                                       count was used and the word rewritten) */
 
 typedef struct spin_config {
   uint32_t struct_size;         /* sizeof(spin_config), for versioning */
@@ -133,6 +135,8 @@ typedef struct spin_stats_t {
   uint64_t host_pages_in_use;
   uint64_t first_error_site;      /* where the first device-side check tripped: source file id x
                                      100000 + line (1 append, 2 select, 3 cache, 4 attention); 0 = none */
+  uint32_t debug_words[4];        /* first SPIN_DEV_ERR_STATE: set index + 1, the device's token count,
+                                     the host's, the decode call's number (-1: stand-alone append) */
 } spin_stats_t;
 
 /* Logical view of one set after its last decode step (what the parity tests compare).

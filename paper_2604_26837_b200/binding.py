@@ -54,7 +54,8 @@ class spin_stats_t(C.Structure):
                                   "hit_pages", "miss_pages", "evicted_pages", "bypass_pages",
                                   "candidates_scored", "pcie_bytes", "hbm_bytes", "kernel_launches",
                                   "gpu_meta_bytes", "host_meta_bytes", "summary_bytes",
-                                  "gpu_pages_in_use", "host_pages_in_use", "first_error_site")]
+                                  "gpu_pages_in_use", "host_pages_in_use", "first_error_site")] + [
+        ("debug_words", C.c_uint32 * 4)]
 
 
 class spin_profile_t(C.Structure):
@@ -245,7 +246,9 @@ class Spin:
         s = spin_stats_t()
         s.struct_size = C.sizeof(spin_stats_t)
         self._ck(self.lib.spin_stats(self.h, C.byref(s)))
-        return {n: getattr(s, n) for n, _ in spin_stats_t._fields_ if n != "struct_size"}
+        out = {n: getattr(s, n) for n, _ in spin_stats_t._fields_ if n not in ("struct_size", "debug_words")}
+        out["debug_words"] = list(s.debug_words)
+        return out
 
     def profile(self, enable: bool):
         self._ck(self.lib.spin_profile(self.h, 1 if enable else 0))

@@ -384,6 +384,7 @@ int append_paged_device(spin_ctx *ctx, int req, int layer, const __nv_bfloat16 *
   a.n_req = 1;
   a.layer = layer;
   a.req[0] = req;
+  a.n_tokens[0] = (int32_t)n0;
   ctx->launches += launch_append_edge(ctx->d, a, k, v, (int)n, st, &ctx->prof);
   return SPIN_OK;
 }
@@ -885,6 +886,7 @@ int spin_append_kv(spin_ctx *ctx, int32_t req, int32_t layer, const void *k, con
       if (rc) return rc;
       AppendEdgeArgs a{};
       a.n_req = 1; a.layer = layer; a.req[0] = req;
+      a.n_tokens[0] = (int32_t)(L.n_tokens - m);
       ctx->launches += launch_append_edge(ctx->d, a, kk, vv, (int)m, st, &ctx->prof);
     } else {
       rc = append_paged_device(ctx, req, layer, kk, vv, m, st);
@@ -916,6 +918,7 @@ int spin_append_kv_batch(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, i
     if (cluster && !L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req_ids[i]);
     int rc = cluster ? grow_cluster_tail(ctx, req_ids[i], layer, 1, st) : grow_paged(ctx, req_ids[i], layer, L.n_tokens + 1, st);
     if (rc) return rc;
+    a.n_tokens[i] = (int32_t)(L.n_tokens - 1);
   }
   const __nv_bfloat16 *kk = reinterpret_cast<const __nv_bfloat16 *>(k), *vv = reinterpret_cast<const __nv_bfloat16 *>(v);
   if (!is_device_ptr(k)) {
@@ -984,7 +987,10 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
       AppendEdgeArgs a{};
       a.n_req = n_req;
       a.layer = layer;
-      for (int i = 0; i < n_req; ++i) a.req[i] = req_ids[i];
+      for (int i = 0; i < n_req; ++i) {
+        a.req[i] = req_ids[i];
+        a.n_tokens[i] = (int32_t)(ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer].n_tokens - 1);
+      }
       prof_mark(&ctx->prof, st, -1);
       ctx->launches += launch_append_edge(ctx->d, a, kk, vv, 1, st, &ctx->prof);
     }
@@ -1004,6 +1010,7 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     b.slots[i] = (int32_t)ctx->reqs[(size_t)req_ids[i]].slots;
     b.step[i] = L.steps++;
     b.n_partitions[i] = L.n_partitions;
+    b.n_tokens[i] = (int32_t)(L.n_tokens - (with_append ? 1 : 0));
   }
   const __nv_bfloat16 *qd = reinterpret_cast<const __nv_bfloat16 *>(q);
   __nv_bfloat16 *od = reinterpret_cast<__nv_bfloat16 *>(out);
@@ -1048,6 +1055,7 @@ int spin_stats(spin_ctx *ctx, spin_stats_t *out) {
   const Geometry &g = ctx->g;
   out->error_bits = c.error_bits;
   out->first_error_site = c.first_site;
+  for (int i = 0; i < 4; ++i) out->debug_words[i] = c.dbg[i];
   out->set_steps = c.set_steps;
   out->selected_partitions = c.selected_partitions;
   out->selected_pages = c.selected_pages;

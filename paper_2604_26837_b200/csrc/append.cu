@@ -43,7 +43,7 @@ k_append_edge(DevCtx c, AppendEdgeArgs a, const __nv_bfloat16 *__restrict__ k,
   const int head = blockIdx.x, i = blockIdx.y;
   pdl_launch_next();
   pdl_wait_prev();
-  append_edge_body(c, set_index(c, a.req[i], a.layer, head), i, head, k, v, n_new, krows);
+  append_edge_body(c, set_index(c, a.req[i], a.layer, head), i, head, k, v, n_new, a.n_tokens[i], -1, krows);
 }
 
 // Cluster prefill: row `tok` of head `h` goes to row dest[tok][h] of the host tier (page id *

@@ -72,11 +72,20 @@ __device__ __forceinline__ void index_page(const DevCtx &c, int set, int part,
 __device__ __forceinline__ void append_edge_body(const DevCtx &c, int set, int i, int head,
                                                  const __nv_bfloat16 *__restrict__ k,
                                                  const __nv_bfloat16 *__restrict__ v, int n_new,
-                                                 __nv_bfloat16 (*krows)[kHeadDim]) {
+                                                 int n0_host, int epoch, __nv_bfloat16 (*krows)[kHeadDim]) {
   const int tid = threadIdx.x;
   const int r = tid >> 4, piece = tid & 15;
   SetState st = c.state[set];
-  const int n0 = st.n_tokens, n1 = n0 + n_new;
+  __syncthreads();       // every thread has read the state before thread 0 rewrites it at the end
+  // the host has counted every append; its count is the one used, and a device word that
+  // disagrees is reported (it is rewritten below)
+  if (threadIdx.x == 0 && st.n_tokens != n0_host) {
+    dev_error(c, kErrState);
+    if (atomicCAS(&c.counters->dbg[0], 0u, (unsigned)set + 1u) == 0u) {
+      c.counters->dbg[1] = (unsigned)st.n_tokens; c.counters->dbg[2] = (unsigned)n0_host; c.counters->dbg[3] = (unsigned)epoch;
+    }
+  }
+  const int n0 = n0_host, n1 = n0 + n_new;
   const uint8_t *kin = reinterpret_cast<const uint8_t *>(k) + (size_t)i * n_new * c.Hkv * kRowBytes;
   const uint8_t *vin = reinterpret_cast<const uint8_t *>(v) + (size_t)i * n_new * c.Hkv * kRowBytes;
   auto in_off = [&](int tok) { return ((size_t)(tok - n0) * c.Hkv + head) * kRowBytes + piece * 16; };

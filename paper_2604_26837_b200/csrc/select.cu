@@ -84,7 +84,7 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
     // the set's tail CTA: appends this step's token (unless a stand-alone append already ran)
     // and tells the attention kernel that the tail page is complete
     __shared__ __align__(16) __nv_bfloat16 krows[kPageTokens][kHeadDim];
-    if (bt.append_in_grid) append_edge_body(c, set, i_req, head, k_new, v_new, 1, krows);
+    if (bt.append_in_grid) append_edge_body(c, set, i_req, head, k_new, v_new, 1, bt.n_tokens[i_req], bt.epoch, krows);
     __syncthreads();
     if (threadIdx.x == 0) flag_publish(c.tail_ready + b, bt.epoch);
     return;
@@ -222,14 +222,21 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
   // fused: one CTA can hold a set's keys and the cache manager's tables in shared memory
   const size_t cache_smem = cache_stage_smem_bytes(c.max_parts, c.max_pages, c.max_slots);
   int fuse = (max_cand <= 16384 && cache_smem <= 96 * 1024) ? 1 : 0;
-  const int keys_cap = fuse ? max_cand : 0;
+  int keys_cap = fuse ? max_cand : 0;
   size_t smem = 0;
   if (fuse) smem = cache_smem > (size_t)keys_cap * 4 ? cache_smem : (size_t)keys_cap * 4;
-  if (fuse && c.kind != kKindToken) {
+  {
+    // the low-latency continuation: keys (unless token-granular) and the whole GPU page table
+    // of a set in shared memory
     int max_slots_batch = 0;
     for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
-    if (max_slots_batch <= kFastSlots && fs <= 64 * 1024) { fuse = 2; smem = fs > smem ? fs : smem; }
+    const bool token = c.kind == kKindToken;
+    const size_t fs = fast_smem_bytes(token ? 0 : max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
+    if (max_slots_batch <= kFastSlots && (token || max_cand <= 16384) && fs <= (token ? 100 : 64) * 1024) {
+      fuse = 2;
+      keys_cap = token ? 0 : max_cand;
+      smem = fs;
+    }
   }
   if (smem < 64 * 1024) smem = 64 * 1024;         // the scoring CTAs' staging area: one summary segment
   switch (c.G) {

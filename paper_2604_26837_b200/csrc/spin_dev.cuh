@@ -21,7 +21,7 @@ constexpr int kMaxBuckets = 64;
 
 enum : int { kKindPage = 0, kKindToken = 1, kKindCluster = 2, kKindPageMean = 3 };
 // sticky device error bits (same values as SPIN_DEV_ERR_* of the public header)
-constexpr unsigned kErrBounds = 1u, kErrPageList = 2u, kErrTimeout = 4u;
+constexpr unsigned kErrBounds = 1u, kErrPageList = 2u, kErrTimeout = 4u, kErrState = 8u;
 constexpr int kChunkPages = 8;                              // pages per attention split
 
 // Per-set scalars (device resident, updated only by kernels).
@@ -46,6 +46,7 @@ struct Counters {
       miss_pages, evicted_pages, bypass_pages, candidates_scored;
   unsigned int error_bits;
   unsigned int first_site;   // where the first device-side error was raised (file id * 100000 + line)
+  unsigned int dbg[4];       // payload of the first state mismatch: set, device value, host value, epoch
 };
 
 struct FetchItem { int32_t host_page; int32_t gpu_page; };
@@ -121,6 +122,7 @@ struct Batch {
   int32_t slots[kMaxBatch];
   int32_t step[kMaxBatch];
   int32_t n_partitions[kMaxBatch];
+  int32_t n_tokens[kMaxBatch];   // tokens before this step's append
   int32_t epoch;            // number of this decode call: value of the ready flags it sets
   int32_t append_in_grid;   // the scoring kernel's tail CTAs append this step's tokens
 };
@@ -264,6 +266,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 struct AppendEdgeArgs {     // one (request) per entry; all its kv heads are processed
   int32_t n_req, layer;
   int32_t req[kMaxBatch];
+  int32_t n_tokens[kMaxBatch];   // tokens of the request before this append, as the host has counted them
 };
 int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,

@@ -662,20 +662,26 @@ template <int T>
 __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
                                             uint8_t *dyn, FastShared &sh) {
   const int tid = threadIdx.x;
-  const int n = bt.n_partitions[i_req];
+  // token-granular selection has far more candidates than shared memory holds: its keys are
+  // re-read from the scores (L2 resident: the scoring CTAs have just written them)
+  const bool token = c.kind == kKindToken;
+  const int n = token ? bt.n_partitions[i_req] * kPageTokens : bt.n_partitions[i_req];
   const int k = min(c.topk, n);
   const int S = bt.slots[i_req];
 
-  const FastLayout L = fast_layout(c, dyn, n, S);
+  const FastLayout L = fast_layout(c, dyn, token ? 0 : n, S);
   uint32_t *s_keys = L.s_keys;
   int32_t *s_parts = L.s_parts;
+  int32_t *s_sel = token ? L.s_host : L.s_parts;     // chosen candidates; tokens are folded into pages below
 
   dbg_ts(b, 1);
   // ---- directories on their way (consumed after the keys are loaded) ------------------------
   fast_prefetch_dirs<T>(c, L, set, S);
 
   const float *scores = c.scores + (size_t)b * c.max_cand;
-  for (int i = tid; i < n; i += T) s_keys[i] = order_key(__ldcg(scores + i));
+  if (!token)
+    for (int i = tid; i < n; i += T) s_keys[i] = order_key(__ldcg(scores + i));
+  auto key_at = [&](int i) { return token ? order_key(__ldcg(scores + i)) : s_keys[i]; };
   for (int i = tid; i < 512; i += T) (&sh.hist[0][0])[i] = 0;
   if (tid == 0) {
     sh.lhist[0] = 0u;                        // OR / AND of the keys (reused as the timestamp histogram later)
@@ -694,13 +700,14 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   int32_t *g_sel = c.sel_ids + (size_t)b * c.max_sel;
   int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
   if (k == n) {
-    for (int i = tid; i < n; i += T) { s_parts[i] = i; g_sel[i] = i; g_parts[i] = i; }
+    for (int i = tid; i < n; i += T) { s_sel[i] = i; g_sel[i] = i; }
   } else {
     // The scores of one set share their sign, exponent and often a few mantissa bits, so the
     // leading radix passes would put every key into one bin (and serialise on its counter).
     // Bytes on which all keys agree (OR == AND over the set) are skipped outright.
     uint32_t k_or = 0, k_and = 0xffffffffu;
-    for (int i = tid; i < n; i += T) { const uint32_t key = s_keys[i]; k_or |= key; k_and &= key; }
+#pragma unroll 8
+    for (int i = tid; i < n; i += T) { const uint32_t key = key_at(i); k_or |= key; k_and &= key; }
     k_or = __reduce_or_sync(0xffffffffu, k_or);
     k_and = __reduce_and_sync(0xffffffffu, k_and);
     if ((tid & 31) == 0) { atomicOr(&sh.lhist[0], k_or); atomicAnd(&sh.lhist[1], k_and); }
@@ -715,8 +722,9 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
     }
     int buf = 0;
     for (int shift = first_shift; shift >= 0; shift -= 8, buf ^= 1) {
+#pragma unroll 8
       for (int i = tid; i < n; i += T) {
-        const uint32_t key = s_keys[i];
+        const uint32_t key = key_at(i);
         if ((key & mask) == prefix) atomicAdd(&sh.hist[buf][(key >> shift) & 255u], 1u);
       }
       __syncthreads();
@@ -752,25 +760,59 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
       // the buffer just searched is cleared by the next pass's idle warps (it is used again two passes on)
     }
     const uint32_t thr = prefix, need_eq = remaining;
+    // every thread owns a contiguous run of candidates: two block scans place all of them
     const int E = (n + T - 1) / T, lo = min(n, tid * E), hi = min(n, lo + E);
     uint32_t gt = 0, eq = 0;
-    for (int i = lo; i < hi; ++i) { const uint32_t key = s_keys[i]; gt += key > thr; eq += key == thr; }
-    uint32_t total;
-    const uint32_t ex = block_scan<T>(gt | (eq << 16), sh.wsum, &total);
-    uint32_t gt_before = ex & 0xffffu, eq_before = ex >> 16;
+#pragma unroll 8
+    for (int i = lo; i < hi; ++i) { const uint32_t key = key_at(i); gt += key > thr; eq += key == thr; }
+    uint32_t tot_gt, tot_eq;
+    uint32_t gt_before = block_scan<T>(gt, sh.wsum, &tot_gt);
+    uint32_t eq_before = block_scan<T>(eq, sh.wsum, &tot_eq);
     for (int i = lo; i < hi; ++i) {
-      const uint32_t key = s_keys[i];
+      const uint32_t key = key_at(i);
       if (key > thr || (key == thr && eq_before < need_eq)) {
         const uint32_t pos = gt_before + min(eq_before, need_eq);
-        s_parts[pos] = i; g_sel[pos] = i; g_parts[pos] = i;
+        s_sel[pos] = i; g_sel[pos] = i;
       }
       gt_before += key > thr;
       eq_before += key == thr;
     }
   }
+  __syncthreads();
+  int np = k;
+  if (!token) {
+    for (int i = tid; i < k; i += T) g_parts[i] = s_sel[i];
+  } else {
+    // chosen tokens (ascending) -> their pages (ascending, unique) + a 16-bit token mask per page
+    uint32_t *s_mask = reinterpret_cast<uint32_t *>(L.s_free);
+    for (int i = tid; i < k; i += T) s_mask[i] = 0;
+    __syncthreads();
+    uint32_t run = 0;
+    for (int base = 0; base < k; base += T) {
+      const int i = base + tid;
+      uint32_t first = 0;
+      int tok = 0;
+      if (i < k) {
+        tok = s_sel[i];
+        first = (i == 0) || ((s_sel[i - 1] >> 4) != (tok >> 4));
+      }
+      uint32_t total;
+      const uint32_t ex = block_scan<T>(first, sh.wsum, &total);
+      if (i < k) {
+        const uint32_t rank_ = run + ex + first - 1;
+        if (first) { s_parts[rank_] = tok >> 4; g_parts[rank_] = tok >> 4; }
+        atomicOr(&s_mask[rank_], 1u << (tok & 15));
+      }
+      run += total;
+    }
+    np = (int)run;
+    __syncthreads();
+    uint32_t *g_mask = c.part_mask + (size_t)b * c.max_parts;
+    for (int i = tid; i < np; i += T) g_mask[i] = s_mask[i];
+  }
   dbg_ts(b, 3);
   __syncthreads();
-  cache_fast<T>(c, bt, b, i_req, set, L, k, sh);
+  cache_fast<T>(c, bt, b, i_req, set, L, np, sh);
 }
 
 

@@ -130,7 +130,7 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
                             assert np.array_equal(gpu[0][:valid], st.page_k[page][:valid]), where
                             assert np.array_equal(gpu[1][:valid], st.page_v[page][:valid]), where
     stats = run.spin.stats()
-    assert stats["error_bits"] == 0, (stats["error_bits"], stats["first_error_site"])
+    assert stats["error_bits"] == 0, (stats["error_bits"], stats["first_error_site"], stats["debug_words"])
     # every set of the batch (not only the mirrored requests) must have counted its appends and steps
     for r in range(w.batch):
         for l in range(w.num_layers):
