@@ -381,13 +381,13 @@ def main():
 
     peaks = load_peaks()
     value = aggregate_value(B * K, world, elapsed_ms)
-    d = {k: st1[k] - st0[k] for k in st0 if k != "error_bits"}
+    d = {k: st1[k] - st0[k] for k in st0 if k not in ("error_bits", "debug_words")}
     hbm_step = d["hbm_bytes"] / K
     pcie_step = d["pcie_bytes"] / K
     t_hbm = hbm_step / (peaks["hbm_gbs"] * 1e9)
     t_pcie = pcie_step / (pcie_gbs * 1e9)
     t_step = elapsed_ms * 1e-3 / K
-    dp = {k: stp1[k] - stp0[k] for k in stp0 if k != "error_bits"}
+    dp = {k: stp1[k] - stp0[k] for k in stp0 if k not in ("error_bits", "debug_words")}
     kern = {}
     miss_b = dp["miss_pages"] * PAGE_BYTES
     admit_b = (dp["miss_pages"] - dp["bypass_pages"]) * PAGE_BYTES

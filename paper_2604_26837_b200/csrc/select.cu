@@ -174,7 +174,7 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
   __threadfence();
   if (threadIdx.x == 0) c.sel_count[b] = 0;                 // ready for the next step
   if (fuse == 2) {
-    select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, shm.fast);
+    select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, keys_cap, shm.fast);
     return;
   }
   topk_stage<kScoreThreads, false>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, shm.staged.t);
@@ -226,15 +226,14 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
   size_t smem = 0;
   if (fuse) smem = cache_smem > (size_t)keys_cap * 4 ? cache_smem : (size_t)keys_cap * 4;
   {
-    // the low-latency continuation: keys (unless token-granular) and the whole GPU page table
+    // the low-latency continuation: the keys and the whole GPU page table
     // of a set in shared memory
     int max_slots_batch = 0;
     for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-    const bool token = c.kind == kKindToken;
-    const size_t fs = fast_smem_bytes(token ? 0 : max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
-    if (max_slots_batch <= kFastSlots && (token || max_cand <= 16384) && fs <= (token ? 100 : 64) * 1024) {
+    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
+    if (max_slots_batch <= kFastSlots && max_cand <= 16384 && fs <= 100 * 1024) {
       fuse = 2;
-      keys_cap = token ? 0 : max_cand;
+      keys_cap = max_cand;
       smem = fs;
     }
   }

@@ -660,16 +660,17 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
 
 template <int T>
 __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
-                                            uint8_t *dyn, FastShared &sh) {
+                                            uint8_t *dyn, int keys_cap, FastShared &sh) {
   const int tid = threadIdx.x;
-  // token-granular selection has far more candidates than shared memory holds: its keys are
-  // re-read from the scores (L2 resident: the scoring CTAs have just written them)
   const bool token = c.kind == kKindToken;
   const int n = token ? bt.n_partitions[i_req] * kPageTokens : bt.n_partitions[i_req];
   const int k = min(c.topk, n);
   const int S = bt.slots[i_req];
+  // keys that do not fit in shared memory are re-read from the scores (L2 resident: the
+  // scoring CTAs have just written them); the launcher avoids that for large sets
+  const bool cached = n <= keys_cap;
 
-  const FastLayout L = fast_layout(c, dyn, token ? 0 : n, S);
+  const FastLayout L = fast_layout(c, dyn, keys_cap, S);
   uint32_t *s_keys = L.s_keys;
   int32_t *s_parts = L.s_parts;
   int32_t *s_sel = token ? L.s_host : L.s_parts;     // chosen candidates; tokens are folded into pages below
@@ -679,9 +680,9 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   fast_prefetch_dirs<T>(c, L, set, S);
 
   const float *scores = c.scores + (size_t)b * c.max_cand;
-  if (!token)
+  if (cached)
     for (int i = tid; i < n; i += T) s_keys[i] = order_key(__ldcg(scores + i));
-  auto key_at = [&](int i) { return token ? order_key(__ldcg(scores + i)) : s_keys[i]; };
+  auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(__ldcg(scores + i)); };
   for (int i = tid; i < 512; i += T) (&sh.hist[0][0])[i] = 0;
   if (tid == 0) {
     sh.lhist[0] = 0u;                        // OR / AND of the keys (reused as the timestamp histogram later)
