@@ -234,6 +234,8 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.sel_count = a.take<int32_t>(B);
   d.ready = a.take<int32_t>(B);
   d.tail_ready = a.take<int32_t>(B);
+  d.ready1 = a.take<int32_t>(B);
+  d.n_miss = a.take<int32_t>(B);
   d.counters = a.take<Counters>(1);
   __nv_bfloat16 *sq = a.take<__nv_bfloat16>((size_t)cfg.max_requests * cfg.num_q_heads * kHeadDim);
   __nv_bfloat16 *so = a.take<__nv_bfloat16>((size_t)cfg.max_requests * cfg.num_q_heads * kHeadDim);
@@ -665,6 +667,8 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   fill(d.sel_count, 0, (size_t)g.max_batch_sets * 4);
   fill(d.ready, 0, (size_t)g.max_batch_sets * 4);
   fill(d.tail_ready, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.ready1, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.n_miss, 0, (size_t)g.max_batch_sets * 4);
   fill(d.state, 0, (size_t)g.n_sets * sizeof(SetState));
   fill(d.counters, 0, sizeof(Counters));
   fill(d.fetch_count, 0, 4);

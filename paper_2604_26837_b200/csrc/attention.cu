@@ -153,6 +153,24 @@ __device__ __forceinline__ void store_page(const uint8_t *spage_generic, uint8_t
   }
 }
 
+// A page that came over the host link goes to the HBM slot it was admitted to.  With an early
+// descriptor (open_idx >= 0) the slot is read from page_src once the set's second flag is up
+// (long since, as a rule: the page took microseconds to arrive); a bypassed page has none.
+__device__ __forceinline__ void fetched_page_to_slot(const DevCtx &c, const Batch &bt, int b, size_t pl,
+                                                     const uint8_t *spage_generic, int slot_page, int open_idx,
+                                                     bool slots_known, int lane) {
+  if (open_idx >= 0) {
+    int ok = 1;
+    if (!slots_known) {
+      if (lane == 0) ok = flag_wait(c, c.ready + b, bt.epoch);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+    }
+    slot_page = ok ? __ldcg(c.page_src + pl + open_idx) : -1;
+    if (slot_page >= c.n_gpu_pages) { if (lane == 0) dev_error(c, kErrBounds); slot_page = -1; }
+  }
+  if (slot_page >= 0) store_page(spage_generic, c.gpu_pages + (size_t)slot_page * kPageBytes, lane);
+}
+
 template <int G>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out) {
@@ -161,18 +179,32 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   __shared__ int sh_last;
   const int b = blockIdx.x, chunk = blockIdx.y;       // chunk-major launch order: chunk 0 of every set first
   pdl_launch_next();
+  const int first = chunk * kChunkPages;
+  bool slots_known = true;                 // false: the chunk holds early descriptors only
   if (c.ready) {
-    // start as soon as this set's page list and tail page are complete (see flag_wait)
-    __shared__ int sh_ok;
-    if (threadIdx.x == 0) sh_ok = flag_wait(c, c.ready + b, bt.epoch) && flag_wait(c, c.tail_ready + b, bt.epoch);
+    // A set raises two flags.  The first says that its missed pages are listed (the leading
+    // n_miss descriptors, slot still open): a chunk made of those alone starts at once, so
+    // the pages cross the host link while the cache manager is still freeing slots for them.
+    // Every other chunk waits for the second flag (complete list) and for the tail page.
+    __shared__ int sh_ok, sh_np, sh_nm;
+    if (threadIdx.x == 0) {
+      int ok = flag_wait(c, c.ready1 + b, bt.epoch);
+      int np_ = 0, nm_ = 0;
+      if (ok) {
+        np_ = c.n_pages[b]; nm_ = c.n_miss[b];
+        if (first < np_ && min(np_, first + kChunkPages) > nm_)
+          ok = flag_wait(c, c.ready + b, bt.epoch) && flag_wait(c, c.tail_ready + b, bt.epoch);
+      }
+      sh_ok = ok; sh_np = np_; sh_nm = nm_;
+    }
     __syncthreads();
     if (!sh_ok) return;
+    slots_known = first >= sh_np || min(sh_np, first + kChunkPages) > sh_nm;
   } else {
     pdl_wait_prev();
   }
   if (chunk == 0) dbg_ta(b, 10);
   const int np = c.n_pages[b];
-  const int first = chunk * kChunkPages;
   if (first >= np) return;
   const int last = min(np, first + kChunkPages);
   const int i_req = b / c.Hkv, head = b % c.Hkv;
@@ -182,12 +214,14 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   // the warp's two pages; the one that has to cross the host link is waited for last
   int pg[2] = {first + warp, first + warp + kAttnWarps};
   int n_mine = (pg[0] < last) + (pg[1] < last);
-  int src[2] = {0, 0}, fill[2] = {-1, -1};
+  int src[2] = {0, 0}, fill[2] = {-1, -1}, open_idx[2] = {-1, -1};
   uint32_t mask[2] = {0, 0};
   for (int i = 0; i < n_mine; ++i) {
     if (c.page_desc) {                      // work-ordered descriptors written by the cache manager
       const int4 dsc = c.page_desc[pl + pg[i]];
       src[i] = dsc.x; fill[i] = dsc.y; mask[i] = (uint32_t)dsc.z;
+      const bool open = dsc.x == -3;        // early descriptor: page_src[dsc.w] names the slot later
+      if (open) { open_idx[i] = dsc.w; src[i] = 0; }
       if (fill[i] == -2) {
         // Retrieve step 3 for a missed page: Partition Offset -> CPU page table, both in pinned
         // host memory (two dependent reads over the host link, all lanes read the same words)
@@ -196,20 +230,22 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
         const int32_t *hp = off ? cpt_lookup(c, set, *off + c.page_pidx[pl + dsc.w]) : nullptr;
         const int host_page = hp ? *hp : -1;
         if (host_page < 0) { src[i] = -1; fill[i] = c.n_host_pages; }       // fails the range check below
-        else if (src[i] >= 0) fill[i] = host_page;                          // admitted: fetch into slot src
+        else if (open || src[i] >= 0) fill[i] = host_page;                  // fetched (admitted, or not yet known)
         else { src[i] = ~host_page; fill[i] = -1; }                         // bypassed: attend from host
       }
+      if (open && fill[i] < 0) { src[i] = -1; fill[i] = c.n_host_pages; }   // an early descriptor always names a host page
     } else {                                // plain lists, attended in the order given
       src[i] = c.page_src[pl + pg[i]];
       mask[i] = c.page_mask[pl + pg[i]];
     }
     // a descriptor that points outside the pools is dropped (and reported), never followed
     const bool ok = (src[i] >= 0 ? src[i] < c.n_gpu_pages : ~src[i] < c.n_host_pages) && fill[i] < c.n_host_pages;
-    if (!ok) { if (lane == 0) dev_error(c, kErrBounds); src[i] = 0; fill[i] = -1; mask[i] = 0; }
+    if (!ok) { if (lane == 0) dev_error(c, kErrBounds); src[i] = 0; fill[i] = -1; mask[i] = 0; open_idx[i] = -1; }
   }
   if (n_mine == 2 && (fill[0] >= 0 || src[0] < 0) && !(fill[1] >= 0 || src[1] < 0)) {
     int t = src[0]; src[0] = src[1]; src[1] = t;
     t = fill[0]; fill[0] = fill[1]; fill[1] = t;
+    t = open_idx[0]; open_idx[0] = open_idx[1]; open_idx[1] = t;
     uint32_t u = mask[0]; mask[0] = mask[1]; mask[1] = u;
   }
   if (chunk == 0) dbg_ta(b, 11);
@@ -245,14 +281,14 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
   if (chunk == 0) dbg_ta(b, 12);
   if (n_mine >= 1) {
     attend_page(smem_u32(spage[0]), qa, mask[0], scale2, acc, lane);
-    if (fill[0] >= 0) store_page(spage[0], c.gpu_pages + (size_t)src[0] * kPageBytes, lane);
+    if (fill[0] >= 0) fetched_page_to_slot(c, bt, b, pl, spage[0], src[0], open_idx[0], slots_known, lane);
   }
   cp_async_wait<0>();
   __syncwarp();
   if (chunk == 0) dbg_ta(b, 13);
   if (n_mine >= 2) {
     attend_page(smem_u32(spage[1]), qa, mask[1], scale2, acc, lane);
-    if (fill[1] >= 0) store_page(spage[1], c.gpu_pages + (size_t)src[1] * kPageBytes, lane);
+    if (fill[1] >= 0) fetched_page_to_slot(c, bt, b, pl, spage[1], src[1], open_idx[1], slots_known, lane);
   }
 
   // row sums live in the 4 lanes of a quad
@@ -465,6 +501,8 @@ extern "C" int spin_paged_attention_static(const void *q, const void *page_pool,
   c.page_desc = nullptr;                                    // the lists are attended in the order given
   c.ready = nullptr;                                        // plain stream order: no per-set flags
   c.tail_ready = nullptr;
+  c.ready1 = nullptr;
+  c.n_miss = nullptr;
   c.att_count = reinterpret_cast<int32_t *>(g_static_partials_addr[dev]);
   c.att_part = g_static_partials_addr[dev] + counter_floats;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);

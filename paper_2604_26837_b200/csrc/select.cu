@@ -90,8 +90,9 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
     return;
   }
   if (blockIdx.x == 0) dbg_ts(b, 0);
-  const SetState st = c.state[set];
-  const int n_cand = c.kind == kKindToken ? st.n_partitions * kPageTokens : st.n_partitions;
+  // the host's count: the in-grid append never completes a page, so it equals the set's state
+  const int n_partitions = bt.n_partitions[i_req];
+  const int n_cand = c.kind == kKindToken ? n_partitions * kPageTokens : n_partitions;
   const int seg_entries = 1 << c.sum_shift;
   const int e0 = blockIdx.x * seg_entries;
   // the CTAs that count towards the set's arrival counter: one per non-empty segment, and
@@ -177,7 +178,7 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
     select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, keys_cap, shm.fast);
     return;
   }
-  topk_stage<kScoreThreads, false>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, shm.staged.t);
+  topk_stage<kScoreThreads, false>(c, b, n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, shm.staged.t);
   cache_stage<kScoreThreads>(c, b, set, __ldcg(c.n_parts + b), bt.tail_pages[i_req], bt.tail_len[i_req],
                              bt.epoch, reinterpret_cast<int32_t *>(dyn_smem), shm.staged.c);
 }
@@ -266,6 +267,6 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
 #ifdef SPIN_TIMING
 extern "C" __attribute__((visibility("default"))) int spin_debug_timestamps(unsigned long long *out) {
   cudaDeviceSynchronize();
-  return (int)cudaMemcpyFromSymbol(out, spin::g_dbg_ts, sizeof(unsigned long long) * 256 * 16);
+  return (int)cudaMemcpyFromSymbol(out, spin::g_dbg_ts, sizeof(unsigned long long) * 256 * 32);
 }
 #endif

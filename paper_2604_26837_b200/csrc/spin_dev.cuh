@@ -104,6 +104,8 @@ struct DevCtx {
   int32_t *sel_count;           // [b] scoring CTAs of the set that have finished (zero between steps)
   int32_t *ready;               // [b] epoch of the last step whose page list is complete
   int32_t *tail_ready;          // [b] epoch of the last step whose appended rows are in the tail page
+  int32_t *ready1;              // [b] epoch of the last step whose missed pages are listed (before their slots are known)
+  int32_t *n_miss;              // [b] leading descriptors of the page list that may be followed once ready1 is set
   int32_t max_chunks;
   int32_t fetch_mode;           // 0: misses are fetched by the attention kernel; 1: by k_fetch
   Counters *counters;

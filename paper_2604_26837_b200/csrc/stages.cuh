@@ -559,6 +559,8 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
     atomicAdd(&k->miss_pages, (unsigned long long)miss_pages);
     atomicAdd(&k->evicted_pages, (unsigned long long)sh.evicted);
     atomicAdd(&k->bypass_pages, (unsigned long long)sh.bypass_pages);
+    c.n_miss[b] = 0;                             // no early list on this path: both flags go up together
+    flag_publish(c.ready1 + b, epoch);
     flag_publish(c.ready + b, epoch);            // attention may start on this set
   }
 }
@@ -574,7 +576,7 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
 constexpr int kFastSlots = 1024;
 
 #ifdef SPIN_TIMING
-__device__ unsigned long long g_dbg_ts[256][16];
+__device__ unsigned long long g_dbg_ts[256][32];
 __device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; } }
 #else
 __device__ __forceinline__ void dbg_ts(int, int) {}
@@ -713,6 +715,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
     k_and = __reduce_and_sync(0xffffffffu, k_and);
     if ((tid & 31) == 0) { atomicOr(&sh.lhist[0], k_or); atomicAnd(&sh.lhist[1], k_and); }
     __syncthreads();
+    dbg_ts(b, 16);
     const uint32_t differ = sh.lhist[0] ^ sh.lhist[1];           // bits on which some keys differ
     uint32_t prefix = 0, mask = 0, remaining = k;
     int first_shift = 24;
@@ -760,6 +763,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
       mask |= 255u << shift;
       // the buffer just searched is cleared by the next pass's idle warps (it is used again two passes on)
     }
+    dbg_ts(b, 17);
     const uint32_t thr = prefix, need_eq = remaining;
     // every thread owns a contiguous run of candidates: two block scans place all of them
     const int E = (n + T - 1) / T, lo = min(n, tid * E), hi = min(n, lo + E);
@@ -863,14 +867,17 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     run_all += tot_a;
     run_miss += tot_m;
   }
+  dbg_ts(b, 18);
   if (tid == 0) s_pageoff[np] = run_all;
   int total_pages = (int)run_all;
-  const int demand = (int)run_miss;
+  int demand = (int)run_miss;
   if (total_pages > c.max_pages) {
+    // more pages than the list holds (reported): whole partitions are dropped from the end
     if (tid == 0) dev_error(c, kErrPageList);
     __syncthreads();
     while (np > 0 && s_pageoff[np] > c.max_pages) --np;
     total_pages = s_pageoff[np];
+    demand = np < np_sel ? s_missbefore[np] : demand;
   }
   for (int i = tid; i < (S + 31) / 32; i += T) s_hit[i] = 0;
   for (int i = tid; i < kMaxBuckets + 2; i += T) sh.lhist[i] = 0;
@@ -878,26 +885,48 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   __syncthreads();
 
   dbg_ts(b, 4);
-  // Retrieve step 3 started early (pinned host tables, two dependent reads over the host link)
-  int early_off[2] = {-1, -1}, early_i[2] = {0, 0};
-#pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    const int mi = tid + j * T;
-    if (resolve_in_manager(c) && mi < demand && mi < c.max_pages && np > 0) {
-      const int r = owner_of(s_missbefore, np, mi);
-      early_i[j] = mi - s_missbefore[r];
-      const int32_t *off = off_lookup(c, set, s_parts[r]);
-      if (off) early_off[j] = *off;
-    }
-  }
-
-  // ---- step 2: one pass over the page table copy: promote, demote, histogram ----------------
+  // ---- the early list: Retrieve step 3 for the missed pages, then they may start to move -----
+  // Which pages are missing and where they live in host memory is known before a single slot
+  // has been freed.  With the fetch fused into attention those descriptors (slot still open,
+  // x = -3) are published now under the set's first flag: the attention CTAs that own them
+  // put the pages on the host link while this CTA goes on to promote, evict and admit, and
+  // pick the slot up from page_src once the second flag is set.
   const size_t pl = (size_t)b * (c.max_pages + c.tail_cap);
   int32_t *page_src = c.page_src + pl, *page_slot = c.page_slot + pl;
   int32_t *page_part = c.page_part + pl, *page_pidx = c.page_pidx + pl;
   uint32_t *page_mask = c.page_mask + pl;
   int32_t *page_fill = c.page_fill + pl;
   int4 *page_desc = c.page_desc + pl;
+  const bool early = c.fetch_mode == 0;
+  for (int mi = tid; mi < demand; mi += T) {
+    const int r = owner_of(s_missbefore, np, mi);
+    const int i = mi - s_missbefore[r], p = s_parts[r];
+    int host_page = -2;                     // -2: the fetching warp resolves it (host tables only)
+    if (resolve_in_manager(c)) {
+      const int32_t *off = off_lookup(c, set, p);
+      const int32_t *hp = off ? cpt_lookup(c, set, *off + i) : nullptr;
+      host_page = hp ? *hp : -1;
+      if (host_page < -1) host_page = -1;
+    }
+    s_host[mi] = host_page;
+    if (early) {
+      const int idx = s_pageoff[r] + i;
+      const int valid = min(kPageTokens, s_tokens[r] - i * kPageTokens);
+      const uint32_t pmask = c.kind == kKindToken ? c.part_mask[(size_t)b * c.max_parts + r] : ((1u << valid) - 1u);
+      page_part[idx] = p;
+      page_pidx[idx] = i;
+      page_desc[mi] = host_page == -1 ? make_int4(0, -1, 0, idx) : make_int4(-3, host_page, (int)pmask, idx);
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    c.n_pages[b] = total_pages + tail_pages;
+    c.n_miss[b] = early ? demand : 0;
+    flag_publish(c.ready1 + b, bt.epoch);
+  }
+
+  dbg_ts(b, 19);
+  // ---- step 2: one pass over the page table copy: promote, demote, histogram ----------------
   for (int s_ = tid; s_ < S; s_ += T) {
     int4 e = s_gpt[s_];
     if (c.trace) {
@@ -921,14 +950,6 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   __syncthreads();
 
   dbg_ts(b, 5);
-  int early_host[2] = {-1, -1};
-#pragma unroll
-  for (int j = 0; j < 2; ++j)
-    if (early_off[j] >= 0) {
-      const int32_t *hp = cpt_lookup(c, set, early_off[j] + early_i[j]);
-      if (hp) early_host[j] = *hp;
-    }
-
   // ---- step 3: threshold, eviction, free slots in ascending order (one scan) ----------------
   if (tid == 0) {
     int x = -2;
@@ -944,6 +965,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   }
   __syncthreads();
   const int x = sh.x;
+  dbg_ts(b, 20);
   uint32_t run_free = 0;
   if (demand > 0) {
     const int E = (S + T - 1) / T, lo = min(S, tid * E), hi = min(S, lo + E);
@@ -969,8 +991,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
       if (s_gpt[s_].x < 0) { if (pos < (uint32_t)c.max_pages) s_free[pos] = s_; ++pos; }
     run_free = tot;
   }
-#pragma unroll
-  for (int j = 0; j < 2; ++j) { const int mi = tid + j * T; if (mi < c.max_pages) s_host[mi] = early_host[j]; }
+  dbg_ts(b, 21);
   __syncthreads();
 
   dbg_ts(b, 6);
@@ -991,6 +1012,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   if (tid == 0) sh.qbase = (sh.demand > 0 && c.fetch_mode != 0) ? atomicAdd(c.fetch_count, sh.demand) : 0;
   __syncthreads();
   const int qbase = sh.qbase;
+  dbg_ts(b, 22);
   for (int r = tid; r < np; r += T) {
     c.part_state[(size_t)b * c.max_parts + r] = s_state[r];
     if (s_state[r] == kAdmit) {
@@ -999,6 +1021,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     }
   }
   int my_admit = 0, my_bypass = 0;
+  dbg_ts(b, 23);
   for (int idx = tid; idx < total_pages; idx += T) {
     const int r = owner_of(s_pageoff, np, idx);
     const int i = idx - s_pageoff[r], p = s_parts[r], state = s_state[r];
@@ -1011,43 +1034,38 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     const int pos = state == kHit ? demand + (s_pageoff[r] - s_missbefore[r]) + i : s_missbefore[r] + i;
     if (state == kHit) { page_desc[pos] = make_int4(page_src[idx], -1, (int)pmask, idx); continue; }
     const int mi = s_missbefore[r] + i;
-    // Retrieve step 3 (Partition Offset -> CPU page table, both in pinned host memory): with
-    // the fetch fused into attention, the warp that brings the page in looks its CPU page id up
-    // itself (fill = -2), so this set's page list does not wait on the host link; with the
-    // stand-alone copy kernel the ids are resolved here
-    int host_page = -2;
-    if (resolve_in_manager(c)) {
-      host_page = mi < 2 * T && mi < c.max_pages ? s_host[mi] : -1;
-      if (host_page < 0) {
-        const int32_t *off = off_lookup(c, set, p);
-        const int32_t *hp = off ? cpt_lookup(c, set, *off + i) : nullptr;
-        if (hp) host_page = *hp;
-      }
-      if (host_page < 0) { dev_error(c, kErrBounds); page_src[idx] = 0; page_mask[idx] = 0; page_desc[pos] = make_int4(0, -1, 0, idx); continue; }
+    // the CPU page id found for the early list (-2: left to the fetching warp, which then reads
+    // the two pinned host tables itself, so that no page list waits on the host link)
+    const int host_page = s_host[mi];
+    if (host_page == -1) {
+      dev_error(c, kErrBounds);
+      page_src[idx] = 0; page_mask[idx] = 0;
+      if (!early) page_desc[pos] = make_int4(0, -1, 0, idx);
+      continue;
     }
     if (state == kAdmit) {
       const int slot = s_free[s_missoff[r] + i];
       const int phys = s_gpt[slot].y;
       s_gpt[slot] = make_int4(p, phys, i, top);
-      page_src[idx] = phys;
+      page_src[idx] = phys;                  // what the owner of an early descriptor comes back for
       page_slot[idx] = slot;
-      int fill = -1;
-      if (c.fetch_mode == 0) { fill = host_page; page_fill[idx] = host_page; }    // host_page is -2 if unresolved
+      if (c.fetch_mode == 0) page_fill[idx] = host_page;
       else {
         const int qi = qbase + s_missoff[r] + i;
         if (qi < c.fetch_cap) c.fetch_queue[qi] = FetchItem{host_page, phys};
         else dev_error(c, kErrBounds);
+        page_desc[pos] = make_int4(phys, -1, (int)pmask, idx);
       }
-      page_desc[pos] = make_int4(phys, fill, (int)pmask, idx);
       ++my_admit;
     } else {
-      // bypassed: attended from host memory, never cached (x = -1: no slot)
+      // bypassed: attended from host memory, never cached (no slot)
       page_src[idx] = host_page == -2 ? -1 : ~host_page;
       page_slot[idx] = -1;
-      page_desc[pos] = host_page == -2 ? make_int4(-1, -2, (int)pmask, idx) : make_int4(~host_page, -1, (int)pmask, idx);
+      if (!early) page_desc[pos] = make_int4(~host_page, -1, (int)pmask, idx);
       ++my_bypass;
     }
   }
+  dbg_ts(b, 24);
   if (my_admit) atomicAdd(&sh.admit_pages, my_admit);
   if (my_bypass) atomicAdd(&sh.bypass_pages, my_bypass);
   for (int j = tid; j < tail_pages; j += T) {
