@@ -108,7 +108,7 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
   static size_t configured = 0;
   int max_slots_batch = 0;
   for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
+  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages);
   const int fast = (max_slots_batch <= kFastSlots && fs <= 96 * 1024) ? 1 : 0;
   const size_t smem = fast ? fs : cache_smem_bytes(c);
   if (smem > configured) {

@@ -231,7 +231,7 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
     // of a set in shared memory
     int max_slots_batch = 0;
     for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.max_parts, c.max_pages);
+    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages);
     if (max_slots_batch <= kFastSlots && max_cand <= 16384 && fs <= 100 * 1024) {
       fuse = 2;
       keys_cap = max_cand;

@@ -590,12 +590,12 @@ struct FastShared {
   int x, demand, evicted, qbase, admit_pages, bypass_pages;
 };
 
-__host__ __device__ inline size_t fast_smem_bytes(int n_keys, int slots, int dir_part, int dir_slot,
+__host__ __device__ inline size_t fast_smem_bytes(int n_keys, int slots, int dir_part, int dir_slot, int dir_page,
                                                   int max_parts, int max_pages) {
   size_t b = (size_t)((n_keys + 3) / 4 * 4) * 4;                 // keys
   b += (size_t)slots * 16;                                       // GPU page table copy
-  b += (size_t)((dir_part + dir_slot + 3) / 4 * 4) * 4;          // directories
-  b += (size_t)(6 * max_parts + 4 + 2 * max_pages) * 4;          // cache manager tables, free list, host ids
+  b += (size_t)((2 * dir_part + dir_slot + dir_page + 3) / 4 * 4) * 4;   // the four directories
+  b += (size_t)(7 * max_parts + 4 + 2 * max_pages) * 4;          // cache manager tables, free list, host ids
   b += (size_t)((slots + 31) / 32 + 4) * 4;                      // hit bitmask
   return b + 64;
 }
@@ -613,7 +613,7 @@ __device__ __forceinline__ void cp_async_commit_wait_all() {
 struct FastLayout {
   uint32_t *s_keys;
   int4 *s_gpt;
-  int32_t *s_mdir, *s_gdir, *s_parts, *s_tokens, *s_pageoff, *s_missoff, *s_missbefore, *s_state, *s_free, *s_host;
+  int32_t *s_mdir, *s_gdir, *s_odir, *s_cdir, *s_parts, *s_tokens, *s_off, *s_pageoff, *s_missoff, *s_missbefore, *s_state, *s_free, *s_host;
   uint32_t *s_hit;
 };
 
@@ -623,9 +623,12 @@ __device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn,
   L.s_gpt = reinterpret_cast<int4 *>(L.s_keys + (n_keys + 3) / 4 * 4);
   L.s_mdir = reinterpret_cast<int32_t *>(L.s_gpt + S);
   L.s_gdir = L.s_mdir + c.dir_part;
-  L.s_parts = L.s_mdir + (c.dir_part + c.dir_slot + 3) / 4 * 4;
+  L.s_odir = L.s_gdir + c.dir_slot;
+  L.s_cdir = L.s_odir + c.dir_part;
+  L.s_parts = L.s_mdir + (2 * c.dir_part + c.dir_slot + c.dir_page + 3) / 4 * 4;
   L.s_tokens = L.s_parts + c.max_parts;
-  L.s_pageoff = L.s_tokens + c.max_parts;        // [max_parts + 1]
+  L.s_off = L.s_tokens + c.max_parts;            // Partition Offset entries of the selected partitions
+  L.s_pageoff = L.s_off + c.max_parts;           // [max_parts + 1]
   L.s_missoff = L.s_pageoff + c.max_parts + 1;
   L.s_missbefore = L.s_missoff + c.max_parts;
   L.s_state = L.s_missbefore + c.max_parts;
@@ -635,13 +638,18 @@ __device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn,
   return L;
 }
 
-// Directories of the Meta-partition table and of the GPU page table -> shared memory (one
+// Directories of the Meta-partition table and of the GPU page table (and, when this CTA
+// resolves CPU page ids, of the Partition Offset and CPU page tables) -> shared memory (one
 // cp.async group; the caller waits for it and barriers before fast_prefetch_gpt).
 template <int T>
 __device__ __forceinline__ void fast_prefetch_dirs(const DevCtx &c, const FastLayout &L, int set, int S) {
   const int tid = threadIdx.x, n_gdir = (S + (1 << c.seg_shift) - 1) >> c.seg_shift;
   for (int i = tid; i < c.dir_part; i += T) cp_async4(L.s_mdir + i, c.dir_meta + (size_t)set * c.dir_part + i);
   for (int i = tid; i < n_gdir; i += T) cp_async4(L.s_gdir + i, c.dir_gpt + (size_t)set * c.dir_slot + i);
+  if (resolve_in_manager(c)) {
+    for (int i = tid; i < c.dir_part; i += T) cp_async4(L.s_odir + i, c.dir_off + (size_t)set * c.dir_part + i);
+    for (int i = tid; i < c.dir_page; i += T) cp_async4(L.s_cdir + i, c.dir_cpt + (size_t)set * c.dir_page + i);
+  }
   asm volatile("cp.async.commit_group;\n" ::: "memory");
 }
 // The set's whole GPU page table -> shared memory (one cp.async group).
@@ -834,7 +842,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   int4 *s_gpt = L.s_gpt;
   int32_t *s_mdir = L.s_mdir, *s_gdir = L.s_gdir, *s_parts = L.s_parts, *s_tokens = L.s_tokens;
   int32_t *s_pageoff = L.s_pageoff, *s_missoff = L.s_missoff, *s_missbefore = L.s_missbefore;
-  int32_t *s_state = L.s_state, *s_free = L.s_free, *s_host = L.s_host;
+  int32_t *s_state = L.s_state, *s_free = L.s_free, *s_host = L.s_host, *s_off = L.s_off;
   uint32_t *s_hit = L.s_hit;
   if (tid == 0) { c.att_count[b] = 0; sh.evicted = 0; sh.admit_pages = 0; sh.bypass_pages = 0; }
   // ---- cache manager step 1: Meta-partition lookups, classification, page demand ------------
@@ -855,6 +863,11 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
       miss = res ? 0 : 1;
       s_tokens[r] = tokens;
       s_state[r] = res ? kHit : kAdmit;
+      if (miss && resolve_in_manager(c)) {
+        // Retrieve step 3, first half: where the partition's pages start in the CPU page table
+        const int oseg = L.s_odir[p >> c.seg_shift];
+        s_off[r] = oseg >= 0 ? (c.off_mirror ? c.off_mirror : c.off_pool)[((size_t)oseg << c.seg_shift) + (p & seg_mask)] : -1;
+      }
     }
     uint32_t tot_a, tot_m;
     const uint32_t ex_a = block_scan<T>(npg, sh.wsum, &tot_a);
@@ -903,9 +916,10 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     const int i = mi - s_missbefore[r], p = s_parts[r];
     int host_page = -2;                     // -2: the fetching warp resolves it (host tables only)
     if (resolve_in_manager(c)) {
-      const int32_t *off = off_lookup(c, set, p);
-      const int32_t *hp = off ? cpt_lookup(c, set, *off + i) : nullptr;
-      host_page = hp ? *hp : -1;
+      // second half: the CPU page table entry (directory in shared memory, one global read)
+      const int e = s_off[r] + i;
+      const int cseg = (s_off[r] >= 0 && (e >> c.seg_shift) < c.dir_page) ? L.s_cdir[e >> c.seg_shift] : -1;
+      host_page = cseg >= 0 ? (c.cpt_mirror ? c.cpt_mirror : c.cpt_pool)[((size_t)cseg << c.seg_shift) + (e & seg_mask)] : -1;
       if (host_page < -1) host_page = -1;
     }
     s_host[mi] = host_page;
