@@ -29,7 +29,7 @@ constexpr int kCacheThreads = 512;
 // fits, so the page table is staged in shared memory (cache_fast); else it is worked on in
 // global memory (cache_stage).
 __global__ void __launch_bounds__(kCacheThreads)
-k_cache(DevCtx c, Batch bt, int fast) {
+k_cache(DevCtx c, Batch bt, int fast, int tbl_cap) {
   extern __shared__ __align__(16) uint8_t dyn_smem[];
   __shared__ union { CacheShared staged; FastShared fast; } shm;
   const int b = blockIdx.x, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
@@ -43,13 +43,16 @@ k_cache(DevCtx c, Batch bt, int fast) {
     return;
   }
   const int S = bt.slots[i_req];
-  const FastLayout L = fast_layout(c, dyn_smem, 0, S);
+  const FastLayout L = fast_layout(c, dyn_smem, 0, S, tbl_cap);
   fast_prefetch_dirs<kCacheThreads>(c, L, set, S);
   const int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
   for (int r = tid; r < np; r += kCacheThreads) L.s_parts[r] = g_parts[r];
   asm volatile("cp.async.wait_group 0;\n" ::: "memory");
   __syncthreads();
   fast_prefetch_gpt<kCacheThreads>(c, L, S);
+  fast_prefetch_tables<kCacheThreads>(c, L, bt.n_partitions[i_req]);
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+  __syncthreads();
   cache_fast<kCacheThreads>(c, bt, b, i_req, set, L, np, shm.fast);
 }
 
@@ -108,14 +111,22 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
   static size_t configured = 0;
   int max_slots_batch = 0;
   for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages);
+  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, 0);
   const int fast = (max_slots_batch <= kFastSlots && fs <= 96 * 1024) ? 1 : 0;
-  const size_t smem = fast ? fs : cache_smem_bytes(c);
+  size_t smem = fast ? fs : cache_smem_bytes(c);
+  int tbl_cap = 0;
+  if (fast && c.kind != kKindCluster) {
+    // one CTA per set: the snapshot of the partition tables may take what shared memory is left
+    int max_parts_batch = 0;
+    for (int i = 0; i < b.n_req; ++i) max_parts_batch = b.n_partitions[i] > max_parts_batch ? b.n_partitions[i] : max_parts_batch;
+    const size_t ft = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, max_parts_batch);
+    if (max_parts_batch > 0 && ft <= 200 * 1024) { tbl_cap = max_parts_batch; smem = ft; }
+  }
   if (smem > configured) {
     cudaFuncSetAttribute(k_cache, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b, fast);
+  launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b, fast, tbl_cap);
   prof_mark(prof, st, kProfCache);
   return 1;
 }

@@ -73,7 +73,7 @@ __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, con
 template <int G, bool MINMAX>
 __global__ void __launch_bounds__(kScoreThreads, 3)
 k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
-        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap) {   // fuse: 0 none, 1 staged, 2 fast
+        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap, int tbl_cap) {   // fuse: 0 none, 1 staged, 2 fast
   extern __shared__ __align__(16) uint8_t dyn_smem[];      // used by the fused continuation only
   const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
@@ -175,7 +175,7 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
   __threadfence();
   if (threadIdx.x == 0) c.sel_count[b] = 0;                 // ready for the next step
   if (fuse == 2) {
-    select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, keys_cap, shm.fast);
+    select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, keys_cap, tbl_cap, shm.fast);
     return;
   }
   topk_stage<kScoreThreads, false>(c, b, n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, shm.staged.t);
@@ -200,15 +200,15 @@ k_topk(DevCtx c, Batch bt, int keys_cap) {
 
 template <int G>
 void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
-                    const __nv_bfloat16 *v_new, dim3 grid, size_t smem, int fuse, int keys_cap, cudaStream_t st) {
+                    const __nv_bfloat16 *v_new, dim3 grid, size_t smem, int fuse, int keys_cap, int tbl_cap, cudaStream_t st) {
   static size_t configured = 0;
   if (smem > configured) {
     cudaFuncSetAttribute(k_score<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     cudaFuncSetAttribute(k_score<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap);
-  else launch_pdl(k_score<G, false>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap);
+  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap, tbl_cap);
+  else launch_pdl(k_score<G, false>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap, tbl_cap);
 }
 
 }  // namespace
@@ -223,7 +223,7 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
   // fused: one CTA can hold a set's keys and the cache manager's tables in shared memory
   const size_t cache_smem = cache_stage_smem_bytes(c.max_parts, c.max_pages, c.max_slots);
   int fuse = (max_cand <= 16384 && cache_smem <= 96 * 1024) ? 1 : 0;
-  int keys_cap = fuse ? max_cand : 0;
+  int keys_cap = fuse ? max_cand : 0, tbl_cap = 0;
   size_t smem = 0;
   if (fuse) smem = cache_smem > (size_t)keys_cap * 4 ? cache_smem : (size_t)keys_cap * 4;
   {
@@ -231,19 +231,25 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
     // of a set in shared memory
     int max_slots_batch = 0;
     for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages);
+    const size_t fs = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, 0);
     if (max_slots_batch <= kFastSlots && max_cand <= 16384 && fs <= 100 * 1024) {
       fuse = 2;
       keys_cap = max_cand;
       smem = fs;
+      // page granularity (partition j = page j of the set): if the set's partition tables fit
+      // beside the rest without costing a resident CTA, the continuation snapshots them
+      int max_parts_batch = 0;
+      for (int i = 0; i < b.n_req; ++i) max_parts_batch = b.n_partitions[i] > max_parts_batch ? b.n_partitions[i] : max_parts_batch;
+      const size_t ft = fast_smem_bytes(max_cand, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, max_parts_batch);
+      if (c.kind != kKindCluster && max_parts_batch > 0 && ft <= 72 * 1024) { tbl_cap = max_parts_batch; smem = ft; }
     }
   }
   if (smem < 64 * 1024) smem = 64 * 1024;         // the scoring CTAs' staging area: one summary segment
   switch (c.G) {
-    case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
-    case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
-    case 4: launch_score_g<4>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
-    default: launch_score_g<8>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, st); break;
+    case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
+    case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
+    case 4: launch_score_g<4>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
+    default: launch_score_g<8>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
   }
   prof_mark(prof, st, kProfScore);
   if (fuse) return 1;

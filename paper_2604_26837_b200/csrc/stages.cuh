@@ -53,6 +53,30 @@ __device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t *wsum, uint3
   return res;
 }
 
+// The same with a single barrier: every thread adds up the warp totals itself.  wsum: T/32
+// words that no thread still reads from an earlier call (callers alternate two buffers).
+template <int T>
+__device__ __forceinline__ uint32_t block_scan1(uint32_t v, uint32_t *wsum, uint32_t *total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[w] = inc;
+  __syncthreads();
+  uint32_t base = 0, tot = 0;
+#pragma unroll
+  for (int j = 0; j < T / 32; ++j) {
+    const uint32_t x = wsum[j];
+    base += j < w ? x : 0u;
+    tot += x;
+  }
+  *total = tot;
+  return base + inc - v;
+}
+
 // index of `p` in the ascending array a[0..n), or -1
 __device__ __forceinline__ int find_sorted(const int32_t *a, int n, int p) {
   int lo = 0, hi = n;
@@ -582,8 +606,13 @@ __device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) 
 __device__ __forceinline__ void dbg_ts(int, int) {}
 #endif
 
+constexpr int kFastDigitBits = 11, kFastBins = 1 << kFastDigitBits;
+constexpr int kFastSmall = 32;               // a threshold bin this small is finished by one warp
+
 struct FastShared {
-  uint32_t hist[2][256];
+  uint32_t wor[32], wand[32];  // per-warp OR / AND of the keys
+  uint32_t cand[kFastSmall];   // keys of the threshold bin
+  uint32_t ncand, bin_count;
   uint32_t wsum[33];
   uint32_t lhist[kMaxBuckets + 2];
   uint32_t prefix, remaining;
@@ -591,12 +620,14 @@ struct FastShared {
 };
 
 __host__ __device__ inline size_t fast_smem_bytes(int n_keys, int slots, int dir_part, int dir_slot, int dir_page,
-                                                  int max_parts, int max_pages) {
+                                                  int max_parts, int max_pages, int tbl_cap) {
   size_t b = (size_t)((n_keys + 3) / 4 * 4) * 4;                 // keys
   b += (size_t)slots * 16;                                       // GPU page table copy
   b += (size_t)((2 * dir_part + dir_slot + dir_page + 3) / 4 * 4) * 4;   // the four directories
   b += (size_t)(7 * max_parts + 4 + 2 * max_pages) * 4;          // cache manager tables, free list, host ids
   b += (size_t)((slots + 31) / 32 + 4) * 4;                      // hit bitmask
+  b += (size_t)((tbl_cap + 3) / 4 * 4) * 16 + 16;                // snapshot of the set's three partition tables
+  b += (size_t)2048 * 4;                                         // digit histogram of the select
   return b + 64;
 }
 
@@ -615,9 +646,16 @@ struct FastLayout {
   int4 *s_gpt;
   int32_t *s_mdir, *s_gdir, *s_odir, *s_cdir, *s_parts, *s_tokens, *s_off, *s_pageoff, *s_missoff, *s_missbefore, *s_state, *s_free, *s_host;
   uint32_t *s_hit;
+  // Optional snapshot of the set's Meta-partition, Partition Offset and CPU page tables (entries
+  // [0, tbl_cap), 0 = none): taken while the radix select runs, so that classifying the
+  // selection and finding the missed pages' host ids costs no further trip to memory.
+  int2 *s_meta;
+  int32_t *s_offt, *s_cptt;
+  int tbl_cap;
+  uint32_t *s_hist;            // [kFastBins]
 };
 
-__device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn, int n_keys, int S) {
+__device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn, int n_keys, int S, int tbl_cap) {
   FastLayout L;
   L.s_keys = reinterpret_cast<uint32_t *>(dyn);
   L.s_gpt = reinterpret_cast<int4 *>(L.s_keys + (n_keys + 3) / 4 * 4);
@@ -635,7 +673,18 @@ __device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn,
   L.s_free = L.s_state + c.max_parts + 3;        // [max_pages]
   L.s_host = L.s_free + c.max_pages;             // [max_pages] CPU page ids of missed pages
   L.s_hit = reinterpret_cast<uint32_t *>(L.s_host + c.max_pages);
+  const uintptr_t t = (reinterpret_cast<uintptr_t>(L.s_hit + (S + 31) / 32 + 4) + 15) & ~(uintptr_t)15;
+  const int tc = (tbl_cap + 3) / 4 * 4;
+  L.tbl_cap = tbl_cap;
+  L.s_meta = reinterpret_cast<int2 *>(t);
+  L.s_offt = reinterpret_cast<int32_t *>(L.s_meta + tc);
+  L.s_cptt = L.s_offt + tc;
+  L.s_hist = reinterpret_cast<uint32_t *>(L.s_cptt + tc);
   return L;
+}
+// true when the snapshot also holds the two host-side tables (read from their HBM copies)
+__device__ __forceinline__ bool fast_snap_host(const DevCtx &c, const FastLayout &L) {
+  return L.tbl_cap > 0 && resolve_in_manager(c) && c.off_mirror && c.cpt_mirror;
 }
 
 // Directories of the Meta-partition table and of the GPU page table (and, when this CTA
@@ -644,10 +693,14 @@ __device__ __forceinline__ FastLayout fast_layout(const DevCtx &c, uint8_t *dyn,
 template <int T>
 __device__ __forceinline__ void fast_prefetch_dirs(const DevCtx &c, const FastLayout &L, int set, int S) {
   const int tid = threadIdx.x, n_gdir = (S + (1 << c.seg_shift) - 1) >> c.seg_shift;
+#pragma unroll 1
   for (int i = tid; i < c.dir_part; i += T) cp_async4(L.s_mdir + i, c.dir_meta + (size_t)set * c.dir_part + i);
+#pragma unroll 1
   for (int i = tid; i < n_gdir; i += T) cp_async4(L.s_gdir + i, c.dir_gpt + (size_t)set * c.dir_slot + i);
   if (resolve_in_manager(c)) {
+#pragma unroll 1
     for (int i = tid; i < c.dir_part; i += T) cp_async4(L.s_odir + i, c.dir_off + (size_t)set * c.dir_part + i);
+#pragma unroll 1
     for (int i = tid; i < c.dir_page; i += T) cp_async4(L.s_cdir + i, c.dir_cpt + (size_t)set * c.dir_page + i);
   }
   asm volatile("cp.async.commit_group;\n" ::: "memory");
@@ -656,11 +709,36 @@ __device__ __forceinline__ void fast_prefetch_dirs(const DevCtx &c, const FastLa
 template <int T>
 __device__ __forceinline__ void fast_prefetch_gpt(const DevCtx &c, const FastLayout &L, int S) {
   const int tid = threadIdx.x, seg_mask = (1 << c.seg_shift) - 1;
+#pragma unroll 1
   for (int s_ = tid; s_ < S; s_ += T) {
     const int seg = L.s_gdir[s_ >> c.seg_shift];
     if (seg >= 0) cp_async16_ca(L.s_gpt + s_, c.gpt_pool + ((size_t)seg << c.seg_shift) + (s_ & seg_mask));
     else { dev_error(c, kErrBounds); L.s_gpt[s_] = make_int4(-1, 0, 0, -1); }
   }
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+}
+
+// The first min(n_part, tbl_cap) entries of the set's partition tables -> shared memory (one
+// cp.async group; needs the directories in shared memory).
+template <int T>
+__device__ __forceinline__ void fast_prefetch_tables(const DevCtx &c, const FastLayout &L, int n_part) {
+  const int tid = threadIdx.x, seg_mask = (1 << c.seg_shift) - 1, n = min(n_part, L.tbl_cap);
+#pragma unroll 1
+  for (int e = 2 * tid; e < n; e += 2 * T) {
+    const int seg = L.s_mdir[e >> c.seg_shift];
+    if (seg >= 0) cp_async16_ca(L.s_meta + e, c.meta_pool + ((size_t)seg << c.seg_shift) + (e & seg_mask));
+    else { L.s_meta[e] = make_int2(0, 1); L.s_meta[e + 1] = make_int2(0, 1); }
+  }
+  if (fast_snap_host(c, L))
+#pragma unroll 1
+    for (int e = 4 * tid; e < n; e += 4 * T) {
+      const int oseg = L.s_odir[e >> c.seg_shift];
+      const int cseg = (e >> c.seg_shift) < c.dir_page ? L.s_cdir[e >> c.seg_shift] : -1;
+      if (oseg >= 0) cp_async16_ca(L.s_offt + e, c.off_mirror + ((size_t)oseg << c.seg_shift) + (e & seg_mask));
+      else for (int j = 0; j < 4; ++j) L.s_offt[e + j] = -1;
+      if (cseg >= 0) cp_async16_ca(L.s_cptt + e, c.cpt_mirror + ((size_t)cseg << c.seg_shift) + (e & seg_mask));
+      else for (int j = 0; j < 4; ++j) L.s_cptt[e + j] = -1;
+    }
   asm volatile("cp.async.commit_group;\n" ::: "memory");
 }
 
@@ -670,7 +748,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
 
 template <int T>
 __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
-                                            uint8_t *dyn, int keys_cap, FastShared &sh) {
+                                            uint8_t *dyn, int keys_cap, int tbl_cap, FastShared &sh) {
   const int tid = threadIdx.x;
   const bool token = c.kind == kKindToken;
   const int n = token ? bt.n_partitions[i_req] * kPageTokens : bt.n_partitions[i_req];
@@ -680,7 +758,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   // scoring CTAs have just written them); the launcher avoids that for large sets
   const bool cached = n <= keys_cap;
 
-  const FastLayout L = fast_layout(c, dyn, keys_cap, S);
+  const FastLayout L = fast_layout(c, dyn, keys_cap, S, tbl_cap);
   uint32_t *s_keys = L.s_keys;
   int32_t *s_parts = L.s_parts;
   int32_t *s_sel = token ? L.s_host : L.s_parts;     // chosen candidates; tokens are folded into pages below
@@ -690,13 +768,22 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   fast_prefetch_dirs<T>(c, L, set, S);
 
   const float *scores = c.scores + (size_t)b * c.max_cand;
-  if (cached)
-    for (int i = tid; i < n; i += T) s_keys[i] = order_key(__ldcg(scores + i));
   auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(__ldcg(scores + i)); };
-  for (int i = tid; i < 512; i += T) (&sh.hist[0][0])[i] = 0;
+  // keys -> shared memory, with the OR and AND of all keys taken on the way (see the select)
+  uint32_t k_or = 0, k_and = 0xffffffffu;
+#pragma unroll 8
+  for (int i = tid; i < n; i += T) {
+    const uint32_t key = order_key(__ldcg(scores + i));
+    if (cached) s_keys[i] = key;
+    k_or |= key; k_and &= key;
+  }
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  if ((tid & 31) == 0) { sh.wor[tid >> 5] = k_or; sh.wand[tid >> 5] = k_and; }
+#pragma unroll 1
+  for (int i = tid; i < kFastBins; i += T) L.s_hist[i] = 0;
   if (tid == 0) {
-    sh.lhist[0] = 0u;                        // OR / AND of the keys (reused as the timestamp histogram later)
-    sh.lhist[1] = 0xffffffffu;
+    sh.ncand = 0;
     c.n_sel[b] = k;
     atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
   }
@@ -706,81 +793,107 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   dbg_ts(b, 2);
   // ---- the GPU page table on its way (consumed after top-k) ---------------------------------
   fast_prefetch_gpt<T>(c, L, S);
+  fast_prefetch_tables<T>(c, L, bt.n_partitions[i_req]);
 
   // ---- top-k: radix select (two barriers per pass), one-scan ordered compaction -------------
   int32_t *g_sel = c.sel_ids + (size_t)b * c.max_sel;
   int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
   if (k == n) {
+#pragma unroll 1
     for (int i = tid; i < n; i += T) { s_sel[i] = i; g_sel[i] = i; }
   } else {
-    // The scores of one set share their sign, exponent and often a few mantissa bits, so the
-    // leading radix passes would put every key into one bin (and serialise on its counter).
-    // Bytes on which all keys agree (OR == AND over the set) are skipped outright.
-    uint32_t k_or = 0, k_and = 0xffffffffu;
-#pragma unroll 8
-    for (int i = tid; i < n; i += T) { const uint32_t key = key_at(i); k_or |= key; k_and &= key; }
-    k_or = __reduce_or_sync(0xffffffffu, k_or);
-    k_and = __reduce_and_sync(0xffffffffu, k_and);
-    if ((tid & 31) == 0) { atomicOr(&sh.lhist[0], k_or); atomicAnd(&sh.lhist[1], k_and); }
-    __syncthreads();
-    dbg_ts(b, 16);
-    const uint32_t differ = sh.lhist[0] ^ sh.lhist[1];           // bits on which some keys differ
-    uint32_t prefix = 0, mask = 0, remaining = k;
-    int first_shift = 24;
-    while (first_shift >= 0 && ((differ >> first_shift) & 255u) == 0) {
-      prefix |= sh.lhist[1] & (255u << first_shift);
-      mask |= 255u << first_shift;
-      first_shift -= 8;
-    }
-    int buf = 0;
-    for (int shift = first_shift; shift >= 0; shift -= 8, buf ^= 1) {
-#pragma unroll 8
-      for (int i = tid; i < n; i += T) {
-        const uint32_t key = key_at(i);
-        if ((key & mask) == prefix) atomicAdd(&sh.hist[buf][(key >> shift) & 255u], 1u);
-      }
-      __syncthreads();
-      if (tid < 32) {
-        uint32_t loc[8], sum = 0;
+    // Radix select with wide digits.  The scores of one set share their sign, exponent and often
+    // a few mantissa bits: the bits on which all keys agree (OR == AND) are skipped, and the
+    // first digit is the next kFastDigitBits bits.  One histogram then leaves a handful of keys
+    // in the bin of the k-th best, which one warp ranks directly; a bin that is still crowded
+    // goes round again on the following bits.
+    uint32_t a_or = 0, a_and = 0xffffffffu;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { loc[j] = sh.hist[buf][255 - 8 * tid - j]; sum += loc[j]; }
-        uint32_t inc = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
-          if (tid >= o) inc += v;
+    for (int j = 0; j < T / 32; ++j) { a_or |= sh.wor[j]; a_and &= sh.wand[j]; }
+    const uint32_t differ = a_or ^ a_and;                          // bits on which some keys differ
+    uint32_t thr = a_and, need_eq = k;                             // differ == 0: all keys are equal
+    if (differ != 0) {
+      int topbit = 31 - __clz(differ);                             // highest undecided bit
+      uint32_t mask = topbit == 31 ? 0u : ~((2u << topbit) - 1u);  // decided bits
+      uint32_t prefix = a_and & mask, remaining = k;
+      int wb = 0;
+      constexpr int kPer = kFastBins / T;
+#pragma unroll 1
+      for (;;) {
+        const int shift = max(0, topbit + 1 - kFastDigitBits), width = topbit + 1 - shift;
+        const uint32_t dmask = (1u << width) - 1u;
+#pragma unroll 1
+        for (int i = tid; i < n; i += T) {
+          const uint32_t key = key_at(i);
+          if ((key & mask) == prefix) atomicAdd(&L.s_hist[(key >> shift) & dmask], 1u);
         }
-        const uint32_t before = inc - sum;
-        if (before < remaining && inc >= remaining) {
+        __syncthreads();
+        uint32_t loc[kPer], sum = 0;                               // this thread's bins, best first
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) { loc[j] = L.s_hist[kFastBins - 1 - kPer * tid - j]; sum += loc[j]; }
+        uint32_t tot;
+        const uint32_t before = block_scan1<T>(sum, sh.wsum + wb, &tot);
+        wb ^= 16;
+        if (before < remaining && before + sum >= remaining) {
           uint32_t cum = before;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
+          for (int j = 0; j < kPer; ++j) {
             if (cum < remaining && cum + loc[j] >= remaining) {
-              sh.prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
+              sh.prefix = prefix | ((uint32_t)(kFastBins - 1 - kPer * tid - j) << shift);
               sh.remaining = remaining - cum;
+              sh.bin_count = loc[j];
             }
             cum += loc[j];
           }
         }
-      } else {
-        for (int i = tid - 32; i < 256; i += T - 32) sh.hist[buf ^ 1][i] = 0;   // for the pass after next
+        __syncthreads();
+        prefix = sh.prefix;
+        remaining = sh.remaining;
+        mask |= dmask << shift;
+        const uint32_t m = sh.bin_count;
+        if (shift == 0) break;                                     // the key is decided to its last bit
+        if (m <= (uint32_t)kFastSmall) {
+          // the bin's keys, gathered in any order; warp 0 finds the one with `remaining - 1` above it
+#pragma unroll 1
+          for (int i = tid; i < n; i += T) {
+            const uint32_t key = key_at(i);
+            if ((key & mask) == prefix) sh.cand[atomicAdd(&sh.ncand, 1u) & (kFastSmall - 1)] = key;
+          }
+          __syncthreads();
+          if (tid < 32) {
+            const uint32_t mine = tid < (int)m ? sh.cand[tid] : 0u;
+            uint32_t gt = 0, ge = 0;
+#pragma unroll 1
+            for (uint32_t j = 0; j < m; ++j) {
+              const uint32_t o = __shfl_sync(0xffffffffu, mine, (int)j);
+              gt += o > mine; ge += o >= mine;
+            }
+            if (tid < (int)m && gt < remaining && ge >= remaining) { sh.prefix = mine; sh.remaining = remaining - gt; }
+          }
+          __syncthreads();
+          prefix = sh.prefix;
+          remaining = sh.remaining;
+          break;
+        }
+        topbit = shift - 1;
+#pragma unroll 1
+        for (int i = tid; i < kFastBins; i += T) L.s_hist[i] = 0;
+        __syncthreads();
       }
-      __syncthreads();
-      prefix = sh.prefix;
-      remaining = sh.remaining;
-      mask |= 255u << shift;
-      // the buffer just searched is cleared by the next pass's idle warps (it is used again two passes on)
+      thr = prefix;
+      need_eq = remaining;
     }
     dbg_ts(b, 17);
-    const uint32_t thr = prefix, need_eq = remaining;
-    // every thread owns a contiguous run of candidates: two block scans place all of them
+    // every thread owns a contiguous run of candidates: one block scan (both counts packed into
+    // a word) places all of them in index order
     const int E = (n + T - 1) / T, lo = min(n, tid * E), hi = min(n, lo + E);
-    uint32_t gt = 0, eq = 0;
-#pragma unroll 8
-    for (int i = lo; i < hi; ++i) { const uint32_t key = key_at(i); gt += key > thr; eq += key == thr; }
-    uint32_t tot_gt, tot_eq;
-    uint32_t gt_before = block_scan<T>(gt, sh.wsum, &tot_gt);
-    uint32_t eq_before = block_scan<T>(eq, sh.wsum, &tot_eq);
+    uint32_t cnt = 0;                                              // above: low half, equal: high half
+#pragma unroll 1
+    for (int i = lo; i < hi; ++i) { const uint32_t key = key_at(i); cnt += (key > thr) + ((uint32_t)(key == thr) << 16); }
+    uint32_t tot_cnt;
+    const uint32_t ex = block_scan1<T>(cnt, sh.wsum + 8, &tot_cnt);
+    uint32_t gt_before = ex & 0xffffu, eq_before = ex >> 16;
+#pragma unroll 1
     for (int i = lo; i < hi; ++i) {
       const uint32_t key = key_at(i);
       if (key > thr || (key == thr && eq_before < need_eq)) {
@@ -794,13 +907,16 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   __syncthreads();
   int np = k;
   if (!token) {
+#pragma unroll 1
     for (int i = tid; i < k; i += T) g_parts[i] = s_sel[i];
   } else {
     // chosen tokens (ascending) -> their pages (ascending, unique) + a 16-bit token mask per page
     uint32_t *s_mask = reinterpret_cast<uint32_t *>(L.s_free);
+#pragma unroll 1
     for (int i = tid; i < k; i += T) s_mask[i] = 0;
     __syncthreads();
     uint32_t run = 0;
+#pragma unroll 1
     for (int base = 0; base < k; base += T) {
       const int i = base + tid;
       uint32_t first = 0;
@@ -821,9 +937,11 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
     np = (int)run;
     __syncthreads();
     uint32_t *g_mask = c.part_mask + (size_t)b * c.max_parts;
+#pragma unroll 1
     for (int i = tid; i < np; i += T) g_mask[i] = s_mask[i];
   }
   dbg_ts(b, 3);
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");     // page table copy and table snapshot have landed
   __syncthreads();
   cache_fast<T>(c, bt, b, i_req, set, L, np, sh);
 }
@@ -843,11 +961,13 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   int32_t *s_mdir = L.s_mdir, *s_gdir = L.s_gdir, *s_parts = L.s_parts, *s_tokens = L.s_tokens;
   int32_t *s_pageoff = L.s_pageoff, *s_missoff = L.s_missoff, *s_missbefore = L.s_missbefore;
   int32_t *s_state = L.s_state, *s_free = L.s_free, *s_host = L.s_host, *s_off = L.s_off;
+  const bool snap_host = fast_snap_host(c, L);
   uint32_t *s_hit = L.s_hit;
   if (tid == 0) { c.att_count[b] = 0; sh.evicted = 0; sh.admit_pages = 0; sh.bypass_pages = 0; }
   // ---- cache manager step 1: Meta-partition lookups, classification, page demand ------------
   int np = np_sel;
   uint32_t run_all = 0, run_miss = 0;
+#pragma unroll 1
   for (int base = 0; base < np; base += T) {
     const int r = base + tid;
     uint32_t npg = 0, miss = 0;
@@ -856,7 +976,8 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
       const int seg = s_mdir[p >> c.seg_shift];
       int tokens = 0, res = 1;
       if (seg >= 0) {
-        const int2 m = *reinterpret_cast<const int2 *>(c.meta_pool + ((size_t)seg << c.seg_shift) + (p & seg_mask));
+        const int2 m = p < L.tbl_cap ? L.s_meta[p]
+                                     : *reinterpret_cast<const int2 *>(c.meta_pool + ((size_t)seg << c.seg_shift) + (p & seg_mask));
         tokens = m.x; res = m.y;
       } else dev_error(c, kErrBounds);
       npg = (tokens + kPageTokens - 1) / kPageTokens;
@@ -866,7 +987,8 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
       if (miss && resolve_in_manager(c)) {
         // Retrieve step 3, first half: where the partition's pages start in the CPU page table
         const int oseg = L.s_odir[p >> c.seg_shift];
-        s_off[r] = oseg >= 0 ? (c.off_mirror ? c.off_mirror : c.off_pool)[((size_t)oseg << c.seg_shift) + (p & seg_mask)] : -1;
+        s_off[r] = (snap_host && p < L.tbl_cap) ? L.s_offt[p]
+                   : oseg >= 0 ? (c.off_mirror ? c.off_mirror : c.off_pool)[((size_t)oseg << c.seg_shift) + (p & seg_mask)] : -1;
       }
     }
     uint32_t tot_a, tot_m;
@@ -888,11 +1010,14 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     // more pages than the list holds (reported): whole partitions are dropped from the end
     if (tid == 0) dev_error(c, kErrPageList);
     __syncthreads();
+#pragma unroll 1
     while (np > 0 && s_pageoff[np] > c.max_pages) --np;
     total_pages = s_pageoff[np];
     demand = np < np_sel ? s_missbefore[np] : demand;
   }
+#pragma unroll 1
   for (int i = tid; i < (S + 31) / 32; i += T) s_hit[i] = 0;
+#pragma unroll 1
   for (int i = tid; i < kMaxBuckets + 2; i += T) sh.lhist[i] = 0;
   asm volatile("cp.async.wait_group 0;\n" ::: "memory");     // the GPU page table copy has landed
   __syncthreads();
@@ -911,6 +1036,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   int32_t *page_fill = c.page_fill + pl;
   int4 *page_desc = c.page_desc + pl;
   const bool early = c.fetch_mode == 0;
+#pragma unroll 1
   for (int mi = tid; mi < demand; mi += T) {
     const int r = owner_of(s_missbefore, np, mi);
     const int i = mi - s_missbefore[r], p = s_parts[r];
@@ -919,7 +1045,8 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
       // second half: the CPU page table entry (directory in shared memory, one global read)
       const int e = s_off[r] + i;
       const int cseg = (s_off[r] >= 0 && (e >> c.seg_shift) < c.dir_page) ? L.s_cdir[e >> c.seg_shift] : -1;
-      host_page = cseg >= 0 ? (c.cpt_mirror ? c.cpt_mirror : c.cpt_pool)[((size_t)cseg << c.seg_shift) + (e & seg_mask)] : -1;
+      host_page = (snap_host && e >= 0 && e < L.tbl_cap && e < bt.n_partitions[i_req]) ? L.s_cptt[e]
+                  : cseg >= 0 ? (c.cpt_mirror ? c.cpt_mirror : c.cpt_pool)[((size_t)cseg << c.seg_shift) + (e & seg_mask)] : -1;
       if (host_page < -1) host_page = -1;
     }
     s_host[mi] = host_page;
@@ -941,6 +1068,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
 
   dbg_ts(b, 19);
   // ---- step 2: one pass over the page table copy: promote, demote, histogram ----------------
+#pragma unroll 1
   for (int s_ = tid; s_ < S; s_ += T) {
     int4 e = s_gpt[s_];
     if (c.trace) {
@@ -970,6 +1098,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     if (demand > 0) {
       x = nb - 1;
       uint32_t cum = 0;
+#pragma unroll 1
       for (int bk = -1; bk < nb; ++bk) {
         cum += sh.lhist[bk + 1];
         if ((int)cum >= demand) { x = bk; break; }
@@ -984,6 +1113,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   if (demand > 0) {
     const int E = (S + T - 1) / T, lo = min(S, tid * E), hi = min(S, lo + E);
     uint32_t nfree = 0;
+#pragma unroll 1
     for (int s_ = lo; s_ < hi; ++s_) {
       int4 e = s_gpt[s_];
       if (e.x < 0) { ++nfree; continue; }
@@ -1001,6 +1131,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     }
     uint32_t tot;
     uint32_t pos = block_scan<T>(nfree, sh.wsum, &tot);
+#pragma unroll 1
     for (int s_ = lo; s_ < hi; ++s_)
       if (s_gpt[s_].x < 0) { if (pos < (uint32_t)c.max_pages) s_free[pos] = s_; ++pos; }
     run_free = tot;
@@ -1013,6 +1144,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   if (demand > (int)run_free) {
     if (tid == 0) {
       int used = 0;
+#pragma unroll 1
       for (int r = 0; r < np; ++r) {
         if (s_state[r] == kHit) continue;
         const int npg = (s_tokens[r] + kPageTokens - 1) / kPageTokens;
@@ -1027,6 +1159,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   __syncthreads();
   const int qbase = sh.qbase;
   dbg_ts(b, 22);
+#pragma unroll 1
   for (int r = tid; r < np; r += T) {
     c.part_state[(size_t)b * c.max_parts + r] = s_state[r];
     if (s_state[r] == kAdmit) {
@@ -1036,6 +1169,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   }
   int my_admit = 0, my_bypass = 0;
   dbg_ts(b, 23);
+#pragma unroll 1
   for (int idx = tid; idx < total_pages; idx += T) {
     const int r = owner_of(s_pageoff, np, idx);
     const int i = idx - s_pageoff[r], p = s_parts[r], state = s_state[r];
@@ -1082,6 +1216,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   dbg_ts(b, 24);
   if (my_admit) atomicAdd(&sh.admit_pages, my_admit);
   if (my_bypass) atomicAdd(&sh.bypass_pages, my_bypass);
+#pragma unroll 1
   for (int j = tid; j < tail_pages; j += T) {
     const int idx = total_pages + j;
     const int src = c.tail_phys[(size_t)set * c.tail_cap + j];
@@ -1113,6 +1248,7 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     flag_publish(c.ready + b, bt.epoch);
   }
   // ---- the page table goes back in one sweep; attention does not wait for it -----------------
+#pragma unroll 1
   for (int s_ = tid; s_ < S; s_ += T) {
     const int seg = s_gdir[s_ >> c.seg_shift];
     if (seg >= 0) *reinterpret_cast<int4 *>(c.gpt_pool + ((size_t)seg << c.seg_shift) + (s_ & seg_mask)) = s_gpt[s_];
