@@ -172,13 +172,11 @@ __device__ __forceinline__ void fetched_page_to_slot(const DevCtx &c, const Batc
 }
 
 template <int G>
-__global__ void __launch_bounds__(kAttnWarps * 32)
-k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out) {
-  extern __shared__ __align__(128) uint8_t smem_pages[];          // [8][8192]
+__device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const __nv_bfloat16 *__restrict__ q,
+                                         __nv_bfloat16 *__restrict__ out, uint8_t *smem_pages) {
   __shared__ float sh[kAttnWarps][G][kPartStride];
   __shared__ int sh_last;
   const int b = blockIdx.x, chunk = blockIdx.y;       // chunk-major launch order: chunk 0 of every set first
-  pdl_launch_next();
   const int first = chunk * kChunkPages;
   bool slots_known = true;                 // false: the chunk holds early descriptors only
   if (c.ready) {
@@ -382,6 +380,19 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
     const float den = s_den[g];
     out[((size_t)i_req * c.Hq + head * G + g) * kHeadDim + ch] = __float2bfloat16(den > 0.f ? a_o / den : 0.f);
   }
+}
+
+// The kernel: the CTA's work; one CTA then waits for the kernel before this one.  CTAs that
+// go by the per-set flags never wait for the scoring kernel as a whole; with one CTA doing so
+// before it exits, this grid cannot complete ahead of that one, and whatever the stream runs
+// next (the next step's scoring kernel waits for this grid) comes after all of its writes.
+template <int G>
+__global__ void __launch_bounds__(kAttnWarps * 32)
+k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out) {
+  extern __shared__ __align__(128) uint8_t smem_pages[];          // [8][8192]
+  pdl_launch_next();
+  attn_cta<G>(c, bt, q, out, smem_pages);
+  if (blockIdx.x == 0 && blockIdx.y == 0) pdl_wait_prev();
 }
 
 // Sets whose page list is empty get a zero output (no CTA of k_attn reaches them).

@@ -48,7 +48,7 @@ template <int G, bool MINMAX>
 __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, const float (&qf)[G][8],
                                              const uint32_t (&qsel)[G][4], uint32_t row_mask) {
   const uint32_t a[4] = {lo.x, lo.y, lo.z, lo.w}, m[4] = {hi.x, hi.y, hi.z, hi.w};
-  float tot = 0.f;
+  float v[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     float x[8];
@@ -61,11 +61,40 @@ __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, con
     float s = qf[g][0] * x[0];
 #pragma unroll
     for (int i = 1; i < 8; ++i) s = fmaf(qf[g][i], x[i], s);     // exact product, one rounding: s + q*x
-    s = s + __shfl_xor_sync(row_mask, s, 1);
-    s = s + __shfl_xor_sync(row_mask, s, 2);
-    s = s + __shfl_xor_sync(row_mask, s, 4);
-    s = s + __shfl_xor_sync(row_mask, s, 8);
-    tot = g == 0 ? s : tot + s;
+    v[g] = s;
+  }
+  // The 16 block sums of every head go up the balanced tree (lanes l and l^1, then l^2, l^4,
+  // l^8: both partners form the same sum, addition being commutative).  While more than one
+  // head is left in a lane, a level also halves that number: the partners keep one half of
+  // the heads each and trade the other, so a level costs n/2 shuffles instead of n.  Lane l
+  // of a row ends up with the total of the head whose index is l's low bits reversed.
+  const int lane = threadIdx.x & 15;
+  int n = G;
+#pragma unroll
+  for (int level = 0; level < 4; ++level) {
+    if (n > 1) {
+      const bool up = (lane >> level) & 1;
+      const int half = n / 2;
+#pragma unroll
+      for (int i = 0; i < G / 2; ++i)
+        if (i < half) {
+          const float send = up ? v[i] : v[i + half], keep = up ? v[i + half] : v[i];
+          v[i] = keep + __shfl_xor_sync(row_mask, send, 1 << level);
+        }
+      n = half;
+    } else {
+      v[0] = v[0] + __shfl_xor_sync(row_mask, v[0], 1 << level);
+    }
+  }
+  // heads in ascending order, into the row's first lane
+  float tot = v[0];
+#pragma unroll
+  for (int h = 1; h < G; ++h) {
+    constexpr int kBits = G == 8 ? 3 : G == 4 ? 2 : 1;
+    int src = 0;
+#pragma unroll
+    for (int bit = 0; bit < kBits; ++bit) src |= ((h >> bit) & 1) << (kBits - 1 - bit);
+    tot = tot + __shfl_sync(row_mask, v[0], src, 16);
   }
   return tot + 0.0f;                              // -0.0 -> +0.0
 }
