@@ -232,6 +232,7 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.att_part = a.take<float>(B * g.max_chunks * G * (kHeadDim + 2));
   d.att_count = a.take<int32_t>(B);
   d.sel_count = a.take<int32_t>(B);
+  d.scored = a.take<int32_t>(B);
   d.ready = a.take<int32_t>(B);
   d.tail_ready = a.take<int32_t>(B);
   d.ready1 = a.take<int32_t>(B);
@@ -665,6 +666,7 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   memset(ctx->host_base, 0, ctx->host_bytes);
   fill(d.att_count, 0, (size_t)g.max_batch_sets * 4);
   fill(d.sel_count, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.scored, 0, (size_t)g.max_batch_sets * 4);
   fill(d.ready, 0, (size_t)g.max_batch_sets * 4);
   fill(d.tail_ready, 0, (size_t)g.max_batch_sets * 4);
   fill(d.ready1, 0, (size_t)g.max_batch_sets * 4);

@@ -109,19 +109,11 @@ size_t cache_smem_bytes(const DevCtx &c) { return cache_stage_smem_bytes(c.max_p
 
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
   static size_t configured = 0;
-  int max_slots_batch = 0;
-  for (int i = 0; i < b.n_req; ++i) max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
-  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, 0);
-  const int fast = (max_slots_batch <= kFastSlots && fs <= 96 * 1024) ? 1 : 0;
-  size_t smem = fast ? fs : cache_smem_bytes(c);
   int tbl_cap = 0;
-  if (fast && c.kind != kKindCluster) {
-    // one CTA per set: the snapshot of the partition tables may take what shared memory is left
-    int max_parts_batch = 0;
-    for (int i = 0; i < b.n_req; ++i) max_parts_batch = b.n_partitions[i] > max_parts_batch ? b.n_partitions[i] : max_parts_batch;
-    const size_t ft = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, max_parts_batch);
-    if (max_parts_batch > 0 && ft <= 200 * 1024) { tbl_cap = max_parts_batch; smem = ft; }
-  }
+  size_t smem = 0;
+  // one CTA per set: the snapshot of the partition tables may take what shared memory is left
+  const int fast = plan_cache_fast(c, b, 200 * 1024, &tbl_cap, &smem) ? 1 : 0;
+  if (!fast) smem = cache_smem_bytes(c);
   if (smem > configured) {
     cudaFuncSetAttribute(k_cache, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;

@@ -102,7 +102,7 @@ __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, con
 template <int G, bool MINMAX>
 __global__ void __launch_bounds__(kScoreThreads, 3)
 k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
-        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap, int tbl_cap) {   // fuse: 0 none, 1 staged, 2 fast
+        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap, int tbl_cap) {   // fuse: 0 none, 1 staged, 2 fast, 3 flag only
   extern __shared__ __align__(16) uint8_t dyn_smem[];      // used by the fused continuation only
   const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
@@ -203,6 +203,11 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
   dbg_ts(b, 9);
   __threadfence();
   if (threadIdx.x == 0) c.sel_count[b] = 0;                 // ready for the next step
+  if (fuse == 3) {
+    // selection runs in the cluster kernel behind this one: tell it that this set is scored
+    if (threadIdx.x == 0) flag_publish(c.scored + b, bt.epoch);
+    return;
+  }
   if (fuse == 2) {
     select_fast<kScoreThreads>(c, bt, b, i_req, set, dyn_smem, keys_cap, tbl_cap, shm.fast);
     return;
@@ -213,17 +218,58 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
 }
 
 // Stand-alone top-k: one thread-block cluster per set (slices of the keys in shared memory).
-__global__ void __launch_bounds__(kTopkThreads)
-k_topk(DevCtx c, Batch bt, int keys_cap) {
-  extern __shared__ __align__(16) uint8_t dyn_smem[];
-  __shared__ TopkShared tsh;
-  const int C = (int)cg::this_cluster().num_blocks();
-  const int b = blockIdx.x / C, i_req = b / c.Hkv, head = b % c.Hkv;
+// With wait_flags a cluster starts as soon as its own set is scored (the flag the scoring
+// kernel's last CTA of that set raises) instead of when the whole scoring kernel is done; the
+// outcome of the bounded wait is shared through the first CTA so that all CTAs of the
+// cluster take the same path through the cluster barriers.
+__device__ __forceinline__ void topk_cta(const DevCtx &c, const Batch &bt, int keys_cap, int manage, int tbl_cap,
+                                         int wait_flags, uint8_t *dyn_smem) {
+  __shared__ union { TopkShared t; FastShared f; } shm;
+  __shared__ int s_ok;
+  TopkShared &tsh = shm.t;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const int b = blockIdx.x / C, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
+  if (wait_flags) {
+    if (rank == 0 && tid == 0) s_ok = flag_wait(c, c.scored + b, bt.epoch);
+    cluster.sync();
+    const int ok = *cluster.map_shared_rank(&s_ok, 0);
+    cluster.sync();                                   // the first CTA's word is not read after this
+    if (!ok) return;
+  } else {
+    pdl_wait_prev();
+  }
+  if (rank == 0) dbg_ts(b, 9);
+  // the first CTA is also the set's cache manager: its tables start towards shared memory now
+  // (behind the keys' slice) and arrive while the select runs
+  const int S = bt.slots[i_req];
+  const FastLayout L = fast_layout(c, dyn_smem + (((size_t)keys_cap * 4 + 15) & ~(size_t)15), 0, S, tbl_cap);
+  const bool mgr = manage && rank == 0;
+  if (mgr) {
+    fast_prefetch_dirs<kTopkThreads>(c, L, set, S);
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    __syncthreads();
+    fast_prefetch_gpt<kTopkThreads>(c, L, S);
+    fast_prefetch_tables<kTopkThreads>(c, L, bt.n_partitions[i_req]);
+  }
+  const bool first = topk_stage<kTopkThreads, true>(c, b, bt.n_partitions[i_req], reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh);
+  if (!first || !manage) return;
+  const int np = c.n_parts[b];
+  const int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
+  for (int r = tid; r < np; r += kTopkThreads) L.s_parts[r] = g_parts[r];
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+  __syncthreads();
+  cache_fast<kTopkThreads>(c, bt, b, i_req, set, L, np, shm.f);
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+k_topk(DevCtx c, Batch bt, int keys_cap, int manage, int tbl_cap, int wait_flags) {
+  extern __shared__ __align__(16) uint8_t dyn_smem[];
   pdl_launch_next();
-  pdl_wait_prev();
-  const SetState st = c.state[set];
-  topk_stage<kTopkThreads, true>(c, b, st.n_partitions, reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh);
+  topk_cta(c, bt, keys_cap, manage, tbl_cap, wait_flags, dyn_smem);
+  // a grid that went by the flags must still not complete before the scoring kernel has
+  if (wait_flags && blockIdx.x == 0) pdl_wait_prev();
 }
 
 
@@ -274,6 +320,12 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
     }
   }
   if (smem < 64 * 1024) smem = 64 * 1024;         // the scoring CTAs' staging area: one summary segment
+  // not fused: the cluster kernel behind this one selects; when it also manages the cache it
+  // starts set by set, on the flag the last scoring CTA of a set raises (fuse 3)
+  int mgr_tbl_cap = 0;
+  size_t mgr_smem = 0;
+  const int manage = !fuse && plan_cache_fast(c, b, 160 * 1024, &mgr_tbl_cap, &mgr_smem) ? 1 : 0;
+  if (manage) fuse = 3;
   switch (c.G) {
     case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
     case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
@@ -281,7 +333,7 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
     default: launch_score_g<8>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
   }
   prof_mark(prof, st, kProfScore);
-  if (fuse) return 1;
+  if (fuse == 1 || fuse == 2) return 1;
   {
     // cluster size from the largest candidate count: slices of at most 8192 keys stay in smem
     int C = 1;
@@ -289,11 +341,14 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
     int kc = (max_cand + C - 1) / C;
     if (kc > 16384) kc = 0;                              // too many for shared memory: re-read from L2
     static int smem_set = 0;
-    const int ksmem = kc * 4;
+    int ksmem = kc * 4;
+    // the cache manager runs in the same kernel when it can work on shared-memory copies
+    if (manage) ksmem = ((ksmem + 15) & ~15) + (int)mgr_smem;    // the manager's tables sit behind the keys
     if (ksmem > smem_set) { cudaFuncSetAttribute(k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, ksmem); smem_set = ksmem; }
-    launch_pdl(k_topk, dim3(n_sets * C), dim3(kTopkThreads), (size_t)ksmem, st, C, c, b, kc);
+    launch_pdl(k_topk, dim3(n_sets * C), dim3(kTopkThreads), (size_t)ksmem, st, C, c, b, kc, manage, mgr_tbl_cap, manage);
+    prof_mark(prof, st, kProfTopk);
+    if (manage) return 2;
   }
-  prof_mark(prof, st, kProfTopk);
   return 2 + launch_cache(c, b, st, prof);
 }
 

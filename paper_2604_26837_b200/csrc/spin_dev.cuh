@@ -102,6 +102,7 @@ struct DevCtx {
   float *att_part;              // split-K partials [b][max_chunks][G][kHeadDim + 2]
   int32_t *att_count;           // [b] chunks of the set that have finished (zero before attention)
   int32_t *sel_count;           // [b] scoring CTAs of the set that have finished (zero between steps)
+  int32_t *scored;              // [b] epoch of the last step whose scores are complete (stand-alone top-k waits on it)
   int32_t *ready;               // [b] epoch of the last step whose page list is complete
   int32_t *tail_ready;          // [b] epoch of the last step whose appended rows are in the tail page
   int32_t *ready1;              // [b] epoch of the last step whose missed pages are listed (before their slots are known)

@@ -102,12 +102,20 @@ __device__ __forceinline__ int owner_of(const int32_t *off, int n, int idx) {
 // so that a set's page list never waits on the host link.
 __device__ __forceinline__ bool resolve_in_manager(const DevCtx &c) { return c.fetch_mode != 0 || c.cpt_mirror != nullptr; }
 
+#ifdef SPIN_TIMING
+__device__ unsigned long long g_dbg_ts[256][32];
+__device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; } }
+#else
+__device__ __forceinline__ void dbg_ts(int, int) {}
+#endif
+
 struct TopkShared {
   uint32_t hist[256];          // this CTA's histogram (read remotely inside a cluster)
   uint32_t ghist[256];         // histogram over the whole set
   uint32_t wsum[33];
   uint32_t cnt[2];             // this CTA's (above threshold, equal) counts
   uint32_t prefix, remaining;
+  uint32_t orand[2];           // OR and AND of this CTA's keys (read remotely inside a cluster)
 };
 
 template <bool CLUSTER> __device__ __forceinline__ void stage_sync() {
@@ -143,29 +151,61 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
     c.n_sel[b] = k;
     atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
   }
-  if (cached)
-    for (int i = tid; i < m; i += T) s_keys[i] = order_key(__ldcg(scores + lo + i));
+  if (tid == 0) { sh.orand[0] = 0u; sh.orand[1] = 0xffffffffu; }
   __syncthreads();
+  // keys -> shared memory, with the OR and AND of the slice taken on the way
+  {
+    uint32_t k_or = 0, k_and = 0xffffffffu;
+    for (int i = tid; i < m; i += T) {
+      const uint32_t key = order_key(__ldcg(scores + lo + i));
+      if (cached) s_keys[i] = key;
+      k_or |= key; k_and &= key;
+    }
+    k_or = __reduce_or_sync(0xffffffffu, k_or);
+    k_and = __reduce_and_sync(0xffffffffu, k_and);
+    if ((tid & 31) == 0) { atomicOr(&sh.orand[0], k_or); atomicAnd(&sh.orand[1], k_and); }
+  }
+  stage_sync<CLUSTER>();
+  if (rank == 0) dbg_ts(b, 25);
   auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(__ldcg(scores + lo + i)); };
 
   if (k == n) {
     for (int i = tid; i < m; i += T) sel[lo + i] = lo + i;
   } else {
     // ---- radix select: key of the k-th best candidate --------------------------------
-    uint32_t prefix = 0, mask = 0, remaining = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
+    // The scores of one set share their sign, exponent and often some mantissa bits; a digit
+    // taken there would put every key into one bin (and serialise on its counter).  The bits
+    // on which all keys agree (OR == AND over the set) are decided from the start and the
+    // first 8-bit digit begins at the highest bit that differs.
+    uint32_t a_or = 0, a_and = 0xffffffffu;
+    if constexpr (CLUSTER) {
+      cg::cluster_group cluster = cg::this_cluster();
+      for (int r = 0; r < C; ++r) {
+        const uint32_t *ro = cluster.map_shared_rank(sh.orand, r);
+        a_or |= ro[0]; a_and &= ro[1];
+      }
+    } else { a_or = sh.orand[0]; a_and = sh.orand[1]; }
+    const uint32_t differ = a_or ^ a_and;
+    int topbit = differ ? 31 - __clz(differ) : -1;                 // -1: all keys are equal
+    uint32_t mask = topbit >= 31 ? 0u : ~((2u << max(topbit, 0)) - 1u);
+    if (topbit < 0) mask = 0xffffffffu;
+    uint32_t prefix = a_and & mask, remaining = k;
+    for (; topbit >= 0;) {
+      const int shift = max(0, topbit + 1 - 8), width = topbit + 1 - shift;
+      const uint32_t dmask = (1u << width) - 1u;
       if (tid < 256) sh.hist[tid] = 0;
       __syncthreads();
       for (int i = tid; i < m; i += T) {
         const uint32_t key = key_at(i);
-        if ((key & mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
+        if ((key & mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & dmask], 1u);
       }
       stage_sync<CLUSTER>();                          // every CTA's histogram is complete
       for (int bin = tid; bin < 256; bin += T) {
         uint32_t tot = 0;
         if constexpr (CLUSTER) {
           cg::cluster_group cluster = cg::this_cluster();
-          for (int r = 0; r < C; ++r) tot += cluster.map_shared_rank(sh.hist, r)[bin];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) tot += r < C ? cluster.map_shared_rank(sh.hist, r)[bin] : 0u;   // loads issued together
         } else {
           tot = sh.hist[bin];
         }
@@ -200,9 +240,11 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
       __syncthreads();
       prefix = sh.prefix;
       remaining = sh.remaining;
-      mask |= 255u << shift;
+      mask |= dmask << shift;
+      topbit = shift - 1;
     }
     const uint32_t thr = prefix, need_eq = remaining;
+    if (rank == 0) dbg_ts(b, 26);
     // ---- counts of this slice, offsets from the lower-ranked slices ---------------------
     uint32_t run_gt = 0, run_eq = 0;
     if constexpr (CLUSTER) {
@@ -262,8 +304,10 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
       }
     }
   }
+  if (rank == 0) dbg_ts(b, 27);
   stage_sync<CLUSTER>();     // selections of all slices are written; no remote smem is read after this
   if (rank != 0) return false;
+  dbg_ts(b, 28);
 
   // ---- candidates -> partitions of the cache manager (first CTA of the cluster) ----------
   int32_t *parts = c.parts + (size_t)b * c.max_parts;
@@ -273,29 +317,38 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
     __syncthreads();
     return true;
   }
+  // chosen tokens (ascending) -> their pages (ascending, unique) + a 16-bit token mask per page.
+  // Every thread owns a contiguous run of the selection: one block scan numbers the pages.
   uint32_t *pmask = c.part_mask + (size_t)b * c.max_parts;
   for (int i = tid; i < k; i += T) pmask[i] = 0;
-  __syncthreads();
-  uint32_t run = 0;
-  for (int base = 0; base < k; base += T) {
-    const int i = base + tid;
-    uint32_t first = 0;
-    int tok = 0;
-    if (i < k) {
-      tok = __ldcg(sel + i);
-      first = (i == 0) || ((__ldcg(sel + i - 1) >> 4) != (tok >> 4));
+  const int E = (k + T - 1) / T, r0 = min(k, tid * E), r1 = min(k, r0 + E);
+  const int page_before = r0 > 0 && r0 < k ? (__ldcg(sel + r0 - 1) >> 4) : -1;
+  uint32_t firsts = 0;
+  {
+    int pp = page_before;
+    for (int i = r0; i < r1; ++i) { const int pg = __ldcg(sel + i) >> 4; firsts += pg != pp; pp = pg; }
+  }
+  uint32_t run;
+  const uint32_t ex = block_scan<T>(firsts, sh.wsum, &run);      // its barriers also order the zeroing above
+  {
+    int pp = page_before, rank_ = (int)ex - 1;
+    uint32_t acc = 0;
+    for (int i = r0; i < r1; ++i) {
+      const int tok = __ldcg(sel + i), pg = tok >> 4;
+      if (pg != pp) {
+        if (acc) atomicOr(&pmask[rank_], acc);
+        acc = 0;
+        ++rank_;
+        parts[rank_] = pg;
+        pp = pg;
+      }
+      acc |= 1u << (tok & 15);
     }
-    uint32_t total;
-    const uint32_t ex = block_scan<T>(first, sh.wsum, &total);
-    if (i < k) {
-      const uint32_t rank_ = run + ex + first - 1;
-      if (first) parts[rank_] = tok >> 4;
-      atomicOr(&pmask[rank_], 1u << (tok & 15));
-    }
-    run += total;
+    if (acc) atomicOr(&pmask[rank_], acc);
   }
   if (tid == 0) c.n_parts[b] = (int)run;
   __syncthreads();
+  dbg_ts(b, 29);
   return true;
 }
 
@@ -599,12 +652,6 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
 // time before the set's missed pages can start to cross the host link.
 constexpr int kFastSlots = 1024;
 
-#ifdef SPIN_TIMING
-__device__ unsigned long long g_dbg_ts[256][32];
-__device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; } }
-#else
-__device__ __forceinline__ void dbg_ts(int, int) {}
-#endif
 
 constexpr int kFastDigitBits = 11, kFastBins = 1 << kFastDigitBits;
 constexpr int kFastSmall = 32;               // a threshold bin this small is finished by one warp
@@ -629,6 +676,25 @@ __host__ __device__ inline size_t fast_smem_bytes(int n_keys, int slots, int dir
   b += (size_t)((tbl_cap + 3) / 4 * 4) * 16 + 16;                // snapshot of the set's three partition tables
   b += (size_t)2048 * 4;                                         // digit histogram of the select
   return b + 64;
+}
+
+// Host side: can one CTA run the cache manager of every set of this batch on shared-memory
+// copies (cache_fast), and if so with how large a snapshot of the partition tables?
+inline bool plan_cache_fast(const DevCtx &c, const Batch &b, size_t smem_limit, int *tbl_cap, size_t *smem) {
+  int max_slots_batch = 0, max_parts_batch = 0;
+  for (int i = 0; i < b.n_req; ++i) {
+    max_slots_batch = b.slots[i] > max_slots_batch ? b.slots[i] : max_slots_batch;
+    max_parts_batch = b.n_partitions[i] > max_parts_batch ? b.n_partitions[i] : max_parts_batch;
+  }
+  const size_t fs = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, 0);
+  *tbl_cap = 0;
+  *smem = fs;
+  if (max_slots_batch > 1024 || fs > 96 * 1024) return false;
+  if (c.kind != kKindCluster && max_parts_batch > 0) {
+    const size_t ft = fast_smem_bytes(0, max_slots_batch, c.dir_part, c.dir_slot, c.dir_page, c.max_parts, c.max_pages, max_parts_batch);
+    if (ft <= smem_limit) { *tbl_cap = max_parts_batch; *smem = ft; }
+  }
+  return true;
 }
 
 __device__ __forceinline__ void cp_async4(void *smem_dst, const void *gsrc) {
