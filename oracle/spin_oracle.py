@@ -149,7 +149,7 @@ class LruResult:
 
 def bucketed_lru_step(slot_part: np.ndarray, slot_pidx: np.ndarray, slot_ts: np.ndarray,
                       resident: np.ndarray, n_pages_of: np.ndarray,
-                      selected: Sequence[int], t: int, n: int) -> LruResult:
+                      selected: Sequence[int], t: int, n: int, exact: bool = False) -> LruResult:
     """One replacement round of one set; mutates the slot arrays and `resident` in place.
 
     slot_part/slot_pidx/slot_ts: int arrays [S]; an empty slot has partition -1 and
@@ -167,6 +167,10 @@ def bucketed_lru_step(slot_part: np.ndarray, slot_pidx: np.ndarray, slot_ts: np.
             histogram and are never victims; for n >= 2 they sit alone in bucket `top`,
             so this equals the paper's rule whenever the other slots can meet the demand.
             If even x = n-1 does not meet the demand, x = n-1 (everything else goes).
+            Variant `exact` (not the paper's rule; it measures what the over-eviction costs):
+            pages with ts < x go as before, but of bucket x only the first
+            `demand - #(pool pages with ts < x)` pages in ascending slot order are taken;
+            a partition that loses a page this way goes whole (cached whole or not at all).
     Step 4  admission.  Reading (the paper does not say which freed page goes to which
             miss): free slots in ascending slot order, missed pages in ascending
             (partition, page_idx) order, i-th page to i-th free slot, timestamp `top`.
@@ -198,7 +202,13 @@ def bucketed_lru_step(slot_part: np.ndarray, slot_pidx: np.ndarray, slot_ts: np.
             if int(np.count_nonzero(pool & (slot_ts <= x))) >= demand:
                 threshold = x
                 break
-        for s in np.nonzero(occupied & pool & (slot_ts <= threshold))[0]:
+        victim = occupied & pool & (slot_ts <= threshold)
+        if exact and threshold >= 0:
+            need = demand - int(np.count_nonzero(pool & (slot_ts < threshold)))
+            bucket = np.nonzero(occupied & pool & (slot_ts == threshold))[0]      # ascending slots
+            taken = np.unique(slot_part[bucket[:max(need, 0)]])
+            victim = occupied & pool & ((slot_ts < threshold) | np.isin(slot_part, taken))
+        for s in np.nonzero(victim)[0]:
             evicted.append((int(s), int(slot_part[s]), int(slot_pidx[s])))
             resident[slot_part[s]] = 0
             slot_part[s] = -1
@@ -279,6 +289,7 @@ class OracleConfig:
     partition_kind: int = PART_PAGE_MINMAX
     topk: int = 16
     lru_buckets: int = 64
+    evict_exact: bool = False      # evict only what the demand needs (variant, see bucketed_lru_step)
     sm_scale: float = 0.0          # 0 -> 1/sqrt(head_dim) (the paper gives no scale)
 
 
@@ -477,7 +488,7 @@ class OracleSet:
         n_pages_of = np.asarray([self.partition_pages(p) for p in range(P)], dtype=np.int64)
         resident = np.asarray(self.part_resident, dtype=np.int64)
         res = bucketed_lru_step(self.slot_part, self.slot_pidx, self.slot_ts, resident,
-                                n_pages_of, parts, self.t, cfg.lru_buckets)
+                                n_pages_of, parts, self.t, cfg.lru_buckets, cfg.evict_exact)
         self.part_resident = [int(x) for x in resident]
 
         # page list: selected partitions ascending, pages of a partition in order, then tail
