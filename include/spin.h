@@ -106,6 +106,11 @@ typedef struct spin_config {
                                    kernels keep up to date; 1: they read the pinned host tables
                                    over the host link, as in Section 5.2 (saves the mirror's HBM,
                                    but those small reads queue behind the page traffic) */
+  int32_t evict_exact;          /* 0: the paper's eviction (every page up to the threshold
+                                   timestamp goes, Section 5.3); 1: a variant for measuring
+                                   what that over-eviction costs: of the threshold bucket only
+                                   as many pages as the misses still need are taken, lowest
+                                   slots first (a partition that loses a page goes whole) */
   int64_t gpu_cache_pages;      /* HBM pages (8 KiB each) shared by all sets' cache slots */
   int64_t host_pages;           /* pinned host pages (8 KiB each) for the complete KV */
   void *hbm_pool;               /* device pointer, 256-byte aligned, caller-owned */

@@ -289,8 +289,8 @@ class OracleConfig:
     partition_kind: int = PART_PAGE_MINMAX
     topk: int = 16
     lru_buckets: int = 64
-    evict_exact: bool = False      # evict only what the demand needs (variant, see bucketed_lru_step)
     sm_scale: float = 0.0          # 0 -> 1/sqrt(head_dim) (the paper gives no scale)
+    evict_exact: bool = False      # evict only what the demand needs (variant, see bucketed_lru_step)
 
 
 class OracleSet:

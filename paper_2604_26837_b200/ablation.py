@@ -4,9 +4,11 @@ throughput and GPU hit ratio of one workload as the per-set HBM budget goes from
 ("+Mandatory": room for one step's selection, i.e. only last step's pages can hit), to
 multiples of it ("+Buffering": the bucketed LRU keeps older pages).
 
-    python -m paper_2604_26837_b200.ablation [--workload c2] [--batch 2] [--steps 96]
+    python -m paper_2604_26837_b200.ablation [--workload c2] [--batch 2] [--steps 96] [--evict-exact]
 
-Prints one line per budget.  Marshalling and timing only; every stage runs in the library.
+Prints one line per budget; with --evict-exact every budget is run twice, once with the paper's
+eviction (every page up to the threshold timestamp) and once with the exact-demand variant,
+to show what the over-eviction costs in hit ratio.  Marshalling and timing only; every stage runs in the library.
 """
 from __future__ import annotations
 
@@ -20,8 +22,8 @@ import workloads as W
 from .driver import SpinRun
 
 
-def run_budget(w: W.Workload, slots: int, steps: int, prime: int, device="cuda:0") -> dict:
-    run = SpinRun(W.scaled(w, steps=steps + prime + 2), device, slots_per_set=slots)
+def run_budget(w: W.Workload, slots: int, steps: int, prime: int, device="cuda:0", evict_exact: int = 0) -> dict:
+    run = SpinRun(W.scaled(w, steps=steps + prime + 2), device, slots_per_set=slots, evict_exact=evict_exact)
     stream = torch.cuda.Stream(device)
     B, L = w.batch, w.num_layers
     with torch.cuda.stream(stream):
@@ -53,7 +55,8 @@ def run_budget(w: W.Workload, slots: int, steps: int, prime: int, device="cuda:0
     sel = st1["selected_pages"] - st0["selected_pages"]
     hit = st1["hit_pages"] - st0["hit_pages"]
     res = dict(slots=slots, tokens_per_s=B * steps / (ms * 1e-3), ms_per_step=ms / steps,
-               hit_ratio=hit / max(sel, 1), bypass_pages=st1["bypass_pages"] - st0["bypass_pages"],
+               hit_ratio=hit / max(sel, 1), evicted_pages_per_step=(st1["evicted_pages"] - st0["evicted_pages"]) / steps,
+               bypass_pages=st1["bypass_pages"] - st0["bypass_pages"],
                pcie_mb_per_step=(st1["pcie_bytes"] - st0["pcie_bytes"]) / steps / 1e6,
                error_bits=st1["error_bits"])
     run.close()
@@ -66,6 +69,7 @@ def main():
     ap.add_argument("--batch", type=int, default=2)
     ap.add_argument("--steps", type=int, default=96)
     ap.add_argument("--prime", type=int, default=32)
+    ap.add_argument("--evict-exact", action="store_true")
     args = ap.parse_args()
     w = W.scaled(W.CONFIGS[args.workload], batch=args.batch)
     mandatory = w.topk * max(1, w.max_partition_pages // 2 if w.partition_kind == W.PART_CLUSTER_CENTROID else 1)
@@ -76,6 +80,9 @@ def main():
                         (4, "+Buffering 4x"), (5, "+Buffering 5x"), (6, "+Buffering 6x"), (8, "+Buffering 8x")):
         r = run_budget(w, mandatory * mult, args.steps, args.prime)
         r["label"], r["x_mandatory"] = label, mult
+        if args.evict_exact:
+            e = run_budget(w, mandatory * mult, args.steps, args.prime, evict_exact=1)
+            r["exact"] = {k: e[k] for k in ("hit_ratio", "evicted_pages_per_step", "tokens_per_s", "error_bits")}
         rows.append(r)
         print(json.dumps(r), flush=True)
     base = rows[1]["tokens_per_s"]
@@ -84,6 +91,13 @@ def main():
     for r in rows:
         print(f"| {r['label']} | {r['slots']} | {r['hit_ratio']:.3f} | {r['pcie_mb_per_step']:.2f} | "
               f"{r['ms_per_step']:.3f} | {r['tokens_per_s']:.0f} | {r['tokens_per_s'] / base:.2f}x |")
+    if args.evict_exact:
+        print("\n| budget | hit ratio (paper's eviction) | evicted pages/step | hit ratio (exact demand) | evicted pages/step | tokens/s exact / paper's |")
+        print("|---|---|---|---|---|---|")
+        for r in rows:
+            e = r["exact"]
+            print(f"| {r['label']} | {r['hit_ratio']:.3f} | {r['evicted_pages_per_step']:.1f} | {e['hit_ratio']:.3f} | "
+                  f"{e['evicted_pages_per_step']:.1f} | {e['tokens_per_s'] / r['tokens_per_s']:.2f}x |")
 
 
 if __name__ == "__main__":

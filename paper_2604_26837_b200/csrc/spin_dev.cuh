@@ -109,6 +109,7 @@ struct DevCtx {
   int32_t *n_miss;              // [b] leading descriptors of the page list that may be followed once ready1 is set
   int32_t max_chunks;
   int32_t fetch_mode;           // 0: misses are fetched by the attention kernel; 1: by k_fetch
+  int32_t evict_exact;          // 1: exact-demand eviction variant (see spin_config)
   Counters *counters;
 };
 

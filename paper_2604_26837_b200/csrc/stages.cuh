@@ -356,7 +356,7 @@ struct CacheShared {
   uint32_t hist[kMaxBuckets + 2];
   uint32_t wsum[33];
   int32_t hostpage[512];       // CPU page ids of the first missed pages (looked up early)
-  int x, demand, evicted, qbase, admit_pages, bypass_pages;
+  int x, need, demand, evicted, qbase, admit_pages, bypass_pages;
 };
 
 __host__ __device__ inline size_t cache_stage_smem_bytes(int max_parts, int max_pages, int max_slots) {
@@ -480,19 +480,45 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
 
   // ---- step 3: threshold and eviction; free slots in ascending order --------------------
   if (tid == 0) {
-    int x = -2;                                   // nothing is <= -2: no eviction
+    int x = -2, need = 0x7fffffff;                // nothing is <= -2: no eviction
     if (demand > 0) {
       x = n - 1;
       uint32_t cum = 0;
       for (int bk = -1; bk < n; ++bk) {
         cum += sh.hist[bk + 1];
-        if ((int)cum >= demand) { x = bk; break; }
+        if ((int)cum >= demand) { x = bk; need = demand - (int)(cum - sh.hist[bk + 1]); break; }
       }
     }
     sh.x = x;
+    sh.need = need;                               // pages still missing once every older bucket is gone
   }
   __syncthreads();
   const int x = sh.x;
+  const bool exact = c.evict_exact && demand > 0 && x >= 0;
+  if (exact) {
+    // exact-demand variant: of bucket x only the first `need` pages in slot order are taken;
+    // their partitions are marked non-resident here, and the sweep below takes every page of
+    // bucket x whose partition carries the mark (a partition goes whole)
+    const int need = sh.need;
+    uint32_t seen = 0;
+    for (int base = 0; base < S; base += T) {
+      const int s = base + tid;
+      uint32_t in_x = 0;
+      int part = -1;
+      if (s < S) {
+        const GptEntry *e = gpt_at(c, set, s);
+        if (e && e->partition >= 0 && !((s_hit[s >> 5] >> (s & 31)) & 1u) && e->ts == x) { in_x = 1; part = e->partition; }
+      }
+      uint32_t tot;
+      const uint32_t ex = block_scan<T>(in_x, sh.wsum, &tot);
+      if (in_x && (int)(seen + ex) < need) {
+        MetaEntry *m = meta_at(c, set, part);
+        if (m) m->resident = 0;
+      }
+      seen += tot;
+    }
+    __syncthreads();
+  }
   uint32_t run_free = 0;
   if (demand > 0) {
     for (int base = 0; base < S; base += T) {
@@ -503,7 +529,8 @@ __device__ __forceinline__ void cache_stage(const DevCtx &c, int b, int set, int
         if (e) {
           const int part = e->partition;
           if (part < 0) fr = 1;
-          else if (!((s_hit[s >> 5] >> (s & 31)) & 1u) && e->ts <= x) {
+          else if (!((s_hit[s >> 5] >> (s & 31)) & 1u) && e->ts <= x &&
+                   !(exact && e->ts == x && meta_at(c, set, part) && meta_at(c, set, part)->resident != 0)) {
             MetaEntry *m = meta_at(c, set, part);
             if (m) m->resident = 0;
             if (c.trace) {
@@ -663,7 +690,7 @@ struct FastShared {
   uint32_t wsum[33];
   uint32_t lhist[kMaxBuckets + 2];
   uint32_t prefix, remaining;
-  int x, demand, evicted, qbase, admit_pages, bypass_pages;
+  int x, need, demand, evicted, qbase, admit_pages, bypass_pages;
 };
 
 __host__ __device__ inline size_t fast_smem_bytes(int n_keys, int slots, int dir_part, int dir_slot, int dir_page,
@@ -1160,20 +1187,48 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
   dbg_ts(b, 5);
   // ---- step 3: threshold, eviction, free slots in ascending order (one scan) ----------------
   if (tid == 0) {
-    int x = -2;
+    int x = -2, need = 0x7fffffff;
     if (demand > 0) {
       x = nb - 1;
       uint32_t cum = 0;
 #pragma unroll 1
       for (int bk = -1; bk < nb; ++bk) {
         cum += sh.lhist[bk + 1];
-        if ((int)cum >= demand) { x = bk; break; }
+        if ((int)cum >= demand) { x = bk; need = demand - (int)(cum - sh.lhist[bk + 1]); break; }
       }
     }
     sh.x = x;
+    sh.need = need;                               // pages still missing once every older bucket is gone
   }
   __syncthreads();
   const int x = sh.x;
+  const bool exact = c.evict_exact && demand > 0 && x >= 0;
+  if (exact) {
+    // exact-demand variant (see cache_stage): mark the partitions of the first `need` pages
+    // of bucket x in slot order
+    const int need = sh.need;
+    const int E = (S + T - 1) / T, lo = min(S, tid * E), hi = min(S, lo + E);
+    uint32_t in_x = 0;
+#pragma unroll 1
+    for (int s_ = lo; s_ < hi; ++s_) {
+      const int4 e = s_gpt[s_];
+      in_x += e.x >= 0 && !((s_hit[s_ >> 5] >> (s_ & 31)) & 1u) && e.w == x;
+    }
+    uint32_t tot;
+    uint32_t rank_ = block_scan<T>(in_x, sh.wsum, &tot);
+#pragma unroll 1
+    for (int s_ = lo; s_ < hi; ++s_) {
+      const int4 e = s_gpt[s_];
+      if (e.x >= 0 && !((s_hit[s_ >> 5] >> (s_ & 31)) & 1u) && e.w == x) {
+        if ((int)rank_ < need) {
+          const int seg = s_mdir[e.x >> c.seg_shift];
+          if (seg >= 0) c.meta_pool[((size_t)seg << c.seg_shift) + (e.x & seg_mask)].resident = 0;
+        }
+        ++rank_;
+      }
+    }
+    __syncthreads();
+  }
   dbg_ts(b, 20);
   uint32_t run_free = 0;
   if (demand > 0) {
@@ -1185,6 +1240,8 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
       if (e.x < 0) { ++nfree; continue; }
       if (!((s_hit[s_ >> 5] >> (s_ & 31)) & 1u) && e.w <= x) {
         const int seg = s_mdir[e.x >> c.seg_shift];
+        if (exact && e.w == x && seg >= 0 &&
+            c.meta_pool[((size_t)seg << c.seg_shift) + (e.x & seg_mask)].resident != 0) continue;   // spared
         if (seg >= 0) c.meta_pool[((size_t)seg << c.seg_shift) + (e.x & seg_mask)].resident = 0;
         if (c.trace) {
           c.evict_trace[((size_t)set * c.max_slots + s_) * 2] = e.x;

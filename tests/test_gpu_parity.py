@@ -28,17 +28,19 @@ def _wl(kind, **kw):
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
                one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None,
-               oracle_reqs=None, budget_schedule=None, spare_cache_pages=0):
+               oracle_reqs=None, budget_schedule=None, spare_cache_pages=0, evict_exact=0):
     """oracle_reqs: the requests mirrored in the oracle (default all).  Sets are independent, so the
     oracle run on a sample of the batch's requests must agree with those requests of the full batch."""
     from paper_2604_26837_b200.driver import SpinRun
     dev = "cuda:0"
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
                   segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
-                  cache_pages_per_layer=cache_pages_per_layer, spare_cache_pages=spare_cache_pages)
+                  cache_pages_per_layer=cache_pages_per_layer, spare_cache_pages=spare_cache_pages,
+                  evict_exact=evict_exact)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
-                                      w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale))
+                                      w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale,
+                                      bool(evict_exact)))
     sample = list(range(w.batch)) if oracle_reqs is None else list(oracle_reqs)
     oreq = {r: orc.request_open(run.budgets[r]) for r in sample}
     for r in range(w.batch):
@@ -276,6 +278,21 @@ def test_cluster_centroid_tight_budget_with_empty_clusters():
     w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=300, topk=20, slots_per_set=12,
             context=400, steps=20, max_partition_pages=4, batch=1)
     run_parity(w)
+
+
+def test_exact_demand_eviction_variant():
+    # the variant that evicts only what the misses need (not the paper's rule): both cache
+    # managers (shared-memory copy; page table in global memory), single- and multi-page partitions
+    w = _wl(W.PART_PAGE_MINMAX, steps=40, lru_buckets=4, drift=0.4)
+    r = run_parity(w, evict_exact=1)
+    ref = run_parity(w)
+    assert 0 < r["stats"]["evicted_pages"] < ref["stats"]["evicted_pages"]
+    w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=37, topk=5, slots_per_set=30,
+            context=16 * 50 + 3, steps=40, max_partition_pages=8, lru_buckets=3)
+    run_parity(w, evict_exact=1)
+    w = _wl(W.PART_PAGE_MINMAX, context=16 * 1300 + 3, slots_per_set=1100, topk=40, steps=36, batch=1,
+            num_layers=1, lru_buckets=4, drift=0.4)
+    run_parity(w, check_bytes=False, one_call=True, evict_exact=1)
 
 
 def test_tiny_configuration_full_size():
