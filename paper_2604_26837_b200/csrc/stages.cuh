@@ -921,6 +921,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
           if ((key & mask) == prefix) atomicAdd(&L.s_hist[(key >> shift) & dmask], 1u);
         }
         __syncthreads();
+        dbg_ts(b, 16);
         uint32_t loc[kPer], sum = 0;                               // this thread's bins, best first
 #pragma unroll
         for (int j = 0; j < kPer; ++j) { loc[j] = L.s_hist[kFastBins - 1 - kPer * tid - j]; sum += loc[j]; }
@@ -940,6 +941,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
           }
         }
         __syncthreads();
+        dbg_ts(b, 30);
         prefix = sh.prefix;
         remaining = sh.remaining;
         mask |= dmask << shift;
