@@ -1360,6 +1360,8 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     c.n_pages[b] = total_pages + tail_pages;
     c.n_parts[b] = np;
     c.state[set].step = t + 1;
+    flag_publish(c.ready + b, bt.epoch);
+    // the counters go last: the flag's fence should not have to wait for them
     Counters *kc = c.counters;
     const int miss_pages = sh.admit_pages + sh.bypass_pages;
     atomicAdd(&kc->set_steps, 1ull);
@@ -1370,7 +1372,6 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
     atomicAdd(&kc->miss_pages, (unsigned long long)miss_pages);
     atomicAdd(&kc->evicted_pages, (unsigned long long)sh.evicted);
     atomicAdd(&kc->bypass_pages, (unsigned long long)sh.bypass_pages);
-    flag_publish(c.ready + b, bt.epoch);
   }
   // ---- the page table goes back in one sweep; attention does not wait for it -----------------
 #pragma unroll 1

@@ -295,6 +295,20 @@ def test_exact_demand_eviction_variant():
     run_parity(w, check_bytes=False, one_call=True, evict_exact=1)
 
 
+def test_token_dot_more_keys_than_one_cta_holds():
+    # > 16384 candidate keys per set: scoring, then one thread-block cluster per set for the
+    # top-k (ragged slices: 20800 keys over 4 CTAs), which starts on the set's scored flag and
+    # whose first CTA goes on as the cache manager; and the same with more slots than the
+    # shared-memory cache manager takes, so that the cluster only selects and k_cache follows
+    w = _wl(W.PART_TOKEN_DOT, context=16 * 1300 + 5, topk=300, slots_per_set=120, steps=20, batch=2,
+            num_layers=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8, drift=0.3, kv_recipe="page_centre", centre_sd=0.5)
+    r = run_parity(w, check_bytes=False, one_call=True)
+    assert r["stats"]["evicted_pages"] > 0
+    w = _wl(W.PART_TOKEN_DOT, context=16 * 1300 + 5, topk=300, slots_per_set=1100, steps=6, batch=1,
+            num_layers=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8, drift=0.3, kv_recipe="page_centre", centre_sd=0.5)
+    run_parity(w, check_bytes=False, one_call=True)
+
+
 def test_tiny_configuration_full_size():
     # the first benchmark configuration as stated: 4096-token context, top-16, 64 slots, 8 buckets
     r = run_parity(W.CONFIGS["c1"], check_bytes=False, one_call=True)
