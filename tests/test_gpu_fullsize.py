@@ -33,3 +33,17 @@ def test_c4_cluster_granular_full_size_sampled_request():
     w = W.scaled(W.CONFIGS["c4"], steps=8, batch=4)  # 4 of the 16 requests: 131072 tokens, 1024 clusters each
     r = run_parity(w, one_call=True, check_bytes=False, oracle_reqs=[2])
     assert r["stats"]["miss_pages"] > 0
+
+
+def test_c5_mixed_batch_scaled_sampled_requests():
+    # the mixed-length configuration as the benchmark scales it to one box: 16 of the 64 requests,
+    # 1 of the 32 layers, contexts drawn from U[8192, 262144], per-request drift, and the same
+    # per-layer share of the 60 GB budget split in proportion to sequence length
+    w = W.scaled(W.CONFIGS["c5"], batch=16, num_layers=1, steps=6)
+    pages_per_layer = int(60e9 / 32 / 8192 * 16 / 64)
+    from paper_2604_26837_b200.driver import context_sizes
+    ctx = context_sizes(w)
+    longest, shortest = max(range(16), key=lambda r: ctx[r]), min(range(16), key=lambda r: ctx[r])
+    r = run_parity(w, one_call=True, check_bytes=False, cache_pages_per_layer=pages_per_layer,
+                   oracle_reqs=sorted({longest, shortest}))
+    assert r["stats"]["miss_pages"] > 0 and r["stats"]["set_steps"] == 16 * 8 * 6
