@@ -111,6 +111,16 @@ typedef struct spin_config {
                                    what that over-eviction costs: of the threshold bucket only
                                    as many pages as the misses still need are taken, lowest
                                    slots first (a partition that loses a page goes whole) */
+  int64_t offload_stage_bytes;  /* 0: appended pages are written through to pinned host memory on
+                                   the caller's stream (Offload, Section 4.1).  > 0: asynchronous
+                                   offload: the complete pages of an append from device memory are
+                                   indexed and copied into a staging ring of this many bytes of
+                                   the HBM pool on the caller's stream (HBM speed), and move to
+                                   host memory on a stream of the library's own; the caller's
+                                   stream goes on at once (it waits only when the ring is full),
+                                   and a later decode step waits for the pages it may fetch.
+                                   Page / token / page-mean granularity; at least 4 pages of
+                                   every kv head must fit (4 x 8 KiB x num_kv_heads x 4 bytes) */
   int64_t gpu_cache_pages;      /* HBM pages (8 KiB each) shared by all sets' cache slots */
   int64_t host_pages;           /* pinned host pages (8 KiB each) for the complete KV */
   void *hbm_pool;               /* device pointer, 256-byte aligned, caller-owned */

@@ -94,6 +94,9 @@ int compute_geometry(const spin_config &cfg, Geometry &g, std::string &err) {
   if (cfg.topk < 1 || cfg.topk > 4096) return bad("topk must be 1..4096");
   if (cfg.lru_buckets < 1 || cfg.lru_buckets > kMaxBuckets) return bad("lru_buckets must be 1..64");
   if (cfg.gpu_cache_pages < 0 || cfg.host_pages < 1) return bad("bad page counts");
+  if (cfg.offload_stage_bytes < 0 || (cfg.offload_stage_bytes > 0 &&
+      cfg.offload_stage_bytes / 4 / kPageBytes < cfg.num_kv_heads))
+    return bad("offload_stage_bytes must be 0 or hold at least 4 pages of every kv head");
   const bool cluster = cfg.partition_kind == SPIN_PART_CLUSTER_CENTROID;
   if (cluster && cfg.num_clusters < 1) return bad("num_clusters must be >= 1 for the cluster kind");
   g.seg = cfg.segment_entries ? cfg.segment_entries : 256;
@@ -172,6 +175,18 @@ struct spin_ctx {
   size_t dir_bytes_in_use = 0;
   Prof prof;
   int32_t epoch = 0;                 // decode calls so far (value of the per-set ready flags)
+  // asynchronous offload: a ring of kOffloadSlots staging slots in HBM, drained by copy-engine
+  // transfers on offload_stream; slot i is free again once ev_done[i] has happened
+  static constexpr int kOffloadSlots = 4;
+  uint8_t *offload_stage = nullptr;
+  int32_t *offload_hp = nullptr;     // per staged unit: its host page id (what the kernel records in the mirror)
+  int64_t offload_slot_units = 0;    // (page, kv head) units of 8 KiB per slot; 0 = write-through
+  cudaStream_t offload_stream = nullptr;
+  cudaEvent_t ev_staged[kOffloadSlots] = {}, ev_done[kOffloadSlots] = {};
+  bool slot_used[kOffloadSlots] = {};
+  int offload_next = 0, offload_last = -1;
+  uint64_t offload_gen = 0, offload_waited_gen = 0;
+  cudaStream_t offload_waited_stream = nullptr;
 };
 
 namespace {
@@ -245,6 +260,12 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   __nv_bfloat16 *sv = a.take<__nv_bfloat16>(stage_rows * kHeadDim);
   int64_t *sd = a.take<int64_t>(stage_rows);
   if (ctx) { ctx->stage_q = sq; ctx->stage_out = so; ctx->stage_k = sk; ctx->stage_v = sv; ctx->stage_dest = sd; }
+  if (cfg.offload_stage_bytes > 0) {
+    const int64_t units = cfg.offload_stage_bytes / spin_ctx::kOffloadSlots / kPageBytes;
+    uint8_t *os = a.take<uint8_t>((size_t)units * spin_ctx::kOffloadSlots * kPageBytes);
+    int32_t *oh = a.take<int32_t>((size_t)units * spin_ctx::kOffloadSlots);
+    if (ctx) { ctx->offload_stage = os; ctx->offload_hp = oh; ctx->offload_slot_units = units; }
+  }
 }
 
 size_t host_bytes_needed(const Geometry &g, const spin_config &cfg) {
@@ -373,6 +394,18 @@ int grow_cluster_tail(spin_ctx *ctx, int req, int layer, int64_t n_new, cudaStre
   return SPIN_OK;
 }
 
+// Pages still on their way to host memory must have arrived before `st` reads the host tier
+// (a decode step's fetch) or hands host pages back (request close).  The library's stream is
+// in order, so the newest drain event covers all earlier ones.
+int wait_for_offload(spin_ctx *ctx, cudaStream_t st) {
+  if (ctx->offload_last < 0) return SPIN_OK;
+  if (ctx->offload_gen == ctx->offload_waited_gen && st == ctx->offload_waited_stream) return SPIN_OK;
+  CK(cudaStreamWaitEvent(st, ctx->ev_done[ctx->offload_last], 0));
+  ctx->offload_waited_gen = ctx->offload_gen;
+  ctx->offload_waited_stream = st;
+  return SPIN_OK;
+}
+
 int append_paged_device(spin_ctx *ctx, int req, int layer, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         int64_t n, cudaStream_t st) {
   LayerHost &L = ctx->reqs[(size_t)req].layers[(size_t)layer];
@@ -382,7 +415,53 @@ int append_paged_device(spin_ctx *ctx, int req, int layer, const __nv_bfloat16 *
   if (rc) return rc;
   const int64_t j_end = (n0 + n - 1) / kPageTokens;
   // pages strictly between the old tail page and the newest page: complete, all rows new
-  ctx->launches += launch_append_bulk(ctx->d, req, layer, k, v, (int)(j0 + 1), (int)(j_end - (j0 + 1)), (int)n0, st, &ctx->prof);
+  const int64_t first = j0 + 1, nb = j_end - first;
+  if (ctx->offload_slot_units > 0 && nb > 0) {
+    // asynchronous offload: slot by slot through the staging ring (see spin_ctx)
+    const int64_t per = ctx->offload_slot_units / ctx->cfg.num_kv_heads;
+    for (int64_t p = 0; p < nb; p += per) {
+      const int m = (int)std::min<int64_t>(per, nb - p), slot = ctx->offload_next;
+      ctx->offload_next = (slot + 1) % spin_ctx::kOffloadSlots;
+      if (ctx->slot_used[slot]) CK(cudaStreamWaitEvent(st, ctx->ev_done[slot], 0));     // ring full: wait for the drain
+      uint8_t *stage = ctx->offload_stage + (size_t)slot * ctx->offload_slot_units * kPageBytes;
+      int32_t *hp = ctx->offload_hp + (size_t)slot * ctx->offload_slot_units;
+      {
+        // the pages' host ids come with the call (head-major like the slot): while copy-engine
+        // transfers own the host link, a kernel's small reads of the pinned CPU page table
+        // would wait behind them
+        std::vector<int32_t> ids((size_t)m * ctx->cfg.num_kv_heads);
+        for (int h = 0; h < ctx->cfg.num_kv_heads; ++h) {
+          const std::vector<int32_t> &hpv = set_of(ctx, req, layer, h).host_pages;
+          for (int i = 0; i < m; ++i) ids[(size_t)h * m + i] = hpv[(size_t)(first + p + i)];
+        }
+        CK(cudaMemcpyAsync(hp, ids.data(), ids.size() * 4, cudaMemcpyHostToDevice, st));   // pageable source: staged before the call returns
+      }
+      ctx->launches += launch_append_bulk(ctx->d, req, layer, k, v, (int)(first + p), m, (int)n0, st, &ctx->prof, stage, hp);
+      CK(cudaEventRecord(ctx->ev_staged[slot], st));
+      CK(cudaStreamWaitEvent(ctx->offload_stream, ctx->ev_staged[slot], 0));
+      // The slot is laid out head-major, the order in which host pages were handed out, so a
+      // head's pages are as a rule one run of consecutive host pages: one copy-engine transfer
+      // per run, no SM involved (a fragmented host pool means more and shorter transfers).
+      const int H = ctx->cfg.num_kv_heads;
+      for (int h = 0; h < H; ++h) {
+        const std::vector<int32_t> &hpv = set_of(ctx, req, layer, h).host_pages;
+        for (int i = 0; i < m;) {
+          int len = 1;
+          while (i + len < m && hpv[(size_t)(first + p + i + len)] == hpv[(size_t)(first + p + i)] + len) ++len;
+          CK(cudaMemcpyAsync(ctx->h_pages + (size_t)hpv[(size_t)(first + p + i)] * kPageBytes,
+                             stage + ((size_t)h * m + i) * kPageBytes, (size_t)len * kPageBytes,
+                             cudaMemcpyDeviceToHost, ctx->offload_stream));
+          i += len;
+        }
+      }
+      CK(cudaEventRecord(ctx->ev_done[slot], ctx->offload_stream));
+      ctx->slot_used[slot] = true;
+      ctx->offload_last = slot;
+      ++ctx->offload_gen;
+    }
+  } else {
+    ctx->launches += launch_append_bulk(ctx->d, req, layer, k, v, (int)first, (int)nb, (int)n0, st, &ctx->prof);
+  }
   AppendEdgeArgs a{};
   a.n_req = 1;
   a.layer = layer;
@@ -680,6 +759,13 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   fill(d.n_sel, 0, (size_t)g.max_batch_sets * 4);
   if (d.evict_trace) fill(d.evict_trace, 0xff, (size_t)g.n_sets * g.max_slots * 8);
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail("cudaDeviceSynchronize", e);
+  if (ctx->offload_slot_units > 0) {
+    if ((e = cudaStreamCreateWithFlags(&ctx->offload_stream, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail("cudaStreamCreateWithFlags", e);
+    for (int i = 0; i < spin_ctx::kOffloadSlots; ++i) {
+      if ((e = cudaEventCreateWithFlags(&ctx->ev_staged[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail("cudaEventCreateWithFlags", e);
+      if ((e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail("cudaEventCreateWithFlags", e);
+    }
+  }
 
   ctx->gpu_page_pool.init(cfg->gpu_cache_pages);
   ctx->host_page_pool.init(cfg->host_pages);
@@ -701,6 +787,10 @@ int spin_destroy(spin_ctx *ctx) {
     for (size_t i = 0; i < Prof::kMaxMarks; ++i) cudaEventDestroy(ctx->prof.ev[i]);
     delete[] ctx->prof.ev;
     delete[] ctx->prof.id;
+  }
+  if (ctx->offload_stream) {
+    for (int i = 0; i < spin_ctx::kOffloadSlots; ++i) { cudaEventDestroy(ctx->ev_staged[i]); cudaEventDestroy(ctx->ev_done[i]); }
+    cudaStreamDestroy(ctx->offload_stream);
   }
   if (ctx->host_base) cudaFreeHost(ctx->host_base);
   delete ctx;
@@ -771,6 +861,7 @@ int spin_request_close(spin_ctx *ctx, int32_t req) {
   if (!R.open) return fail(ctx, SPIN_ERR_STATE, "request %d is not open", req);
   const Geometry &g = ctx->g;
   const DevCtx &d = ctx->d;
+  if (ctx->offload_stream) CK(cudaStreamSynchronize(ctx->offload_stream));   // its pages may still be on their way
   for (int l = 0; l < ctx->cfg.num_layers; ++l)
     for (int h = 0; h < ctx->cfg.num_kv_heads; ++h) {
       const int set = set_index(d, req, l, h);
@@ -967,6 +1058,7 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
   bool in_grid = false, kv_pinned = false;
   // q and new k/v in pinned host memory: one zero-copy staging kernel brings them in
+  if (int rc = wait_for_offload(ctx, st)) return rc;       // missed pages are fetched from the host tier
   const int qc = classify_ptr(q, &q_alias), oc = classify_ptr(out, &out_alias);
   if (with_append) {
     for (int i = 0; i < n_req; ++i) {

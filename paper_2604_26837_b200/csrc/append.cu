@@ -14,7 +14,8 @@ namespace {
 // come from the input; the page is written to the host tier and indexed.
 __global__ void __launch_bounds__(256)
 k_append_bulk(DevCtx c, int req, int layer, const __nv_bfloat16 *__restrict__ k,
-              const __nv_bfloat16 *__restrict__ v, int first_page, int first_token_of_call) {
+              const __nv_bfloat16 *__restrict__ v, int first_page, int first_token_of_call,
+              uint8_t *__restrict__ stage, const int32_t *__restrict__ stage_hp) {
   __shared__ __align__(16) __nv_bfloat16 krows[kPageTokens][kHeadDim];
   const int head = blockIdx.y, page = first_page + blockIdx.x, tid = threadIdx.x;
   const int set = set_index(c, req, layer, head);
@@ -23,11 +24,20 @@ k_append_bulk(DevCtx c, int req, int layer, const __nv_bfloat16 *__restrict__ k,
   const size_t in_off = (tok * c.Hkv + head) * kHeadDim * 2 + piece * 16;
   uint4 kk = ld16(reinterpret_cast<const uint8_t *>(k) + in_off);
   uint4 vv = ld16(reinterpret_cast<const uint8_t *>(v) + in_off);
-  const int32_t *hp = cpt_at(c, set, page);
-  if (!hp) { if (tid == 0) dev_error(c, 1u); return; }
-  const int32_t host_page = *hp;
+  const size_t unit = (size_t)head * gridDim.x + blockIdx.x;        // head-major, as host pages are handed out
+  int32_t host_page;
+  if (stage) {
+    host_page = stage_hp[unit];
+  } else {
+    const int32_t *hp = cpt_at(c, set, page);
+    if (!hp) { if (tid == 0) dev_error(c, 1u); return; }
+    host_page = *hp;
+  }
   if (tid == 0) cpt_mirror_set(c, set, page, host_page);
+  // Offload: straight to the page's place in pinned host memory, or -- asynchronous offload --
+  // into an HBM staging slot from which copy-engine transfers move it on the library's own stream
   uint8_t *dst = c.host_pages + (size_t)host_page * kPageBytes + r * kRowBytes + piece * 16;
+  if (stage) dst = stage + unit * kPageBytes + r * kRowBytes + piece * 16;
   st16(dst, kk);
   st16(dst + kHalfPageBytes, vv);
   st16(reinterpret_cast<uint8_t *>(krows[r]) + piece * 16, kk);
@@ -104,9 +114,9 @@ int launch_stage_in(void *dq, const void *sq, size_t q_bytes, void *dk, const vo
 
 int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,
-                       cudaStream_t st, Prof *prof) {
+                       cudaStream_t st, Prof *prof, uint8_t *stage, const int32_t *stage_hp) {
   if (n_pages <= 0) return 0;
-  k_append_bulk<<<dim3(n_pages, c.Hkv), 256, 0, st>>>(c, req, layer, k, v, first_page, first_token_of_call);
+  k_append_bulk<<<dim3(n_pages, c.Hkv), 256, 0, st>>>(c, req, layer, k, v, first_page, first_token_of_call, stage, stage_hp);
   prof_mark(prof, st, kProfAppend);
   return 1;
 }

@@ -274,7 +274,7 @@ struct AppendEdgeArgs {     // one (request) per entry; all its kv heads are pro
 };
 int launch_append_bulk(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int first_page, int n_pages, int first_token_of_call,
-                       cudaStream_t st, Prof *prof);
+                       cudaStream_t st, Prof *prof, uint8_t *stage = nullptr, const int32_t *stage_hp = nullptr);
 int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bfloat16 *k,
                        const __nv_bfloat16 *v, int n_new, cudaStream_t st, Prof *prof);
 int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,

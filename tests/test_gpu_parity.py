@@ -28,7 +28,8 @@ def _wl(kind, **kw):
 
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
                one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None,
-               oracle_reqs=None, budget_schedule=None, spare_cache_pages=0, evict_exact=0):
+               oracle_reqs=None, budget_schedule=None, spare_cache_pages=0, evict_exact=0,
+               offload_stage_bytes=0):
     """oracle_reqs: the requests mirrored in the oracle (default all).  Sets are independent, so the
     oracle run on a sample of the batch's requests must agree with those requests of the full batch."""
     from paper_2604_26837_b200.driver import SpinRun
@@ -36,7 +37,7 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
                   segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
                   cache_pages_per_layer=cache_pages_per_layer, spare_cache_pages=spare_cache_pages,
-                  evict_exact=evict_exact)
+                  evict_exact=evict_exact, offload_stage_bytes=offload_stage_bytes)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale,
@@ -307,6 +308,16 @@ def test_token_dot_more_keys_than_one_cta_holds():
     w = _wl(W.PART_TOKEN_DOT, context=16 * 1300 + 5, topk=300, slots_per_set=1100, steps=6, batch=1,
             num_layers=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8, drift=0.3, kv_recipe="page_centre", centre_sd=0.5)
     run_parity(w, check_bytes=False, one_call=True)
+
+
+@pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_TOKEN_DOT])
+def test_asynchronous_offload_of_prefill_pages(kind):
+    # prefill pages go through a staging ring (4 slots x 3 pages x 2 kv heads here, so a
+    # 40-page prefill wraps the ring several times) and reach host memory on the library's own
+    # stream; the first decode step waits for them; results and host bytes as without it
+    w = _wl(kind, topk=6 if kind == W.PART_PAGE_MINMAX else 64, steps=12)
+    r = run_parity(w, offload_stage_bytes=4 * 3 * 2 * 8192, check_bytes=True)
+    assert r["stats"]["miss_pages"] > 0
 
 
 def test_tiny_configuration_full_size():
