@@ -208,7 +208,8 @@ __device__ __forceinline__ void pdl_wait_prev() { asm volatile("griddepcontrol.w
 // ever waits for work that is already running.  The wait is bounded all the same: it gives up
 // after ~0.1 s, reports SPIN_DEV_ERR_TIMEOUT and the CTA returns without touching the set.
 __device__ __forceinline__ void flag_publish(int32_t *flag, int32_t value) {
-  __threadfence();
+  // a release store: everything this thread has written or observed (through the CTA barrier
+  // before the call: the other threads' writes too) is visible to whoever acquires the flag
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
 __device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, int32_t value) {
