@@ -247,6 +247,8 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.att_part = a.take<float>(B * g.max_chunks * G * (kHeadDim + 2));
   d.att_count = a.take<int32_t>(B);
   d.sel_count = a.take<int32_t>(B);
+  d.score_queue = a.take<int32_t>(1);
+  d.score_done = a.take<int32_t>(1);
   d.scored = a.take<int32_t>(B);
   d.ready = a.take<int32_t>(B);
   d.tail_ready = a.take<int32_t>(B);
@@ -746,6 +748,8 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   memset(ctx->host_base, 0, ctx->host_bytes);
   fill(d.att_count, 0, (size_t)g.max_batch_sets * 4);
   fill(d.sel_count, 0, (size_t)g.max_batch_sets * 4);
+  fill(d.score_queue, 0, 4);
+  fill(d.score_done, 0, 4);
   fill(d.scored, 0, (size_t)g.max_batch_sets * 4);
   fill(d.ready, 0, (size_t)g.max_batch_sets * 4);
   fill(d.tail_ready, 0, (size_t)g.max_batch_sets * 4);

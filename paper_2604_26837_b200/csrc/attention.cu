@@ -176,7 +176,8 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
                                          __nv_bfloat16 *__restrict__ out, uint8_t *smem_pages) {
   __shared__ float sh[kAttnWarps][G][kPartStride];
   __shared__ int sh_last;
-  const int b = blockIdx.x, chunk = blockIdx.y;       // chunk-major launch order: chunk 0 of every set first
+  // launch order: chunk 0 of every set first (the chunks that hold the missed pages), or set by set
+  const int b = bt.attn_set_major ? blockIdx.y : blockIdx.x, chunk = bt.attn_set_major ? blockIdx.x : blockIdx.y;
   const int first = chunk * kChunkPages;
   bool slots_known = true;                 // false: the chunk holds early descriptors only
   if (c.ready) {
@@ -425,6 +426,7 @@ int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
   if (chunks < 1) chunks = 1;
   if (chunks > c.max_chunks) chunks = c.max_chunks;
   dim3 grid(n_sets, chunks);
+  if (b.attn_set_major) grid = dim3(chunks, n_sets);
   int launched = 1;
   if (may_be_empty) { k_attn_zero_empty<<<n_sets, 128, 0, st>>>(c, out, n_sets); ++launched; }
   switch (c.G) {

@@ -99,17 +99,24 @@ __device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, con
   return tot + 0.0f;                              // -0.0 -> +0.0
 }
 
+// How the scoring kernel cuts a step into work items.  Items run in this order: the sets' tail
+// items (one per set: in-grid append, tail flag), then request by request, head by head, the
+// summary segments of each set (as many as that request has: mixed lengths cost no idle items).
+struct ScoreGrid {
+  int32_t n_sets, n_items;
+  int32_t persistent;                  // 1: a resident grid draws items from a queue; 0: item = blockIdx.x
+  int32_t item_prefix[kMaxBatch + 1];  // first segment item of each request (all its heads follow)
+};
+
+// One work item (uniform over the CTA): x < 0 is the tail item of batch set b, else summary
+// segment x of that set.
 template <int G, bool MINMAX>
-__global__ void __launch_bounds__(kScoreThreads, 3)
-k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
-        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap, int tbl_cap) {   // fuse: 0 none, 1 staged, 2 fast, 3 flag only
-  extern __shared__ __align__(16) uint8_t dyn_smem[];      // used by the fused continuation only
-  const int b = blockIdx.y, i_req = b / c.Hkv, head = b % c.Hkv;
+__device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, const __nv_bfloat16 *__restrict__ q,
+                                           const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
+                                           int fuse, int keys_cap, int tbl_cap, int b, int x, uint8_t *dyn_smem) {
+  const int i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
-  pdl_launch_next();
-  pdl_wait_prev();
-  if (blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *c.fetch_count = 0;   // new step, new miss queue
-  if (blockIdx.x == gridDim.x - 1) {
+  if (x < 0) {
     // the set's tail CTA: appends this step's token (unless a stand-alone append already ran)
     // and tells the attention kernel that the tail page is complete
     __shared__ __align__(16) __nv_bfloat16 krows[kPageTokens][kHeadDim];
@@ -118,17 +125,17 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
     if (threadIdx.x == 0) flag_publish(c.tail_ready + b, bt.epoch);
     return;
   }
-  if (blockIdx.x == 0) dbg_ts(b, 0);
+  if (x == 0) dbg_ts(b, 0);
   // the host's count: the in-grid append never completes a page, so it equals the set's state
   const int n_partitions = bt.n_partitions[i_req];
   const int n_cand = c.kind == kKindToken ? n_partitions * kPageTokens : n_partitions;
   const int seg_entries = 1 << c.sum_shift;
-  const int e0 = blockIdx.x * seg_entries;
+  const int e0 = x * seg_entries;
   // the CTAs that count towards the set's arrival counter: one per non-empty segment, and
   // segment 0 even when the set has no candidate yet
   const int segs_here = max(1, (n_cand + seg_entries - 1) >> c.sum_shift);
-  if ((int)blockIdx.x >= segs_here) return;
-  const int seg = e0 < n_cand ? c.dir_sumseg[(size_t)set * c.dir_sum + blockIdx.x] : 0;
+  if (x >= segs_here) return;
+  const int seg = e0 < n_cand ? c.dir_sumseg[(size_t)set * c.dir_sum + x] : 0;
   if (seg < 0 && threadIdx.x == 0) dev_error(c, kErrBounds);
   if (e0 < n_cand && seg >= 0) {
   const int lane16 = threadIdx.x & 15, grp = threadIdx.x >> 4;
@@ -217,6 +224,57 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
                              bt.epoch, reinterpret_cast<int32_t *>(dyn_smem), shm.staged.c);
 }
 
+// The scoring kernel: one work item per CTA, or -- when scoring is long (many more items than
+// CTAs fit on the GPU) and the sets' selection continues in this kernel -- a grid that is
+// resident all at once and draws its items from a queue.  A dependent grid is launched once
+// every CTA of this one has started: with thousands of one-item CTAs that is most of the way
+// through scoring, and the host link would idle until then although the first sets' missed
+// pages have long been listed.  The resident form starts all its CTAs at once and leaves room
+// on some SMs, so attention CTAs move in from the beginning.
+template <int G, bool MINMAX>
+__global__ void __launch_bounds__(kScoreThreads, 3)
+k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
+        const __nv_bfloat16 *__restrict__ v_new, int fuse, int keys_cap, int tbl_cap, ScoreGrid sg) {   // fuse: 0 none, 1 staged, 2 fast, 3 flag only
+  extern __shared__ __align__(16) uint8_t dyn_smem[];      // staging area; reused by the fused continuation
+  pdl_launch_next();
+  pdl_wait_prev();
+  __shared__ int s_item[2];
+  const bool pers = sg.persistent != 0;
+  if (pers) {
+    if (threadIdx.x == 0) s_item[0] = atomicAdd(c.score_queue, 1);
+    __syncthreads();
+  }
+  for (int it = 0;; ++it) {
+    const int item = pers ? s_item[it & 1] : (int)blockIdx.x;
+    if (item >= sg.n_items) break;
+    int next = 0;
+    if (pers && threadIdx.x == 0) next = atomicAdd(c.score_queue, 1);   // in flight while this item is worked on
+    if (item == 0 && threadIdx.x == 0) *c.fetch_count = 0;               // new step, new miss queue
+    int b = item, x = -1;                                                // the sets' tail items come first
+    if (item >= sg.n_sets) {
+      const int id = item - sg.n_sets;
+      int lo = 0, hi = bt.n_req;                                         // request whose items hold `id`
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (sg.item_prefix[mid] <= id) lo = mid; else hi = mid;
+      }
+      const int segs_r = (sg.item_prefix[lo + 1] - sg.item_prefix[lo]) / c.Hkv, off = id - sg.item_prefix[lo];
+      b = lo * c.Hkv + off / segs_r;
+      x = off % segs_r;
+    }
+    score_item<G, MINMAX>(c, bt, q, k_new, v_new, fuse, keys_cap, tbl_cap, b, x, dyn_smem);
+    if (!pers) return;
+    if (threadIdx.x == 0) s_item[(it + 1) & 1] = next;
+    __syncthreads();
+  }
+  // the last CTA out leaves the queue ready for the next step (every other CTA has drawn its
+  // last item by then)
+  if (pers && threadIdx.x == 0 && atomicAdd(c.score_done, 1) == (int)gridDim.x - 1) {
+    *c.score_queue = 0;
+    *c.score_done = 0;
+  }
+}
+
 // Stand-alone top-k: one thread-block cluster per set (slices of the keys in shared memory).
 // With wait_flags a cluster starts as soon as its own set is scored (the flag the scoring
 // kernel's last CTA of that set raises) instead of when the whole scoring kernel is done; the
@@ -273,28 +331,54 @@ k_topk(DevCtx c, Batch bt, int keys_cap, int manage, int tbl_cap, int wait_flags
 }
 
 
+int sm_count_of_device() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
 template <int G>
 void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
-                    const __nv_bfloat16 *v_new, dim3 grid, size_t smem, int fuse, int keys_cap, int tbl_cap, cudaStream_t st) {
+                    const __nv_bfloat16 *v_new, dim3 grid, size_t smem, int fuse, int keys_cap, int tbl_cap,
+                    const ScoreGrid &sg, cudaStream_t st) {
   static size_t configured = 0;
   if (smem > configured) {
     cudaFuncSetAttribute(k_score<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     cudaFuncSetAttribute(k_score<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap, tbl_cap);
-  else launch_pdl(k_score<G, false>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap, tbl_cap);
+  if (sg.persistent) {
+    // the resident grid: what fits on the GPU at this shared-memory size, less one CTA on 32
+    // SMs (attention CTAs take that room from the start)
+    static size_t occ_smem = ~(size_t)0;
+    static int occ[2] = {1, 1};
+    if (smem != occ_smem) {
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ[1], k_score<G, true>, kScoreThreads, smem);
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ[0], k_score<G, false>, kScoreThreads, smem);
+      occ_smem = smem;
+    }
+    const int sms = sm_count_of_device(), per_sm = occ[c.kind == kKindPage ? 1 : 0] < 1 ? 1 : occ[c.kind == kKindPage ? 1 : 0];
+    int resident = per_sm * sms - (per_sm > 1 ? 32 : 0);
+    if (resident > sg.n_items) resident = sg.n_items;
+    grid = dim3(resident);
+  }
+  if (c.kind == kKindPage) launch_pdl(k_score<G, true>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap, tbl_cap, sg);
+  else launch_pdl(k_score<G, false>, grid, dim3(kScoreThreads), smem, st, 1, c, b, q, k_new, v_new, fuse, keys_cap, tbl_cap, sg);
 }
 
 }  // namespace
 
 // Select + (fused or separate) cache management.  Returns the kernels launched.
-int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
+int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
                   const __nv_bfloat16 *v_new, int max_cand, cudaStream_t st, Prof *prof) {
   const int n_sets = b.n_req * c.Hkv;
   int segs = (max_cand + (1 << c.sum_shift) - 1) >> c.sum_shift;
   if (segs < 1) segs = 1;                         // segment 0 always runs (arrival counter, miss-queue reset)
-  dim3 grid(segs + 1, n_sets);                    // + one tail CTA per set (in-grid append, tail flag)
   // fused: one CTA can hold a set's keys and the cache manager's tables in shared memory
   const size_t cache_smem = cache_stage_smem_bytes(c.max_parts, c.max_pages, c.max_slots);
   int fuse = (max_cand <= 16384 && cache_smem <= 96 * 1024) ? 1 : 0;
@@ -326,11 +410,27 @@ int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const
   size_t mgr_smem = 0;
   const int manage = !fuse && plan_cache_fast(c, b, 160 * 1024, &mgr_tbl_cap, &mgr_smem) ? 1 : 0;
   if (manage) fuse = 3;
+  // work items: a tail item per set, then every request's segments head by head (segment 0
+  // always runs: arrival counter)
+  ScoreGrid sg;
+  sg.n_sets = n_sets;
+  sg.item_prefix[0] = 0;
+  for (int i = 0; i < b.n_req; ++i) {
+    const int cand = c.kind == kKindToken ? b.n_partitions[i] * kPageTokens : b.n_partitions[i];
+    int segs_r = (cand + (1 << c.sum_shift) - 1) >> c.sum_shift;
+    if (segs_r < 1) segs_r = 1;
+    sg.item_prefix[i + 1] = sg.item_prefix[i] + segs_r * c.Hkv;
+  }
+  sg.n_items = n_sets + sg.item_prefix[b.n_req];
+  // resident form (grid sized in launch_score_g) when scoring is many waves long
+  sg.persistent = (fuse == 2 && c.ready && sg.n_items > 12 * sm_count_of_device()) ? 1 : 0;
+  dim3 grid(sg.n_items);
+  b.attn_set_major = sg.persistent;
   switch (c.G) {
-    case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
-    case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
-    case 4: launch_score_g<4>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
-    default: launch_score_g<8>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, st); break;
+    case 1: launch_score_g<1>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, sg, st); break;
+    case 2: launch_score_g<2>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, sg, st); break;
+    case 4: launch_score_g<4>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, sg, st); break;
+    default: launch_score_g<8>(c, b, q, k_new, v_new, grid, smem, fuse, keys_cap, tbl_cap, sg, st); break;
   }
   prof_mark(prof, st, kProfScore);
   if (fuse == 1 || fuse == 2) return 1;

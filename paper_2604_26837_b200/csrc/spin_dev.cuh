@@ -102,6 +102,8 @@ struct DevCtx {
   float *att_part;              // split-K partials [b][max_chunks][G][kHeadDim + 2]
   int32_t *att_count;           // [b] chunks of the set that have finished (zero before attention)
   int32_t *sel_count;           // [b] scoring CTAs of the set that have finished (zero between steps)
+  int32_t *score_queue;         // next work item of the resident scoring grid (zero between steps)
+  int32_t *score_done;          // CTAs of that grid that have left (zero between steps)
   int32_t *scored;              // [b] epoch of the last step whose scores are complete (stand-alone top-k waits on it)
   int32_t *ready;               // [b] epoch of the last step whose page list is complete
   int32_t *tail_ready;          // [b] epoch of the last step whose appended rows are in the tail page
@@ -129,6 +131,8 @@ struct Batch {
   int32_t n_tokens[kMaxBatch];   // tokens before this step's append
   int32_t epoch;            // number of this decode call: value of the ready flags it sets
   int32_t append_in_grid;   // the scoring kernel's tail CTAs append this step's tokens
+  int32_t attn_set_major;   // attention CTAs ordered set by set (sets become ready one after the
+                            // other over a long scoring phase) instead of chunk 0 of every set first
 };
 
 __host__ __device__ inline int set_index(const DevCtx &c, int req, int layer, int head) {
@@ -213,11 +217,15 @@ __device__ __forceinline__ void flag_publish(int32_t *flag, int32_t value) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
 __device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, int32_t value) {
-  for (int spin = 0; spin < (1 << 20); ++spin) {
+  // polls back off from 64 ns to ~1 us: hundreds of waiting CTAs must not keep the L2 lines
+  // of the flags (and the producers' accesses next to them) busy
+  unsigned pause = 64;
+  for (int spin = 0; spin < (1 << 17); ++spin) {
     int32_t v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (v == value) return true;
-    __nanosleep(100);
+    __nanosleep(pause);
+    if (pause < 1024) pause <<= 1;
   }
   dev_error(c, kErrTimeout);
   return false;
@@ -285,7 +293,7 @@ int launch_stage_in(void *dq, const void *sq, size_t q_bytes, void *dk, const vo
                     size_t kv_bytes, cudaStream_t st);
 int launch_copy_centroids(const DevCtx &c, int req, int layer, const __nv_bfloat16 *cen,
                           int n_clusters, cudaStream_t st);
-int launch_select(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
+int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
                   const __nv_bfloat16 *v_new, int max_cand, cudaStream_t st, Prof *prof);
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
 int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
