@@ -111,6 +111,13 @@ typedef struct spin_config {
                                    what that over-eviction costs: of the threshold bucket only
                                    as many pages as the misses still need are taken, lowest
                                    slots first (a partition that loses a page goes whole) */
+  int32_t resident_scoring;     /* how the scoring kernel is laid out when the selection continues
+                                   in it: 0 = automatic (one CTA per work item; a grid that is
+                                   resident all at once and draws items from a queue when a step
+                                   has more than 12 items per SM, so that attention can start
+                                   fetching from the first sets), 1 = always the resident
+                                   form, -1 = never */
+  int32_t reserved0;
   int64_t offload_stage_bytes;  /* 0: appended pages are written through to pinned host memory on
                                    the caller's stream (Offload, Section 4.1).  > 0: asynchronous
                                    offload: the complete pages of an append from device memory are

@@ -44,7 +44,8 @@ class spin_config(C.Structure):
                 ("max_selected_pages", C.c_int32), ("max_tail_tokens", C.c_int32),
                 ("lru_buckets", C.c_int32), ("segment_entries", C.c_int32),
                 ("sm_scale", C.c_float), ("trace", C.c_int32), ("fetch_mode", C.c_int32),
-                ("host_tables_only", C.c_int32), ("evict_exact", C.c_int32), ("offload_stage_bytes", C.c_int64),
+                ("host_tables_only", C.c_int32), ("evict_exact", C.c_int32), ("resident_scoring", C.c_int32), ("reserved0", C.c_int32),
+                ("offload_stage_bytes", C.c_int64),
                 ("gpu_cache_pages", C.c_int64),
                 ("host_pages", C.c_int64), ("hbm_pool", C.c_void_p), ("hbm_pool_bytes", C.c_size_t)]
 

@@ -733,6 +733,7 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   d.n_host_pages = (int32_t)cfg->host_pages;
   d.fetch_mode = cfg->fetch_mode ? 1 : 0;
   d.evict_exact = cfg->evict_exact ? 1 : 0;
+  d.resident_scoring = cfg->resident_scoring > 0 ? 1 : cfg->resident_scoring < 0 ? -1 : 0;
   d.sm_scale = cfg->sm_scale != 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)kHeadDim);
 
   // directories start unmapped (-1); states, counters and the miss queue start at zero

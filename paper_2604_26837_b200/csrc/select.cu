@@ -423,7 +423,8 @@ int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_
   }
   sg.n_items = n_sets + sg.item_prefix[b.n_req];
   // resident form (grid sized in launch_score_g) when scoring is many waves long
-  sg.persistent = (fuse == 2 && c.ready && sg.n_items > 12 * sm_count_of_device()) ? 1 : 0;
+  sg.persistent = (fuse == 2 && c.ready && c.resident_scoring >= 0 &&
+                   (c.resident_scoring > 0 || sg.n_items > 12 * sm_count_of_device())) ? 1 : 0;
   dim3 grid(sg.n_items);
   b.attn_set_major = sg.persistent;
   switch (c.G) {

@@ -112,6 +112,7 @@ struct DevCtx {
   int32_t max_chunks;
   int32_t fetch_mode;           // 0: misses are fetched by the attention kernel; 1: by k_fetch
   int32_t evict_exact;          // 1: exact-demand eviction variant (see spin_config)
+  int32_t resident_scoring;     // 0 automatic, 1 always, -1 never (see spin_config)
   Counters *counters;
 };
 

@@ -48,7 +48,7 @@ class SpinRun:
 
     def __init__(self, w: W.Workload, device="cuda:0", trace=False, sm_scale=0.0,
                  slots_per_set=None, segment_entries=0, fetch_mode=0, host_tables_only=0,
-                 cache_pages_per_layer=None, spare_cache_pages=0, evict_exact=0, offload_stage_bytes=0):
+                 cache_pages_per_layer=None, spare_cache_pages=0, evict_exact=0, offload_stage_bytes=0, resident_scoring=0):
         self.w = w
         self.device = torch.device(device)
         T = w.page_tokens
@@ -71,7 +71,7 @@ class SpinRun:
             max_selected_pages=(w.topk * w.max_partition_pages if cluster else 0),
             max_tail_tokens=(w.steps + T if cluster else 0), lru_buckets=w.lru_buckets,
             segment_entries=segment_entries, sm_scale=sm_scale, trace=1 if trace else 0, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
-            evict_exact=evict_exact, offload_stage_bytes=offload_stage_bytes, gpu_cache_pages=sum(self.budgets) * sets_per_req + spare_cache_pages, host_pages=host_pages)
+            evict_exact=evict_exact, offload_stage_bytes=offload_stage_bytes, resident_scoring=resident_scoring, gpu_cache_pages=sum(self.budgets) * sets_per_req + spare_cache_pages, host_pages=host_pages)
         self.spin = B.Spin(cfg, self.device)
         self.reqs: List[int] = [self.spin.request_open(bud) for bud in self.budgets]
         self.ctx = ctx

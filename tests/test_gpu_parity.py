@@ -29,7 +29,7 @@ def _wl(kind, **kw):
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
                one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None,
                oracle_reqs=None, budget_schedule=None, spare_cache_pages=0, evict_exact=0,
-               offload_stage_bytes=0):
+               offload_stage_bytes=0, resident_scoring=0):
     """oracle_reqs: the requests mirrored in the oracle (default all).  Sets are independent, so the
     oracle run on a sample of the batch's requests must agree with those requests of the full batch."""
     from paper_2604_26837_b200.driver import SpinRun
@@ -37,7 +37,8 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     run = SpinRun(w, dev, trace=True, sm_scale=sm_scale, slots_per_set=slots,
                   segment_entries=segment_entries, fetch_mode=fetch_mode, host_tables_only=host_tables_only,
                   cache_pages_per_layer=cache_pages_per_layer, spare_cache_pages=spare_cache_pages,
-                  evict_exact=evict_exact, offload_stage_bytes=offload_stage_bytes)
+                  evict_exact=evict_exact, offload_stage_bytes=offload_stage_bytes,
+                  resident_scoring=resident_scoring)
     S = run.slots
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets, sm_scale,
@@ -317,6 +318,21 @@ def test_asynchronous_offload_of_prefill_pages(kind):
     # stream; the first decode step waits for them; results and host bytes as without it
     w = _wl(kind, topk=6 if kind == W.PART_PAGE_MINMAX else 64, steps=12)
     r = run_parity(w, offload_stage_bytes=4 * 3 * 2 * 8192, check_bytes=True)
+    assert r["stats"]["miss_pages"] > 0
+
+
+@pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_CLUSTER_CENTROID, W.PART_TOKEN_DOT])
+def test_resident_scoring_grid(kind):
+    # the queue-fed form of the scoring kernel (automatic only for long scoring phases), forced
+    # on: mixed lengths (requests own different numbers of work items), an empty request,
+    # steps that complete a page (stand-alone append first) and steps that do not
+    if kind == W.PART_CLUSTER_CENTROID:
+        w = _wl(kind, kv_recipe="mixture", num_clusters=37, topk=5, slots_per_set=30,
+                context=16 * 50 + 3, steps=24, max_partition_pages=8, lru_buckets=8)
+    else:
+        w = _wl(kind, batch=5, num_layers=1, context=16 * 300, ctx_range=(0, 16 * 300),
+                drift_choices=(0.01, 0.1, 0.5), topk=10 if kind == W.PART_PAGE_MINMAX else 100, steps=36, lru_buckets=8)
+    r = run_parity(w, one_call=True, resident_scoring=1, check_bytes=kind != W.PART_CLUSTER_CENTROID)
     assert r["stats"]["miss_pages"] > 0
 
 
