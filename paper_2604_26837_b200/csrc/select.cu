@@ -32,13 +32,6 @@ __device__ __forceinline__ void unpack8(uint4 raw, float *f) {
   }
 }
 
-__device__ __forceinline__ uint4 ld_stream16(const void *p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-
 // Score of one entry for this lane's 8 channels, all G heads; the 16 lanes of the row are
 // combined by the caller-visible butterfly.  For min/max summaries max(q*min, q*max) equals
 // q * (q >= 0 ? max : min) exactly (min <= max and the products are exact), so the operand is
