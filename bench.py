@@ -316,7 +316,7 @@ def main():
 
     props = torch.cuda.get_device_properties(device)
     sampler = ClockSampler(f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank))
-    timed_steps(P + Wm)                                    # cache priming + warm-up, untimed
+    cold_steps = timed_steps(P + Wm)                       # cache priming + warm-up: reported apart (cold start)
     st0 = run.spin.stats()
     barrier()
     t_begin = datetime.datetime.now()
@@ -433,6 +433,11 @@ def main():
                            frac_vs_nominal_8tbs=max(hbm_step / 8e12, t_pcie) / t_step,
                            miss_ratio=d["miss_pages"] / max(d["selected_pages"], 1)),
         roofline=roofline, kernels=kern, error_bits=final["error_bits"])
+    n_cold = min(8, len(cold_steps))
+    if n_cold:
+        # the first steps after prefill start from an empty GPU cache (every selected page misses)
+        line["cold_start"] = dict(steps=n_cold, first_step_ms=cold_steps[0],
+                                  mean_ms_per_step=sum(cold_steps[:n_cold]) / n_cold)
     if e2e_steps:
         line["e2e"] = dict(value=B * e2e_steps * world / (e2e_ms * 1e-3), unit=unit, h2d_bytes_per_step=h2d,
                            d2h_bytes_per_step=d2h, ms_per_step=e2e_ms / e2e_steps)
