@@ -419,6 +419,57 @@ class OracleSet:
                 self.page_v[page, : rows.shape[0]] = v_bits[rows]
         self.n_tokens = int(k_bits.shape[0])
 
+    # ---- Index during decode, cluster granularity (Section 4.1: "invoked periodically") ------
+    def reindex(self) -> List[Tuple[int, int]]:
+        """Fold the full pages of the local tail into the clusters.
+
+        The paper says that Index also runs during decode to take in new tokens and leaves the
+        rest to the algorithm.  Reading: every token of a FULL tail page, in arrival order,
+        joins the cluster whose centroid scores highest against its key (the same fp32
+        summation tree as Select, ties to the lower cluster); centroids stay as they are; the
+        token goes to the end of that cluster (a new page when the last one is full).  A
+        cluster that takes a token is no longer GPU-resident (its cached copy is stale): its
+        slots are cleared, timestamps of the others untouched.  The partly filled newest
+        page stays the tail.  Returns (token index in the folded run, cluster) pairs.
+        """
+        assert self.clustered
+        T = self.T
+        n_full = len(self.tail_pages) - (0 if (self.tail_pages and self.tail_len == T) else 1)
+        if n_full <= 0:
+            return []
+        P = self.n_partitions()
+        lists = [[self.cpu_page_table[self.part_offset[c] + i] for i in range(self.partition_pages(c))]
+                 for c in range(P)]
+        taken: List[Tuple[int, int]] = []
+        touched = set()
+        folded, self.tail_pages = self.tail_pages[:n_full], self.tail_pages[n_full:]
+        for j, page in enumerate(folded):
+            for r in range(T):
+                key = bf16_to_f32(self.page_k[page, r])[None, :]              # one "query head"
+                c = int(np.argmax(score_dot(key, self.sum_vec[:P])))          # first maximum
+                m = self.part_tokens[c]
+                if m % T == 0:
+                    lists[c].append(self._new_page())
+                dst = lists[c][m // T]
+                self.page_k[dst, m % T] = self.page_k[page, r]
+                self.page_v[dst, m % T] = self.page_v[page, r]
+                self.part_tokens[c] = m + 1
+                touched.add(c)
+                taken.append((j * T + r, c))
+        if not self.tail_pages:
+            self.tail_len = 0
+        # the CPU page table is laid out afresh: clusters in order, each one's pages together
+        self.cpu_page_table, self.part_offset = [], []
+        for c in range(P):
+            self.part_offset.append(len(self.cpu_page_table))
+            self.cpu_page_table.extend(lists[c])
+        self.cpu_page_table.extend(self.tail_pages)
+        for c in touched:
+            self.part_resident[c] = 0
+        gone = np.isin(self.slot_part, np.asarray(sorted(touched), dtype=self.slot_part.dtype))
+        self.slot_part[gone], self.slot_pidx[gone], self.slot_ts[gone] = -1, 0, -1
+        return taken
+
     # ---- buffer elasticity (Section 5.3, "Buffer Elasticity") ------------------------------
     def resize(self, new_slots: int) -> List[Tuple[int, int, int]]:
         """Change the set's number of GPU page table slots between steps.
@@ -567,6 +618,10 @@ class SpinOracle:
         for layer in self.requests[req]:
             for st in layer:
                 st.resize(slots_per_set)
+
+    def reindex(self, req: int, layer: int):
+        """Fold the full tail pages of every kv head's set of (request, layer) into its clusters."""
+        return [st.reindex() for st in self.requests[req][layer]]
 
     def set(self, req: int, layer: int, head: int) -> OracleSet:
         return self.requests[req][layer][head]

@@ -205,3 +205,96 @@ def test_c1_regression_against_stored_oracle_trace():
     lines, outs = _c1_trace_lines()
     stored = [x.rstrip("\n") for x in open(os.path.join(GOLD, "c1_oracle_trace.txt")) if not x.startswith("#")]
     assert lines == stored
+
+
+# ---- Index during decode (cluster granularity): full tail pages fold into the clusters -------
+
+def _bits(x):
+    """fp32 -> bf16 bit patterns (round to nearest even)."""
+    return (O.f32_to_bf16_f32(np.asarray(x, dtype=np.float32)).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def _clustered_set(rng, n_tokens, C, d=128, slots=12, topk=4):
+    cfg = O.OracleConfig(1, 2, 1, d, 16, O.PART_CLUSTER_CENTROID, topk, 4)
+    st = O.OracleSet(cfg, slots)
+    cen = rng.standard_normal((C, d)).astype(np.float32) * 2.0
+    assign = rng.integers(0, C, size=n_tokens)
+    k = cen[assign] + 0.2 * rng.standard_normal((n_tokens, d)).astype(np.float32)
+    v = rng.standard_normal((n_tokens, d)).astype(np.float32)
+    st.append_clustered(_bits(k), _bits(v), assign, _bits(cen))
+    return cfg, st, cen
+
+
+def _all_rows(st):
+    rows = []
+    for c in range(st.n_partitions()):
+        for i in range(st.partition_pages(c)):
+            page = st.cpu_page_table[st.part_offset[c] + i]
+            valid = min(st.T, st.part_tokens[c] - i * st.T)
+            rows += [(st.page_k[page, r].tobytes(), st.page_v[page, r].tobytes()) for r in range(valid)]
+    for j, page in enumerate(st.tail_pages):
+        valid = st.tail_len if j == len(st.tail_pages) - 1 else st.T
+        rows += [(st.page_k[page, r].tobytes(), st.page_v[page, r].tobytes()) for r in range(valid)]
+    return rows
+
+
+def test_reindex_moves_every_tail_token_to_its_best_centroid_and_keeps_all_rows():
+    rng = np.random.default_rng(21)
+    C = 9
+    cfg, st, cen = _clustered_set(rng, 150, C)
+    cen_bf = O.bf16_to_f32(_bits(cen)).astype(np.float64)
+    new_assign = rng.integers(0, C, size=40)
+    nk = cen[new_assign] + 0.2 * rng.standard_normal((40, 128)).astype(np.float32)
+    nv = rng.standard_normal((40, 128)).astype(np.float32)
+    kb, vb = _bits(nk), _bits(nv)
+    st.append_tokens(kb, vb)                       # 2 full tail pages + 8 tokens
+    before = sorted(_all_rows(st))
+    counts = list(st.part_tokens)
+    taken = st.reindex()
+    assert sorted(_all_rows(st)) == before                     # nothing lost, nothing doubled
+    assert len(taken) == 32 and len(st.tail_pages) == 1 and st.tail_len == 8
+    # well separated centroids: the winner is the plain float64 argmax, which is the generating cluster
+    best = np.argmax(O.bf16_to_f32(kb[:32]).astype(np.float64) @ cen_bf.T, axis=1)
+    assert [c for _, c in taken] == [int(x) for x in best] == [int(x) for x in new_assign[:32]]
+    # arrival order at the end of each cluster
+    for t, c in taken:
+        pos = counts[c]
+        page = st.cpu_page_table[st.part_offset[c] + pos // 16]
+        assert st.page_k[page, pos % 16].tobytes() == kb[t].tobytes()
+        counts[c] += 1
+    assert counts == st.part_tokens
+    assert st.reindex() == []                                  # nothing full is left in the tail
+
+
+def test_reindex_leaves_dense_attention_unchanged_and_drops_stale_residency():
+    rng = np.random.default_rng(22)
+    C = 6
+    cfg, st, cen = _clustered_set(rng, 90, C, slots=40, topk=C)    # top-k = every cluster: dense attention
+    q = _bits(rng.standard_normal((2, 128)).astype(np.float32))
+    st.append_tokens(_bits(rng.standard_normal((33, 128)).astype(np.float32)),
+                     _bits(rng.standard_normal((33, 128)).astype(np.float32)))
+    out0, tr0 = st.decode(q)
+    assert all(st.part_resident[c] for c in range(C) if st.part_tokens[c])
+    taken = st.reindex()
+    touched = {c for _, c in taken}
+    assert touched and all(st.part_resident[c] == 0 for c in touched)
+    assert not (set(int(p) for p in st.slot_part if p >= 0) & touched)
+    out1, tr1 = st.decode(q)
+    np.testing.assert_allclose(out1, out0, rtol=0, atol=1e-12)  # same tokens attended, other order
+    assert set(tr1.misses) == touched                            # exactly the stale clusters are fetched again
+
+
+def test_reindex_with_a_full_newest_page_empties_the_tail_and_equal_scores_go_to_the_lower_cluster():
+    rng = np.random.default_rng(23)
+    cfg = O.OracleConfig(1, 1, 1, 128, 16, O.PART_CLUSTER_CENTROID, 2, 4)
+    st = O.OracleSet(cfg, 8)
+    cen = rng.standard_normal((3, 128)).astype(np.float32)
+    cen[2] = cen[1]                                              # clusters 1 and 2 share a centroid
+    k = rng.standard_normal((20, 128)).astype(np.float32)
+    st.append_clustered(_bits(k), _bits(k), rng.integers(0, 3, size=20), _bits(cen))
+    nk = np.repeat(cen[1:2] * 3.0, 16, axis=0)
+    st.append_tokens(_bits(nk), _bits(nk))   # exactly one full page
+    taken = st.reindex()
+    assert [c for _, c in taken] == [1] * 16 and st.tail_pages == [] and st.tail_len == 0
+    st.append_tokens(_bits(nk[:3]), _bits(nk[:3]))
+    assert len(st.tail_pages) == 1 and st.tail_len == 3
