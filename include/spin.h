@@ -211,6 +211,21 @@ SPIN_API int spin_request_open(spin_ctx *ctx, int64_t hbm_budget_pages_per_set, 
  * waits for the device before and after.  The policy -- when to resize whom -- is the caller's
  * (the paper's scheduler); this is the mechanism. */
 SPIN_API int spin_set_budget(spin_ctx *ctx, int32_t req, int64_t hbm_budget_pages_per_set);
+/* Index during decode, cluster granularity (Section 4.1: Index is "invoked ... periodically in
+ * decode to take in new tokens"; the paper leaves the rule to the algorithm).  Folds the FULL
+ * pages of the local tail of every kv head's set of (request, layer) into the clusters: each
+ * token, in arrival order, joins the cluster whose centroid scores highest against its key
+ * (the fp32 summation order of Select, ties to the lower cluster id) and goes to the end of
+ * that cluster (a new host page when its last one is full); centroids stay as they are.  A
+ * cluster that takes a token loses its GPU residency (the cached copy is stale): flag and
+ * slots cleared.  The partly filled newest page stays the tail.  The set's CPU page table and
+ * Partition Offset table are laid out afresh.  Host-driven and synchronous: the call waits for
+ * the stream twice (it needs the assignment on the host) and returns when the fold is done.
+ * At most 2048 tail tokens per call.  SPIN_ERR_INVALID for the other granularities,
+ * SPIN_ERR_STATE before the cluster prefill, SPIN_ERR_OOM_HOST if host pages run out (nothing
+ * has been changed then). */
+SPIN_API int spin_reindex(spin_ctx *ctx, int32_t req, int32_t layer, void *cuda_stream);
+
 /* Give back the request's pages and segments.  No work of this request may be in flight. */
 SPIN_API int spin_request_close(spin_ctx *ctx, int32_t req);
 

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "SPIN_OK", 1: "SPIN_ERR_INVALID", 2: "SPIN_ERR_STATE", 3: "SP
 PART_PAGE_MINMAX, PART_TOKEN_DOT, PART_CLUSTER_CENTROID, PART_PAGE_MEAN = 0, 1, 2, 3
 PAGE_BYTES = 8192
 
-EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open",
+EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open", "spin_reindex",
            "spin_request_close", "spin_set_budget", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
            "spin_decode_step_append", "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
            "spin_debug_read_page", "spin_paged_attention_static", "spin_last_error",
@@ -105,6 +105,7 @@ def load() -> C.CDLL:
     lib.spin_request_open.argtypes = [vp, i64, _I32P]
     lib.spin_request_close.argtypes = [vp, i32]
     lib.spin_set_budget.argtypes = [vp, i32, i64]
+    lib.spin_reindex.argtypes = [vp, i32, i32, vp]
     lib.spin_append_kv.argtypes = [vp, i32, i32, vp, vp, i64, vp, vp, vp]
     lib.spin_append_kv_batch.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
     lib.spin_decode_step.argtypes = [vp, i32, _I32P, i32, vp, vp, vp]
@@ -238,6 +239,9 @@ class Spin:
         arr = (C.c_int32 * len(req_ids))(*req_ids)
         self._ck(self.lib.spin_decode_step(self.h, layer, arr, len(req_ids), _ptr(q), _ptr(out),
                                            _stream_ptr(stream)))
+
+    def reindex(self, req: int, layer: int, stream=None):
+        self._ck(self.lib.spin_reindex(self.h, req, layer, _stream_ptr(stream)))
 
     def decode_step_append(self, layer: int, req_ids: Sequence[int], k_new, v_new, q, out, stream=None):
         arr = (C.c_int32 * len(req_ids))(*req_ids)

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libspin.so")
-SOURCES = ["api.cu", "append.cu", "select.cu", "cache.cu", "attention.cu"]
+SOURCES = ["api.cu", "append.cu", "select.cu", "cache.cu", "attention.cu", "reindex.cu"]
 # -dlcm=cg: global loads are cached in L2 only.  Kernels of consecutive steps overlap (programmatic
 # dependent launch) and hand state to one another through global memory, and an SM's L1 is not
 # coherent with other SMs' writes; the bulk traffic bypasses L1 anyway.

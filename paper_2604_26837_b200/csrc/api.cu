@@ -51,6 +51,7 @@ struct SetHost {                     // host mirror of one (request, layer, kv h
   std::vector<int32_t> dir_meta, dir_gpt, dir_off, dir_cpt, dir_sum;
   std::vector<int32_t> gpu_pages;    // physical pages behind the slots
   std::vector<int32_t> host_pages;   // CPU page table mirror (logical page -> host page)
+  std::vector<int32_t> cl_tokens;    // cluster granularity: tokens of every cluster
 };
 
 struct LayerHost {                   // counts shared by the kv-head sets of (request, layer)
@@ -524,6 +525,7 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
       off += npg;
     }
     total_pages_max = std::max(total_pages_max, off);
+    S.cl_tokens.assign(count.begin() + (size_t)h * C, count.begin() + (size_t)(h + 1) * C);
     // Meta-partition entries, segment by segment
     for (int c0 = 0; c0 < C; c0 += g.seg) {
       const int cnt = std::min(g.seg, C - c0);
@@ -859,6 +861,130 @@ int spin_request_open(spin_ctx *ctx, int64_t slots, int32_t *out_req) {
   return SPIN_OK;
 }
 
+int spin_reindex(spin_ctx *ctx, int32_t req, int32_t layer, void *cuda_stream) {
+  int rc = validate_req_layer(ctx, req, layer);
+  if (rc) return rc;
+  if (ctx->cfg.partition_kind != SPIN_PART_CLUSTER_CENTROID)
+    return fail(ctx, SPIN_ERR_INVALID, "spin_reindex applies to cluster granularity only");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  LayerHost &L = ctx->reqs[(size_t)req].layers[(size_t)layer];
+  if (!L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req);
+  const Geometry &g = ctx->g;
+  const DevCtx &d = ctx->d;
+  const int H = ctx->cfg.num_kv_heads, C = ctx->cfg.num_clusters;
+  // full tail pages, as many as the staging buffers take in one go
+  int n_full = L.tail_pages - (L.tail_pages > 0 && L.tail_len == kPageTokens ? 0 : 1);
+  n_full = std::min<int>(n_full, (int)(g.stage_tokens / kPageTokens));
+  if (n_full <= 0) return SPIN_OK;
+  const int n_tok = n_full * kPageTokens;
+
+  // 1. the best cluster of every token (device), brought to the host; everything enqueued on
+  //    the stream before this call has finished once the copy is here
+  int32_t *d_assign = reinterpret_cast<int32_t *>(ctx->stage_k);
+  ctx->launches += launch_assign(d, req, layer, C, n_tok, d_assign, st);
+  std::vector<int32_t> assign((size_t)n_tok * H);
+  CK(cudaMemcpyAsync(assign.data(), d_assign, assign.size() * 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+
+  // 2. new page lists and layout, head by head.  First pass: how many host pages it takes.
+  int64_t need = 0;
+  for (int h = 0; h < H; ++h) {
+    std::vector<int32_t> cnt = set_of(ctx, req, layer, h).cl_tokens;
+    for (int t = 0; t < n_tok; ++t) {
+      const int32_t c = assign[(size_t)t * H + h];
+      if (c < 0 || c >= C) return fail(ctx, SPIN_ERR_CUDA, "cluster assignment out of range");
+      if (cnt[(size_t)c]++ % kPageTokens == 0) ++need;
+    }
+  }
+  if (ctx->host_page_pool.available() < need) return fail(ctx, SPIN_ERR_OOM_HOST, "out of host pages");
+  std::vector<int64_t> dest((size_t)n_tok * H);
+  std::vector<int32_t> new_tokens((size_t)H * C);
+  const int words = (C + 31) / 32;
+  std::vector<uint32_t> touched((size_t)H * words, 0u);
+  std::vector<std::vector<int32_t>> old_tail((size_t)H);
+  std::vector<std::vector<std::vector<int32_t>>> lists((size_t)H);
+  int32_t total_max = 0;
+  for (int h = 0; h < H; ++h) {
+    SetHost &S = set_of(ctx, req, layer, h);
+    for (int i = 0; i < L.tail_pages; ++i) old_tail[(size_t)h].push_back(S.host_pages[(size_t)(L.tail_first + i)]);
+    auto &ls = lists[(size_t)h];
+    ls.resize((size_t)C);
+    for (int c = 0; c < C; ++c) {
+      const int32_t seg = S.dir_off[(size_t)(c >> g.seg_shift)];
+      const int32_t off = ctx->h_off_pool[((size_t)seg << g.seg_shift) + (c & (g.seg - 1))];
+      const int npg = (S.cl_tokens[(size_t)c] + kPageTokens - 1) / kPageTokens;
+      ls[(size_t)c].assign(S.host_pages.begin() + off, S.host_pages.begin() + off + npg);
+    }
+    for (int t = 0; t < n_tok; ++t) {
+      const int32_t c = assign[(size_t)t * H + h];
+      const int32_t m = S.cl_tokens[(size_t)c];
+      if (m % kPageTokens == 0) ls[(size_t)c].push_back((int32_t)ctx->host_page_pool.alloc());
+      dest[(size_t)t * H + h] = (int64_t)ls[(size_t)c][(size_t)(m / kPageTokens)] * kPageTokens + m % kPageTokens;
+      S.cl_tokens[(size_t)c] = m + 1;
+      touched[(size_t)h * words + (c >> 5)] |= 1u << (c & 31);
+    }
+    int32_t total = 0;
+    for (int c = 0; c < C; ++c) total += (int32_t)ls[(size_t)c].size();
+    total_max = std::max(total_max, total);
+    std::copy(S.cl_tokens.begin(), S.cl_tokens.end(), new_tokens.begin() + (size_t)h * C);
+  }
+
+  // 3. the sets' Partition Offset and CPU page tables laid out afresh (clusters in order, each
+  //    one's pages together), what is left of the tail behind the longest head's clusters
+  const int n_rem = L.tail_pages - n_full;
+  if ((int64_t)total_max + g.tail_cap > (int64_t)g.dir_page * g.seg)
+    return fail(ctx, SPIN_ERR_INVALID, "request %d outgrew its CPU page table", req);
+  for (int h = 0; h < H; ++h) {
+    const int set = set_index(d, req, layer, h);
+    SetHost &S = ctx->sets[(size_t)set];
+    S.host_pages.assign((size_t)(total_max + n_rem), -1);
+    auto put = [&](int64_t j, int32_t hp) -> bool {
+      const int cs = ensure_seg(ctx, ctx->cpt_segs, S.dir_cpt, d.dir_cpt + (size_t)set * g.dir_page, j, g.seg_shift, st);
+      if (cs < 0) return false;
+      ctx->h_cpt_pool[((size_t)cs << g.seg_shift) + (j & (g.seg - 1))] = hp;
+      S.host_pages[(size_t)j] = hp;
+      return true;
+    };
+    int32_t off = 0;
+    for (int c = 0; c < C; ++c) {
+      const int32_t seg = S.dir_off[(size_t)(c >> g.seg_shift)];
+      ctx->h_off_pool[((size_t)seg << g.seg_shift) + (c & (g.seg - 1))] = off;
+      for (int32_t hp : lists[(size_t)h][(size_t)c])
+        if (!put(off++, hp)) return fail(ctx, SPIN_ERR_OOM_HOST, "out of CPU page table segments");
+    }
+    for (int i = 0; i < n_rem; ++i)
+      if (!put((int64_t)total_max + i, old_tail[(size_t)h][(size_t)(n_full + i)])) return fail(ctx, SPIN_ERR_OOM_HOST, "out of CPU page table segments");
+    for (int i = 0; i < n_full; ++i) ctx->host_page_pool.release(old_tail[(size_t)h][(size_t)i]);   // their rows live in the clusters now
+  }
+
+  // 4. device side: rows to their places; counts, residency and tail; the tables' HBM copies
+  int32_t *d_new_tokens = reinterpret_cast<int32_t *>(ctx->stage_v);
+  uint32_t *d_touched = reinterpret_cast<uint32_t *>(d_new_tokens + new_tokens.size());
+  const size_t stage_bytes = (size_t)std::max<int64_t>(g.stage_tokens, ctx->cfg.max_requests) * H * kRowBytes;
+  if ((new_tokens.size() + touched.size()) * 4 > stage_bytes) return fail(ctx, SPIN_ERR_INVALID, "too many clusters for the staging buffer");
+  CK(cudaMemcpyAsync(ctx->stage_dest, dest.data(), dest.size() * 8, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(d_new_tokens, new_tokens.data(), new_tokens.size() * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(d_touched, touched.data(), touched.size() * 4, cudaMemcpyHostToDevice, st));
+  ctx->launches += launch_move_rows(d, req, layer, ctx->stage_dest, n_tok, st);
+  ctx->launches += launch_reindex_apply(d, req, layer, C, n_full, total_max, n_rem, n_rem ? L.tail_len : 0,
+                                        total_max + n_rem, d_new_tokens, d_touched, st);
+  if (d.off_mirror) {
+    for (int h = 0; h < H; ++h) {
+      const SetHost &S = set_of(ctx, req, layer, h);
+      for (int32_t seg : S.dir_off)
+        if (seg >= 0) CK(cudaMemcpyAsync(d.off_mirror + ((size_t)seg << g.seg_shift), ctx->h_off_pool + ((size_t)seg << g.seg_shift), (size_t)g.seg * 4, cudaMemcpyHostToDevice, st));
+      for (int32_t seg : S.dir_cpt)
+        if (seg >= 0) CK(cudaMemcpyAsync(d.cpt_mirror + ((size_t)seg << g.seg_shift), ctx->h_cpt_pool + ((size_t)seg << g.seg_shift), (size_t)g.seg * 4, cudaMemcpyHostToDevice, st));
+    }
+  }
+  L.tail_first = total_max;
+  L.tail_pages = n_rem;
+  if (n_rem == 0) L.tail_len = 0;
+  L.n_host_pages = total_max + n_rem;
+  CK(cudaStreamSynchronize(st));          // the host-side sources of the copies above end here
+  CK(cudaGetLastError());
+  return SPIN_OK;
+}
 int spin_request_close(spin_ctx *ctx, int32_t req) {
   if (!ctx) return SPIN_ERR_INVALID;
   if (req < 0 || req >= ctx->cfg.max_requests) return fail(ctx, SPIN_ERR_INVALID, "request id %d out of range", req);

@@ -299,6 +299,11 @@ int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
 int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
 int launch_shrink(const DevCtx &c, int req, int old_S, int new_S, cudaStream_t st);
+int launch_assign(const DevCtx &c, int req, int layer, int n_clusters, int n_tokens, int32_t *assign, cudaStream_t st);
+int launch_move_rows(const DevCtx &c, int req, int layer, const int64_t *dest, int n_tokens, cudaStream_t st);
+int launch_reindex_apply(const DevCtx &c, int req, int layer, int n_clusters, int n_folded_pages, int tail_first,
+                         int tail_pages, int tail_len, int n_host_pages, const int32_t *new_tokens,
+                         const uint32_t *touched, cudaStream_t st);
 size_t cache_smem_bytes(const DevCtx &c);
 int launch_attention(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q,
                      __nv_bfloat16 *out, int max_pages_hint, bool may_be_empty, cudaStream_t st, Prof *prof);

@@ -109,6 +109,10 @@ class SpinRun:
         """Append one token per request and decode, in one library call."""
         self.spin.decode_step_append(layer, self.reqs, k_new, v_new, q, out, stream)
 
+    def reindex(self, r: int, layer: int, stream=None):
+        """Fold request r's full tail pages into its clusters (cluster granularity)."""
+        self.spin.reindex(self.reqs[r], layer, stream)
+
     def set_budget(self, r: int, slots: int):
         """Resize the GPU slots of every set of request r (buffer elasticity)."""
         self.spin.set_budget(self.reqs[r], slots)

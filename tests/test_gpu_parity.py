@@ -29,7 +29,7 @@ def _wl(kind, **kw):
 def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True, tol_scale=1.0,
                one_call=False, fetch_mode=0, host_tables_only=0, host_io=None, cache_pages_per_layer=None,
                oracle_reqs=None, budget_schedule=None, spare_cache_pages=0, evict_exact=0,
-               offload_stage_bytes=0, resident_scoring=0):
+               offload_stage_bytes=0, resident_scoring=0, reindex_every=0):
     """oracle_reqs: the requests mirrored in the oracle (default all).  Sets are independent, so the
     oracle run on a sample of the batch's requests must agree with those requests of the full batch."""
     from paper_2604_26837_b200.driver import SpinRun
@@ -69,11 +69,18 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     cap_sel = w.topk
     cap_pages = w.topk * max(1, w.max_partition_pages) + (w.steps + 16) // 16 + 2
     worst_abs, worst_mean, rel_num, rel_den = 0.0, 0.0, 0.0, 0.0
+    folded = 0
     for step in range(w.steps):
         for r, new_slots in (budget_schedule or {}).get(step, {}).items():     # buffer elasticity between steps
             run.set_budget(r, new_slots)
             if r in oreq:
                 orc.set_budget(oreq[r], new_slots)
+        if reindex_every and step and step % reindex_every == 0:                # Index during decode (clusters)
+            for r in range(w.batch):
+                for l in range(w.num_layers):
+                    run.reindex(r, l)
+                    if r in oreq:
+                        folded += sum(len(x) for x in orc.reindex(oreq[r], l))
         for l in range(w.num_layers):
             kn, vn = run.gen_step_tokens(l, step)
             kb, vb = W.to_bits(kn), W.to_bits(vn)
@@ -153,7 +160,7 @@ def run_parity(w, sm_scale=0.0, slots=None, segment_entries=0, check_bytes=True,
     assert stats["bypass_pages"] <= stats["miss_pages"] and stats["pcie_bytes"] == stats["miss_pages"] * 8192
     assert worst_abs <= MAX_ABS * tol_scale and worst_mean <= MEAN_ABS * tol_scale, (worst_abs, worst_mean)
     run.close()
-    return dict(max_abs=worst_abs, mean_abs=worst_mean, rel_l2=math.sqrt(rel_num / max(rel_den, 1e-30)),
+    return dict(folded=folded, max_abs=worst_abs, mean_abs=worst_mean, rel_l2=math.sqrt(rel_num / max(rel_den, 1e-30)),
                 stats=stats)
 
 
@@ -334,6 +341,16 @@ def test_resident_scoring_grid(kind):
                 drift_choices=(0.01, 0.1, 0.5), topk=10 if kind == W.PART_PAGE_MINMAX else 100, steps=36, lru_buckets=8)
     r = run_parity(w, one_call=True, resident_scoring=1, check_bytes=kind != W.PART_CLUSTER_CENTROID)
     assert r["stats"]["miss_pages"] > 0
+
+
+def test_cluster_tail_is_folded_into_the_clusters_during_decode():
+    # Index during decode: every 20 steps the full tail pages join the clusters of their best
+    # centroids (new cluster pages, stale residency dropped, layout rewritten, tail rotated);
+    # selections, cache traces, page lists, host bytes and outputs stay equal to the oracle's
+    w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=23, topk=5, slots_per_set=40,
+            context=16 * 30 + 7, steps=70, max_partition_pages=12, lru_buckets=8, batch=2, num_layers=2)
+    r = run_parity(w, reindex_every=20)
+    assert r["stats"]["miss_pages"] > 0 and r["folded"] == 2 * 2 * 2 * 48
 
 
 def test_tiny_configuration_full_size():
