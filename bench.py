@@ -195,6 +195,7 @@ def main():
     ap.add_argument("--prime", type=int, default=24, help="untimed decode steps that warm the KV cache (setup)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--resident-scoring", type=int, default=0, help="spin_config.resident_scoring: 0 automatic, 1 always, -1 never")
     ap.add_argument("--context", type=int, default=0, help="override the context length (smaller captures)")
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (scaled runs of the 32-layer config)")
@@ -256,7 +257,8 @@ def main():
     e2e_steps = 0 if args.no_e2e else K
     total_steps = P + Wm + K + K + prof_steps + (Wm + e2e_steps)
     w = rank_workload(base, rank, total_steps)
-    run = SpinRun(w, device, fetch_mode=args.fetch_mode, cache_pages_per_layer=cache_pages_per_layer)
+    run = SpinRun(w, device, fetch_mode=args.fetch_mode, cache_pages_per_layer=cache_pages_per_layer,
+                  resident_scoring=args.resident_scoring)
     stream = torch.cuda.Stream(device)
     B, L = w.batch, w.num_layers
 
