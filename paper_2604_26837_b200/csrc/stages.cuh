@@ -888,7 +888,7 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
   fast_prefetch_gpt<T>(c, L, S);
   fast_prefetch_tables<T>(c, L, bt.n_partitions[i_req]);
 
-  // ---- top-k: radix select (two barriers per pass), one-scan ordered compaction -------------
+  // ---- top-k: wide-digit radix select, one-scan ordered compaction ---------------------------
   int32_t *g_sel = c.sel_ids + (size_t)b * c.max_sel;
   int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
   if (k == n) {
