@@ -222,6 +222,13 @@ def test_page_minmax_single_bucket_and_gqa1_gqa8():
     run_parity(_wl(W.PART_PAGE_MINMAX, steps=6, num_q_heads=16, num_kv_heads=2))
 
 
+@pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_TOKEN_DOT, W.PART_CLUSTER_CENTROID, W.PART_PAGE_MEAN])
+def test_gqa_group_of_two(kind):
+    # two query heads per kv head: the score reduction trades one head between lane pairs
+    extra = dict(kv_recipe="mixture", num_clusters=19, max_partition_pages=8) if kind == W.PART_CLUSTER_CENTROID else {}
+    run_parity(_wl(kind, num_q_heads=4, num_kv_heads=2, steps=10, topk=6 if kind != W.PART_TOKEN_DOT else 50, **extra))
+
+
 def test_more_slots_than_the_shared_memory_path_holds():
     # > 1024 slots per set: the cache manager works on the page table in global memory
     w = _wl(W.PART_PAGE_MINMAX, context=16 * 1300 + 3, slots_per_set=1100, topk=40, steps=36, batch=1,
