@@ -129,12 +129,14 @@ def load() -> C.CDLL:
 
 def _ptr(x) -> Optional[int]:
     """Address of a torch tensor / numpy array / int / None."""
+    try:
+        return x.data_ptr()                      # torch tensor: the common case, no type tests
+    except AttributeError:
+        pass
     if x is None:
         return None
     if isinstance(x, int):
         return x
-    if hasattr(x, "data_ptr"):
-        return x.data_ptr()
     if hasattr(x, "ctypes"):
         return x.ctypes.data
     raise TypeError(type(x))
@@ -243,10 +245,18 @@ class Spin:
     def reindex(self, req: int, layer: int, stream=None):
         self._ck(self.lib.spin_reindex(self.h, req, layer, _stream_ptr(stream)))
 
-    def decode_step_append(self, layer: int, req_ids: Sequence[int], k_new, v_new, q, out, stream=None):
-        arr = (C.c_int32 * len(req_ids))(*req_ids)
-        self._ck(self.lib.spin_decode_step_append(self.h, layer, arr, len(req_ids), _ptr(k_new),
-                                                  _ptr(v_new), _ptr(q), _ptr(out), _stream_ptr(stream)))
+    def req_array(self, req_ids: Sequence[int]):
+        """The request ids as the int32 array the library takes (callers of the per-step entry
+        points may build it once and pass it instead of the list)."""
+        return (C.c_int32 * len(req_ids))(*req_ids)
+
+    def decode_step_append(self, layer: int, req_ids, k_new, v_new, q, out, stream=None):
+        # the per-token call: as little Python as possible before the library gets control
+        arr = req_ids if isinstance(req_ids, C.Array) else (C.c_int32 * len(req_ids))(*req_ids)
+        rc = self.lib.spin_decode_step_append(self.h, layer, arr, len(arr), _ptr(k_new), _ptr(v_new),
+                                              _ptr(q), _ptr(out), None if stream is None else _stream_ptr(stream))
+        if rc:
+            self._ck(rc)
 
     def stats(self) -> dict:
         s = spin_stats_t()

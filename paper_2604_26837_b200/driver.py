@@ -74,6 +74,7 @@ class SpinRun:
             evict_exact=evict_exact, offload_stage_bytes=offload_stage_bytes, resident_scoring=resident_scoring, gpu_cache_pages=sum(self.budgets) * sets_per_req + spare_cache_pages, host_pages=host_pages)
         self.spin = B.Spin(cfg, self.device)
         self.reqs: List[int] = [self.spin.request_open(bud) for bud in self.budgets]
+        self._req_arr = self.spin.req_array(self.reqs)
         self.ctx = ctx
         self.step_no = 0
 
@@ -107,7 +108,7 @@ class SpinRun:
 
     def step(self, layer: int, k_new, v_new, q, out, stream=None):
         """Append one token per request and decode, in one library call."""
-        self.spin.decode_step_append(layer, self.reqs, k_new, v_new, q, out, stream)
+        self.spin.decode_step_append(layer, self._req_arr, k_new, v_new, q, out, stream)
 
     def reindex(self, r: int, layer: int, stream=None):
         """Fold request r's full tail pages into its clusters (cluster granularity)."""
