@@ -218,15 +218,16 @@ __device__ __forceinline__ void flag_publish(int32_t *flag, int32_t value) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
 __device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, int32_t value) {
-  // polls back off from 64 ns to ~1 us: hundreds of waiting CTAs must not keep the L2 lines
-  // of the flags (and the producers' accesses next to them) busy
-  unsigned pause = 64;
-  for (int spin = 0; spin < (1 << 17); ++spin) {
+  // polls back off from 32 ns to 256 ns: hundreds of waiting CTAs should not keep the L2
+  // lines of the flags busy, and a raised flag should still be seen within a fraction of a
+  // microsecond
+  unsigned pause = 32;
+  for (int spin = 0; spin < (1 << 19); ++spin) {
     int32_t v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (v == value) return true;
     __nanosleep(pause);
-    if (pause < 1024) pause <<= 1;
+    if (pause < 256) pause <<= 1;
   }
   dev_error(c, kErrTimeout);
   return false;
