@@ -234,14 +234,16 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
   __shared__ int s_item[2];
   const bool pers = sg.persistent != 0;
   if (pers) {
-    if (threadIdx.x == 0) s_item[0] = atomicAdd(c.score_queue, 1);
+    // the first item is the CTA's own number (no storm on the counter at the start); the queue
+    // hands out the items from gridDim.x on
+    if (threadIdx.x == 0) s_item[0] = (int)blockIdx.x;
     __syncthreads();
   }
   for (int it = 0;; ++it) {
     const int item = pers ? s_item[it & 1] : (int)blockIdx.x;
     if (item >= sg.n_items) break;
     int next = 0;
-    if (pers && threadIdx.x == 0) next = atomicAdd(c.score_queue, 1);   // in flight while this item is worked on
+    if (pers && threadIdx.x == 0) next = (int)gridDim.x + atomicAdd(c.score_queue, 1);   // in flight while this item is worked on
     if (item == 0 && threadIdx.x == 0) *c.fetch_count = 0;               // new step, new miss queue
     int b = item, x = -1;                                                // the sets' tail items come first
     if (item >= sg.n_sets) {
