@@ -92,6 +92,17 @@ class ClockSampler:
                     reasons=reasons, samples=len(inside))
 
 
+def pcie_link(gpu_id: str):
+    """Generation and width of the GPU's host link as nvidia-smi reports them now (or None)."""
+    try:
+        out = subprocess.run(["nvidia-smi", "-i", gpu_id, "--query-gpu=pcie.link.gen.current,pcie.link.width.current",
+                              "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10).stdout
+        gen, width = [int(x.strip()) for x in out.strip().splitlines()[0].split(",")]
+        return dict(gen=gen, width=width)
+    except Exception:
+        return None
+
+
 def measure_pcie_gbs(torch, device, stream) -> float:
     """Peak of the host link as one large pinned host->device copy (best of 5)."""
     n = 256 << 20
@@ -338,6 +349,7 @@ def main():
     torch.cuda.synchronize(device)
     noflush_ms = e0.elapsed_time(e1) / K
     clocks = sampler.stop(t_begin, t_end)
+    link = pcie_link(f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank))
 
     # per-kernel durations, measured live with CUDA events recorded between the launches
     stp0 = run.spin.stats()
@@ -437,7 +449,7 @@ def main():
                            hbm_gbs_peak=peaks["hbm_gbs"], hbm_peak_source=peaks["source"], pcie_gbs_peak=pcie_gbs,
                            t_hbm_us=1e6 * t_hbm, t_pcie_us=1e6 * t_pcie, t_step_us=1e6 * t_step,
                            bound="pcie" if t_pcie > t_hbm else "hbm", frac=max(t_hbm, t_pcie) / t_step,
-                           frac_vs_nominal_8tbs=max(hbm_step / 8e12, t_pcie) / t_step,
+                           frac_vs_nominal_8tbs=max(hbm_step / 8e12, t_pcie) / t_step, pcie_link=link,
                            miss_ratio=d["miss_pages"] / max(d["selected_pages"], 1)),
         roofline=roofline, kernels=kern, error_bits=final["error_bits"])
     n_cold = min(8, len(cold_steps))
