@@ -43,6 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         s, o = os.path.join(CSRC, src), os.path.join(OBJ, src[:-3] + ".o")
         if force or _stale(o, [s] + headers):
             extra = ["-DSPIN_TIMING"] if os.environ.get("SPIN_TIMING") else []
+            extra += ["-D" + d for d in os.environ.get("SPIN_DEFINES", "").split() if d]
             cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 

@@ -1,7 +1,8 @@
 // Select (Table 1: score(q, k_sums) -> topk; Section 4.1 "Select").
 //
 // k_score streams the summary segments of every set of the batch once (HBM bound: 512 B per
-// page for min/max summaries, 256 B per token key or centroid) and writes one fp32 score per
+// page for min/max summaries, 256 B per token key or centroid; a 64 KiB segment is staged in
+// shared memory by four TMA bulk copies with an mbarrier each) and writes one fp32 score per
 // candidate.  The summation order is fixed so that the CPU oracle reproduces every score bit
 // for bit: a lane owns 8 consecutive channels (one 16-byte load) and adds them left to right;
 // the 16 lanes of a row are then combined by a butterfly (xor 1, 2, 4, 8), which is the
@@ -131,6 +132,36 @@ __device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, con
   const int seg = e0 < n_cand ? c.dir_sumseg[(size_t)set * c.dir_sum + x] : 0;
   if (seg < 0 && threadIdx.x == 0) dev_error(c, kErrBounds);
   if (e0 < n_cand && seg >= 0) {
+  const int n_here = min(seg_entries, n_cand - e0);
+  constexpr int kEntry = MINMAX ? 2 * kRowBytes : kRowBytes;
+  float *out = c.scores + (size_t)b * c.max_cand + e0;
+  constexpr int kPerHalfWarp = MINMAX ? 8 : 16;          // entries of the segment per half-warp
+  constexpr int kPerGroup = kPerHalfWarp / 4;            // entries per half-warp and quarter
+  // The segment (or what the set has of it) comes in as four bulk copies (TMA), 16 KiB each, one
+  // mbarrier per copy, issued by one thread; the warps score a quarter as soon as its barrier
+  // completes, so a CTA keeps its whole 64 KiB in flight with four instructions.  Waits on the
+  // barriers are bounded (a copy that never lands is reported, not waited for).
+  __shared__ __align__(8) unsigned long long s_bar[4];
+  constexpr int kGroupEntries = 16 * kPerGroup;
+  const uint8_t *gseg = c.summaries + ((size_t)seg << c.sum_shift) * kEntry;
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int gI = 0; gI < 4; ++gI)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"((uint32_t)__cvta_generic_to_shared(&s_bar[gI])));
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // earlier generic accesses to the staging area
+#pragma unroll
+    for (int gI = 0; gI < 4; ++gI) {
+      const int first = gI * kGroupEntries, cnt = min(kGroupEntries, n_here - first);
+      if (cnt > 0) {
+        const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&s_bar[gI]), bytes = (uint32_t)cnt * kEntry;
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(dyn_smem + (size_t)first * kEntry);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                     ::"r"(dst), "l"(gseg + (size_t)first * kEntry), "r"(bytes), "r"(bar) : "memory");
+      }
+    }
+  }
   const int lane16 = threadIdx.x & 15, grp = threadIdx.x >> 4;
   // the two 16-lane rows of a warp may leave the loop at different times: each shuffles
   // only among its own lanes
@@ -147,43 +178,25 @@ __device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, con
     for (int j = 0; j < 4; ++j)
       qsel[g][j] = (qf[g][2 * j] >= 0.f ? 0x0000ffffu : 0u) | (qf[g][2 * j + 1] >= 0.f ? 0xffff0000u : 0u);
   }
-  const int n_here = min(seg_entries, n_cand - e0);
-  constexpr int kEntry = MINMAX ? 2 * kRowBytes : kRowBytes;
-  const uint8_t *base = c.summaries + ((size_t)seg << c.sum_shift) * kEntry + lane16 * 16;
-  float *out = c.scores + (size_t)b * c.max_cand + e0;
-
-  // Every lane requests, up front, the 16-byte pieces it will itself consume (cp.async into a
-  // per-CTA staging area, four groups per lane), then scores group by group as they land.
-  // A lane only ever reads what it copied, so waiting on its own groups is all the
-  // synchronisation there is, and a CTA keeps its whole 64 KiB segment in flight.
-  constexpr int kPerHalfWarp = MINMAX ? 8 : 16;          // entries of the segment per half-warp
-  constexpr int kPerGroup = kPerHalfWarp / 4;            // entries per cp.async group
-  uint8_t *stage = dyn_smem + (size_t)grp * kPerHalfWarp * kEntry + lane16 * 16;
+  __syncthreads();                                       // the initialised mbarriers are visible to all
+  uint8_t *stage = dyn_smem + lane16 * 16;
 #pragma unroll
   for (int gI = 0; gI < 4; ++gI) {
-#pragma unroll
-    for (int j = 0; j < kPerGroup; ++j) {
-      const int slot = gI * kPerGroup + j, e = grp + 16 * slot;
-      if (e < n_here) {
-        cp_async16_ca(stage + (size_t)slot * kEntry, base + (size_t)e * kEntry);
-        if (MINMAX) cp_async16_ca(stage + (size_t)slot * kEntry + kRowBytes, base + (size_t)e * kEntry + kRowBytes);
-      }
+    if (gI * kGroupEntries < n_here) {
+      const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&s_bar[gI]);
+      uint32_t done = 0;
+      for (int spin = 0; spin < (1 << 22) && !done; ++spin)
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(done) : "r"(bar) : "memory");
+      if (!done) { if (lane16 == 0) dev_error(c, kErrTimeout); }
     }
-    asm volatile("cp.async.commit_group;\n" ::: "memory");
-  }
-#pragma unroll
-  for (int gI = 0; gI < 4; ++gI) {
-    if (gI == 0) asm volatile("cp.async.wait_group 3;\n" ::: "memory");
-    else if (gI == 1) asm volatile("cp.async.wait_group 2;\n" ::: "memory");
-    else if (gI == 2) asm volatile("cp.async.wait_group 1;\n" ::: "memory");
-    else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
 #pragma unroll
     for (int j = 0; j < kPerGroup; ++j) {
       const int slot = gI * kPerGroup + j, e = grp + 16 * slot;
       if (e < n_here) {
-        const uint4 a0 = *reinterpret_cast<const uint4 *>(stage + (size_t)slot * kEntry);
-        const uint4 m0 = MINMAX ? *reinterpret_cast<const uint4 *>(stage + (size_t)slot * kEntry + kRowBytes)
+        const uint4 a0 = *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry);
+        const uint4 m0 = MINMAX ? *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry + kRowBytes)
                                 : make_uint4(0, 0, 0, 0);
+
         const float s0 = score_entry<G, MINMAX>(a0, m0, qf, qsel, row_mask);
         if (lane16 == 0) out[e] = s0;
       }
