@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 PAGE_BYTES = 8192
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
 # (profiles/), keyed by workload then kernel; None = not captured for this workload.
-NCU_TRAFFIC = {"c2": {"fetch": None, "score": 71.4e6, "attn_split": 65.9e6}}
+NCU_TRAFFIC = {"c2": {"fetch": None, "score": 71.1e6, "attn_split": 65.7e6}}
 
 
 def load_peaks():
