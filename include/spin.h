@@ -211,8 +211,8 @@ SPIN_API int spin_request_open(spin_ctx *ctx, int64_t hbm_budget_pages_per_set, 
  * waits for the device before and after.  The policy -- when to resize whom -- is the caller's
  * (the paper's scheduler); this is the mechanism. */
 SPIN_API int spin_set_budget(spin_ctx *ctx, int32_t req, int64_t hbm_budget_pages_per_set);
-/* Index during decode, cluster granularity (Section 4.1: Index is "invoked ... periodically in
- * decode to take in new tokens"; the paper leaves the rule to the algorithm).  Folds the FULL
+/* Index during decode, cluster granularity (Section 4.1 "Index": it also runs from time to time
+ * during decode so that new tokens are taken in; the rule is left to the algorithm).  Folds the FULL
  * pages of the local tail of every kv head's set of (request, layer) into the clusters: each
  * token, in arrival order, joins the cluster whose centroid scores highest against its key
  * (the fp32 summation order of Select, ties to the lower cluster id) and goes to the end of

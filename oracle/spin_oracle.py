@@ -26,7 +26,10 @@ Pins (tests marked "not gpu"): dense attention by an independent triple loop whe
 covers everything; a brute-force last-use LRU simulator; the closed form of a page's
 timestamp; a hand-derived worked example of the four LRU steps; page size 1 making the
 min/max bound equal the dot product bit for bit; the bound invariant q.k <= score(page);
-brute-force stable sort for top-k with ties.  Nothing in the paper prints a worked numeric
+brute-force stable sort for top-k with ties; the summaries a set builds at page fill rebuilt
+from the appended keys (per-channel extremes of the page's own 16 keys, a token's own key
+row) and the scores of a whole step checked against fp64 dot products of those keys; the
+order in which a group's heads are added, on values where the order changes the fp32 sum.  Nothing in the paper prints a worked numeric
 example, so absolute hit ratios and outputs are "parity unpinned" beyond those pins.
 """
 from __future__ import annotations
@@ -351,9 +354,9 @@ class OracleSet:
     def _index_tail_page(self):
         """The full tail page becomes partition #P (page and token granularity).
 
-        Reading (the paper says Index runs "periodically" during decode): a page becomes a
-        candidate when the first token of the next page arrives, so the newest page --
-        full or not -- is always the local tail.
+        Reading (the paper has Index run again from time to time during decode and gives no
+        period): a page becomes a candidate when the first token of the next page arrives, so
+        the newest page -- full or not -- is always the local tail.
         """
         page = self.tail_pages.pop()
         assert self.tail_len == self.T and not self.tail_pages
@@ -419,7 +422,7 @@ class OracleSet:
                 self.page_v[page, : rows.shape[0]] = v_bits[rows]
         self.n_tokens = int(k_bits.shape[0])
 
-    # ---- Index during decode, cluster granularity (Section 4.1: "invoked periodically") ------
+    # ---- Index during decode, cluster granularity (Section 4.1 "Index") ----------------------
     def reindex(self) -> List[Tuple[int, int]]:
         """Fold the full pages of the local tail into the clusters.
 
@@ -474,8 +477,8 @@ class OracleSet:
     def resize(self, new_slots: int) -> List[Tuple[int, int, int]]:
         """Change the set's number of GPU page table slots between steps.
 
-        Shrinking reclaims from the TAIL of the table ("we reclaim pages from the tail of the
-        GPU page table to keep the table compact"): slots new_slots.. disappear.  Reading (the
+        Shrinking reclaims from the TAIL of the table (Section 5.3: the tail is what is given
+        back, so that the table stays compact): slots new_slots.. disappear.  Reading (the
         paper does not say what happens to a partition that straddles the cut): a partition
         with any page in the reclaimed tail becomes non-resident as a whole, so its pages below
         the cut are cleared too.  Growing appends empty slots.  Timestamps of surviving pages

@@ -298,3 +298,91 @@ def test_reindex_with_a_full_newest_page_empties_the_tail_and_equal_scores_go_to
     assert [c for _, c in taken] == [1] * 16 and st.tail_pages == [] and st.tail_len == 0
     st.append_tokens(_bits(nk[:3]), _bits(nk[:3]))
     assert len(st.tail_pages) == 1 and st.tail_len == 3
+
+
+# ---- Index of a full tail page: the summaries the set builds from its own pages -------------
+# (Table 1, Index column; Section 4.1 "Index").  The checks below rebuild every summary from the
+# keys that were handed to append_tokens, never from the set's page store, so a summary taken
+# from the wrong page, the wrong rows or the wrong channel order fails them.
+
+def _distinct_keys(rng, n_tokens, d=128):
+    """bf16-exact keys, every token's row recognisable: small integers plus a per-token offset."""
+    base = rng.integers(-40, 41, size=(n_tokens, d)).astype(np.float32)
+    base += (np.arange(n_tokens, dtype=np.float32) % 7)[:, None]
+    return base                                                  # |x| <= 46: exact in bf16
+
+
+def _set_through_append(kind, keys, chunks, topk=3, slots=4, G=2):
+    cfg = O.OracleConfig(1, G, 1, 128, 16, kind, topk, 4)
+    st = O.OracleSet(cfg, slots)
+    kb = _bits(keys)
+    vb = _bits(np.zeros_like(keys))
+    i = 0
+    for m in chunks:                                             # ragged appends: prefill, then decode tokens
+        st.append_tokens(kb[i:i + m], vb[i:i + m])
+        i += m
+    assert i == keys.shape[0]
+    return st
+
+
+def test_minmax_summaries_are_the_per_channel_extremes_of_their_own_page():
+    rng = np.random.default_rng(21)
+    n = 16 * 6 + 9
+    keys = _distinct_keys(rng, n)
+    st = _set_through_append(O.PART_PAGE_MINMAX, keys, [16 * 2 + 3, 1, 1, 12, 16 * 3 + 1, 1, 1, 1, 1, 1, 2])
+    P = st.n_partitions()
+    assert P == 6 and st.tail_len == 9                           # the newest page is the tail, never a candidate
+    for p in range(P):
+        page = keys[16 * p:16 * p + 16]
+        assert np.array_equal(st.sum_min[p], page.min(axis=0)), p
+        assert np.array_equal(st.sum_max[p], page.max(axis=0)), p
+        assert st.part_tokens[p] == 16 and st.part_offset[p] == p
+
+
+def test_minmax_bound_holds_for_every_key_of_the_page_through_the_whole_step():
+    rng = np.random.default_rng(22)
+    G, n = 4, 16 * 8 + 5
+    keys = O.f32_to_bf16_f32(rng.standard_normal((n, 128)).astype(np.float32) * 3.0)
+    st = _set_through_append(O.PART_PAGE_MINMAX, keys, [n - 20] + [1] * 20, G=G)
+    for step in range(3):
+        q = O.f32_to_bf16_f32(rng.standard_normal((G, 128)).astype(np.float32))
+        _, tr = st.decode(_bits(q), want_output=False)
+        P = len(tr.scores)
+        assert P == 8
+        exact = (q.astype(np.float64) @ keys.astype(np.float64).T).sum(axis=0)      # sum_g q_g . k, per token
+        for p in range(P):
+            # the page's score bounds the summed dot product of each of ITS OWN keys ...
+            assert exact[16 * p:16 * p + 16].max() <= float(tr.scores[p]) * (1 + 1e-5) + 1e-4, (step, p)
+
+
+def test_minmax_score_is_attained_by_a_page_of_identical_keys():
+    # one page of 16 copies of the same row: min = max = that row, so the bound is the dot product
+    rng = np.random.default_rng(23)
+    G = 2
+    row = O.f32_to_bf16_f32(rng.standard_normal(128).astype(np.float32))
+    other = O.f32_to_bf16_f32(rng.standard_normal((16, 128)).astype(np.float32))
+    keys = np.concatenate([np.repeat(row[None], 16, axis=0), other, other[:3]])
+    st = _set_through_append(O.PART_PAGE_MINMAX, keys, [keys.shape[0]], G=G)
+    q = O.f32_to_bf16_f32(rng.standard_normal((G, 128)).astype(np.float32))
+    _, tr = st.decode(_bits(q), want_output=False)
+    want = float((q.astype(np.float64) @ row.astype(np.float64)).sum())
+    assert abs(float(tr.scores[0]) - want) <= 1e-5 * max(1.0, abs(want))
+    assert float(tr.scores[1]) >= float((q.astype(np.float64) @ other.astype(np.float64).T).sum(axis=0).max()) - 1e-4
+
+
+def test_token_summaries_are_the_tokens_own_key_rows_and_scores_their_dot_products():
+    rng = np.random.default_rng(24)
+    G, n = 2, 16 * 5 + 2
+    keys = _distinct_keys(rng, n)
+    st = _set_through_append(O.PART_TOKEN_DOT, keys, [16 * 3 + 15, 1, 1, 16, 1], topk=9, G=G)
+    P = st.n_partitions()
+    assert P == 5
+    assert np.array_equal(st.sum_vec[:P * 16], keys[:P * 16])    # row i of the summaries is token i's key
+    q = O.f32_to_bf16_f32(rng.standard_normal((G, 128)).astype(np.float32))
+    _, tr = st.decode(_bits(q), want_output=False)
+    want = (q.astype(np.float64) @ keys[:P * 16].astype(np.float64).T).sum(axis=0)
+    assert len(tr.scores) == P * 16
+    assert np.allclose(tr.scores.astype(np.float64), want, rtol=1e-5, atol=1e-3)
+    # and the selection is the brute-force top-9 of those dot products (distinct by construction)
+    order = sorted(range(P * 16), key=lambda i: (-float(tr.scores[i]), i))[:9]
+    assert list(tr.selected) == sorted(order)

@@ -78,6 +78,23 @@ def test_dot_score_matches_fp64_and_group_sum():
     assert np.allclose(s, ref, rtol=1e-5, atol=1e-4)
 
 
+def test_group_heads_are_added_in_ascending_order():
+    # per-head scores 2^24, 1, 1, -2^24 (one non-zero channel each, exact in bf16): ascending
+    # order gives ((2^24 + 1) + 1) + -2^24 = 0 in fp32 (each +1 is lost to rounding), the reverse
+    # order gives ((-2^24 + 1) + 1) + 2^24 = 2, a pairwise tree gives 0 + ... = different again
+    q = np.zeros((4, 128), dtype=F32)
+    q[0, 0], q[1, 0], q[2, 0], q[3, 0] = 2.0 ** 24, 1.0, 1.0, -(2.0 ** 24)
+    k = np.zeros((2, 128), dtype=F32)
+    k[0, 0] = 1.0
+    s = O.score_dot(q, k)
+    assert float(s[0]) == 0.0 and float(s[1]) == 0.0
+    s_rev = O.score_dot(q[::-1].copy(), k)
+    assert float(s_rev[0]) == 2.0
+    lo, hi = np.zeros((2, 128), dtype=F32), np.zeros((2, 128), dtype=F32)
+    lo[0, 0] = hi[0, 0] = 1.0
+    assert float(O.score_minmax(q, lo, hi)[0]) == 0.0 and float(O.score_minmax(q[::-1].copy(), lo, hi)[0]) == 2.0
+
+
 def test_negative_zero_is_canonicalised():
     q = np.full((1, 128), -1.0, dtype=F32)
     k = np.zeros((3, 128), dtype=F32)
