@@ -111,7 +111,7 @@ class Workload:
     lru_buckets: int
     steps: int
     drift: float                 # sigma of the per-step query drift
-    kv_recipe: str               # "normal" | "outlier" | "page_centre" | "mixture"
+    kv_recipe: str               # "normal" | "outlier" | "page_centre" | "mixture" | "tied"
     num_clusters: int = 0
     cluster_sd: float = 0.3
     outlier_channels: int = 0
@@ -120,6 +120,9 @@ class Workload:
     ctx_range: Optional[Tuple[int, int]] = None      # per-request context drawn uniformly
     drift_choices: Optional[Tuple[float, ...]] = None  # per-request drift drawn from these
     max_partition_pages: int = 1
+    tie_period: int = 0                              # "tied": token t carries the key of token t % tie_period
+    zero_run: Optional[Tuple[int, int]] = None       # "tied": tokens [a, b) have all-zero keys
+    tied_centroid_period: int = 0                    # > 0: cluster c carries the centroid of cluster c % period
 
     @property
     def group(self) -> int:
@@ -209,8 +212,10 @@ def _outlier_scale(w: Workload, layer: int, device) -> torch.Tensor:
 def centroids(w: Workload, req: int, layer: int, device="cpu") -> torch.Tensor:
     """Mixture centroids of one request: bf16 [num_clusters][num_kv_heads][head_dim]."""
     n = w.num_clusters * w.num_kv_heads * w.head_dim
-    c = normal(stream_key(w.seed, 3, req, layer), n, device)
-    return _bf16(c.view(w.num_clusters, w.num_kv_heads, w.head_dim))
+    c = normal(stream_key(w.seed, 3, req, layer), n, device).view(w.num_clusters, w.num_kv_heads, w.head_dim)
+    if w.tied_centroid_period > 0:
+        c = c[torch.arange(w.num_clusters, device=device) % w.tied_centroid_period]
+    return _bf16(c)
 
 
 def cluster_assignment(w: Workload, req: int, layer: int, n_tokens: int, device="cpu",
@@ -251,6 +256,15 @@ def kv_tokens(w: Workload, req: int, layer: int, first_token: int, n_tokens: int
         a = cluster_assignment(w, req, layer, n_tokens, device, first_token).long()
         hh = torch.arange(H, device=device).view(1, H).expand(n_tokens, H)
         k = cen[a, hh] + w.cluster_sd * zk
+    elif w.kv_recipe == "tied":
+        # duplicated keys: the key rows repeat with period `tie_period` tokens (a multiple of the
+        # page size makes whole pages repeat), and a run of tokens has all-zero keys; values stay
+        # distinct.  Candidates built from equal keys have equal summaries, whatever the rule.
+        tok = torch.arange(first_token, first_token + n_tokens, device=device)
+        src = normal(stream_key(w.seed, 1, req, layer), w.tie_period * row, device, 0).view(w.tie_period, H, d)
+        k = src[tok % w.tie_period]
+        if w.zero_run is not None:
+            k = torch.where(((tok >= w.zero_run[0]) & (tok < w.zero_run[1])).view(-1, 1, 1), torch.zeros_like(k), k)
     else:
         raise ValueError(w.kv_recipe)
     return _bf16(k), _bf16(zv)
