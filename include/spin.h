@@ -264,8 +264,18 @@ SPIN_API int spin_decode_step_append(spin_ctx *ctx, int32_t layer, const int32_t
                                      int32_t n_req, const void *k_new, const void *v_new,
                                      const void *q, void *out, void *cuda_stream);
 
-/* Counters and sticky device error bits.  Synchronises the device. */
+/* Counters and sticky device error bits.  Synchronises the device.  `out` is always filled; the
+ * status is SPIN_ERR_TIMEOUT (instead of SPIN_OK) when SPIN_DEV_ERR_TIMEOUT is among the bits:
+ * a kernel gave up a bounded wait, so results since then are void (the other bits report
+ * accesses that were skipped and leave the status at SPIN_OK). */
 SPIN_API int spin_stats(spin_ctx *ctx, spin_stats_t *out);
+
+/* Exercises the bounded-wait path (Section 5.3 keeps all control on the GPU, so kernels of a
+ * step wait on one another's flags; every such wait has a poll limit): one warp polls, at most
+ * `max_polls` times (1..4096, well under a millisecond), a flag word for a value that is never
+ * published, gives up, sets SPIN_DEV_ERR_TIMEOUT and returns.  Nothing else is touched; the
+ * context stays usable, the bit is sticky.  Asynchronous on cuda_stream. */
+SPIN_API int spin_debug_wait_probe(spin_ctx *ctx, int32_t max_polls, void *cuda_stream);
 
 /* Per-kernel timing (tracing aid, off by default).  spin_profile(ctx, 1) synchronises, clears
  * the record and makes every later append / decode call record a CUDA event after each kernel
@@ -300,9 +310,13 @@ SPIN_API int spin_debug_read_page(spin_ctx *ctx, int32_t req, int32_t layer, int
  * library image (every GPU that loads the library holds it until the process exits).
  *   q, out      bf16 [n_sets][group][128], device pointers (out is written)
  *   page_pool   device pointer to 8 KiB pages: 16 K rows then 16 V rows of 128 bf16
- *   page_ids    int32 [n_sets][list_stride], device: pages of each set, each id inside the pool
+ *   page_ids    int32 [n_sets][list_stride], device: pages of each set.  The call does not know
+ *               the pool's size: an id is only checked for being non-negative (a negative id is
+ *               skipped, its page contributes nothing); that ids lie inside the pool is the
+ *               caller's responsibility
  *   page_masks  uint32 [n_sets][list_stride], device: bit r set = token r of that page attended
- *   n_pages     int32 [n_sets], device: entries used per set (0..list_stride)
+ *   n_pages     int32 [n_sets], device: entries used per set; values outside 0..list_stride are
+ *               clamped into that range.  A set without pages gets a zero output
  *   group       query heads per set: 1, 2, 4 or 8;  sm_scale 0 = 1/sqrt(128)
  * Limit: n_sets x ceil(list_stride/8) x group x 130 + n_sets (rounded up to 64) <= 2097152
  * four-byte words; a larger request is refused with SPIN_ERR_INVALID and a message on stderr,

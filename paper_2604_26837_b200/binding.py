@@ -24,9 +24,9 @@ PAGE_BYTES = 8192
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open", "spin_reindex",
            "spin_request_close", "spin_set_budget", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
            "spin_decode_step_append", "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
-           "spin_debug_read_page", "spin_paged_attention_static", "spin_last_error",
+           "spin_debug_read_page", "spin_debug_wait_probe", "spin_paged_attention_static", "spin_last_error",
            "spin_version"]
-KERNEL_NAMES = ["append", "score", "topk", "cache", "fetch", "attn_split", "attn_merge"]
+KERNEL_NAMES = ["append", "score", "topk", "cache", "fetch", "attn_split", "unused"]
 
 
 class SpinError(RuntimeError):
@@ -115,6 +115,7 @@ def load() -> C.CDLL:
     lib.spin_profile_read.argtypes = [vp, C.POINTER(spin_profile_t)]
     lib.spin_debug_dump.argtypes = [vp, i32, i32, i32, C.POINTER(spin_dump_t)]
     lib.spin_debug_read_page.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
+    lib.spin_debug_wait_probe.argtypes = [vp, i32, vp]
     lib.spin_paged_attention_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
     lib.spin_last_error.argtypes = [vp]
     lib.spin_last_error.restype = C.c_char_p
@@ -261,10 +262,16 @@ class Spin:
     def stats(self) -> dict:
         s = spin_stats_t()
         s.struct_size = C.sizeof(spin_stats_t)
-        self._ck(self.lib.spin_stats(self.h, C.byref(s)))
+        rc = self.lib.spin_stats(self.h, C.byref(s))
+        if rc not in (0, 7):                     # SPIN_ERR_TIMEOUT still fills the counters: see "status"
+            self._ck(rc)
         out = {n: getattr(s, n) for n, _ in spin_stats_t._fields_ if n not in ("struct_size", "debug_words")}
         out["debug_words"] = list(s.debug_words)
+        out["status"] = rc
         return out
+
+    def debug_wait_probe(self, max_polls: int, stream=None):
+        self._ck(self.lib.spin_debug_wait_probe(self.h, max_polls, _stream_ptr(stream)))
 
     def profile(self, enable: bool):
         self._ck(self.lib.spin_profile(self.h, 1 if enable else 0))

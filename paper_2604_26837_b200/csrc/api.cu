@@ -409,6 +409,47 @@ int wait_for_offload(spin_ctx *ctx, cudaStream_t st) {
   return SPIN_OK;
 }
 
+// One more token for each listed request of one layer: everything that could make grow_paged /
+// grow_cluster_tail fail is checked here for the whole batch, before any of them runs, so that
+// a refused call leaves the host's counts (and with them the device's) untouched.
+int precheck_append_one(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32_t n_req) {
+  const Geometry &g = ctx->g;
+  const bool cluster = ctx->cfg.partition_kind == SPIN_PART_CLUSTER_CENTROID;
+  int64_t new_pages = 0, cpt = 0, meta = 0, off = 0, sum = 0;      // host pages and table segments the batch needs
+  auto unmapped = [](const std::vector<int32_t> &dir, int64_t idx, int shift) {
+    const size_t di = (size_t)(idx >> shift);
+    return di < dir.size() && dir[di] < 0 ? 1 : 0;
+  };
+  for (int i = 0; i < n_req; ++i) {
+    const LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
+    if (cluster && !L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req_ids[i]);
+    if (L.n_tokens + 1 > ctx->cfg.max_context_tokens)
+      return fail(ctx, SPIN_ERR_INVALID, "request %d exceeds max_context_tokens", req_ids[i]);
+    const bool page_starts = cluster ? (L.tail_pages == 0 || L.tail_len == kPageTokens) : L.n_tokens % kPageTokens == 0;
+    if (!page_starts) continue;
+    if (cluster && L.tail_pages + 1 > g.tail_cap) return fail(ctx, SPIN_ERR_INVALID, "request %d exceeds max_tail_tokens", req_ids[i]);
+    new_pages += ctx->cfg.num_kv_heads;
+    for (int h = 0; h < ctx->cfg.num_kv_heads; ++h) {
+      const SetHost &S = set_of(ctx, req_ids[i], layer, h);
+      const int64_t j = cluster ? (int64_t)L.tail_first + L.tail_pages : L.n_tokens / kPageTokens;   // the new page
+      cpt += unmapped(S.dir_cpt, j, g.seg_shift);
+      if (!cluster && j > L.n_partitions) {
+        // the page before it becomes a candidate: one entry in the partition tables, its summaries
+        const int64_t p = j - 1;
+        meta += unmapped(S.dir_meta, p, g.seg_shift);
+        off += unmapped(S.dir_off, p, g.seg_shift);
+        sum += unmapped(S.dir_sum, ctx->cfg.partition_kind == SPIN_PART_TOKEN_DOT ? p * kPageTokens : p, g.sum_shift);
+      }
+    }
+  }
+  if (ctx->host_page_pool.available() < new_pages) return fail(ctx, SPIN_ERR_OOM_HOST, "out of host pages");
+  if (ctx->cpt_segs.available() < cpt) return fail(ctx, SPIN_ERR_OOM_HOST, "out of CPU page table segments");
+  if (ctx->off_segs.available() < off) return fail(ctx, SPIN_ERR_OOM_HOST, "out of Partition Offset segments");
+  if (ctx->meta_segs.available() < meta) return fail(ctx, SPIN_ERR_OOM_DEVICE, "out of Meta-partition segments");
+  if (ctx->sum_segs.available() < sum) return fail(ctx, SPIN_ERR_OOM_DEVICE, "out of summary segments");
+  return SPIN_OK;
+}
+
 int append_paged_device(spin_ctx *ctx, int req, int layer, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                         int64_t n, cudaStream_t st) {
   LayerHost &L = ctx->reqs[(size_t)req].layers[(size_t)layer];
@@ -1142,15 +1183,18 @@ int spin_append_kv_batch(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, i
     a.req[i] = req_ids[i];
   }
   const bool cluster = ctx->cfg.partition_kind == SPIN_PART_CLUSTER_CENTROID;
+  const bool k_dev = is_device_ptr(k);
+  if (k_dev != is_device_ptr(v)) return fail(ctx, SPIN_ERR_INVALID, "k and v must both be device or both be host pointers");
+  if (int rc = precheck_append_one(ctx, layer, req_ids, n_req)) return rc;
+  // all checks passed: from here on the call changes state
   for (int i = 0; i < n_req; ++i) {
     LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
-    if (cluster && !L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req_ids[i]);
     int rc = cluster ? grow_cluster_tail(ctx, req_ids[i], layer, 1, st) : grow_paged(ctx, req_ids[i], layer, L.n_tokens + 1, st);
     if (rc) return rc;
     a.n_tokens[i] = (int32_t)(L.n_tokens - 1);
   }
   const __nv_bfloat16 *kk = reinterpret_cast<const __nv_bfloat16 *>(k), *vv = reinterpret_cast<const __nv_bfloat16 *>(v);
-  if (!is_device_ptr(k)) {
+  if (!k_dev) {
     const size_t bytes = (size_t)n_req * ctx->cfg.num_kv_heads * kRowBytes;
     CK(cudaMemcpyAsync(ctx->stage_k, k, bytes, cudaMemcpyHostToDevice, st));
     CK(cudaMemcpyAsync(ctx->stage_v, v, bytes, cudaMemcpyHostToDevice, st));
@@ -1189,8 +1233,15 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
   const size_t qbytes = (size_t)n_req * ctx->cfg.num_q_heads * kRowBytes;
   bool in_grid = false, kv_pinned = false;
   // q and new k/v in pinned host memory: one zero-copy staging kernel brings them in
-  if (int rc = wait_for_offload(ctx, st)) return rc;       // missed pages are fetched from the host tier
   const int qc = classify_ptr(q, &q_alias), oc = classify_ptr(out, &out_alias);
+  int kc = 0;
+  if (with_append) {
+    // every check comes before the first change of state: a refused call leaves the context as it was
+    kc = classify_ptr(k, &k_alias);
+    if (kc != classify_ptr(v, &v_alias)) return fail(ctx, SPIN_ERR_INVALID, "k_new and v_new must live in the same kind of memory");
+    if (int rc = precheck_append_one(ctx, layer, req_ids, n_req)) return rc;
+  }
+  if (int rc = wait_for_offload(ctx, st)) return rc;       // missed pages are fetched from the host tier
   if (with_append) {
     for (int i = 0; i < n_req; ++i) {
       LayerHost &L = ctx->reqs[(size_t)req_ids[i]].layers[(size_t)layer];
@@ -1199,8 +1250,6 @@ static int step_impl(spin_ctx *ctx, int32_t layer, const int32_t *req_ids, int32
     }
     kk = reinterpret_cast<const __nv_bfloat16 *>(k);
     vv = reinterpret_cast<const __nv_bfloat16 *>(v);
-    const int kc = classify_ptr(k, &k_alias), vc = classify_ptr(v, &v_alias);
-    if (kc != vc) return fail(ctx, SPIN_ERR_INVALID, "k_new and v_new must live in the same kind of memory");
     if (kc == 2) {
       CK(cudaMemcpyAsync(ctx->stage_k, k, kv_bytes, cudaMemcpyHostToDevice, st));
       CK(cudaMemcpyAsync(ctx->stage_v, v, kv_bytes, cudaMemcpyHostToDevice, st));
@@ -1307,6 +1356,16 @@ int spin_stats(spin_ctx *ctx, spin_stats_t *out) {
   out->summary_bytes = (uint64_t)ctx->sum_segs.in_use * g.sum_entries * g.sum_entry_bytes;
   out->gpu_pages_in_use = (uint64_t)ctx->gpu_page_pool.in_use;
   out->host_pages_in_use = (uint64_t)ctx->host_page_pool.in_use;
+  if (c.error_bits & kErrTimeout)
+    return fail(ctx, SPIN_ERR_TIMEOUT, "a bounded device-side wait ran out (first check that tripped: %u)", c.first_site);
+  return SPIN_OK;
+}
+
+int spin_debug_wait_probe(spin_ctx *ctx, int32_t max_polls, void *cuda_stream) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  if (max_polls < 1 || max_polls > 4096) return fail(ctx, SPIN_ERR_INVALID, "max_polls must be 1..4096");
+  ctx->launches += launch_wait_probe(ctx->d, max_polls, reinterpret_cast<cudaStream_t>(cuda_stream));
+  CK(cudaGetLastError());
   return SPIN_OK;
 }
 

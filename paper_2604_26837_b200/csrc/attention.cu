@@ -190,7 +190,7 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
       int ok = flag_wait(c, c.ready1 + b, bt.epoch);
       int np_ = 0, nm_ = 0;
       if (ok) {
-        np_ = c.n_pages[b]; nm_ = c.n_miss[b];
+        np_ = max(0, min(c.n_pages[b], c.max_pages + c.tail_cap)); nm_ = c.n_miss[b];
         if (first < np_ && min(np_, first + kChunkPages) > nm_)
           ok = flag_wait(c, c.ready + b, bt.epoch) && flag_wait(c, c.tail_ready + b, bt.epoch);
       }
@@ -203,7 +203,9 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
     pdl_wait_prev();
   }
   if (chunk == 0) dbg_ta(b, 10);
-  const int np = c.n_pages[b];
+  // a count beyond the list's stride can neither read past the set's row nor leave the merge
+  // waiting for chunks that no CTA of the grid owns
+  const int np = max(0, min(c.n_pages[b], c.max_pages + c.tail_cap));
   if (first >= np) return;
   const int last = min(np, first + kChunkPages);
   const int i_req = b / c.Hkv, head = b % c.Hkv;
@@ -337,49 +339,76 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
   if (!sh_last) return;
   dbg_ta(b, 14);
   __threadfence();
-  // merge: the per-chunk (max, sum) pairs first, then the outputs, with the loads of a batch
-  // of chunks issued together
+  // merge.  Nothing here grows with the number of chunks: the per-chunk (max, sum) pairs are
+  // reduced to the set's max and denominator first (a thread's pairs all belong to one head,
+  // the stride being a multiple of the group), then the outputs are accumulated over tiles of
+  // kMergeTile chunks whose weights exp2(m_k - m) sit in shared memory.
+  constexpr int kThreads = kAttnWarps * 32, kMergeTile = 512;
   const float *parts = c.att_part + (size_t)b * c.max_chunks * G * kPartStride;
-  float *s_scale = reinterpret_cast<float *>(smem_pages);         // [n_chunks][G] weights exp2(m_k - m)
-  float *s_m = s_scale + (size_t)n_chunks * G;                    // [n_chunks][G]
-  float *s_l = s_m + (size_t)n_chunks * G;                        // [n_chunks][G]
-  float *s_den = s_l + (size_t)n_chunks * G;                      // [G]
-  for (int e = threadIdx.x; e < n_chunks * G; e += kAttnWarps * 32) {
-    const int k = e / G, g = e % G;
-    const float *pp = parts + ((size_t)k * G + g) * kPartStride;
-    s_m[e] = __ldcg(pp + kHeadDim);
-    s_l[e] = __ldcg(pp + kHeadDim + 1);
-  }
-  __syncthreads();
-  if (threadIdx.x < G) {
-    const int g = threadIdx.x;
-    float mn = -INFINITY;
-    for (int k = 0; k < n_chunks; ++k) mn = fmaxf(mn, s_m[k * G + g]);
+  float *s_red = reinterpret_cast<float *>(smem_pages);           // [kThreads]
+  float *s_mx = s_red + kThreads;                                 // [G] the set's max per head
+  float *s_den = s_mx + G;                                        // [G]
+  float *s_scale = s_den + G;                                     // [kMergeTile][G]
+  {
+    float mx = -INFINITY;
+    for (int e = threadIdx.x; e < n_chunks * G; e += kThreads)
+      mx = fmaxf(mx, __ldcg(parts + (size_t)e * kPartStride + kHeadDim));
+    s_red[threadIdx.x] = mx;
+    __syncthreads();
+    if (threadIdx.x < G) {
+      float m_ = -INFINITY;
+      for (int i = threadIdx.x; i < kThreads; i += G) m_ = fmaxf(m_, s_red[i]);
+      s_mx[threadIdx.x] = m_;
+    }
+    __syncthreads();
+    const float mn = s_mx[threadIdx.x % G];
     float den = 0.f;
-    for (int k = 0; k < n_chunks; ++k) {
-      const float mk = s_m[k * G + g];
-      const float a = mk == -INFINITY ? 0.f : exp2f(mk - mn);
-      s_scale[k * G + g] = a;
-      den += s_l[k * G + g] * a;
+    for (int e = threadIdx.x; e < n_chunks * G; e += kThreads) {
+      const float *pp = parts + (size_t)e * kPartStride;
+      const float mk = __ldcg(pp + kHeadDim);
+      den += mk == -INFINITY ? 0.f : __ldcg(pp + kHeadDim + 1) * exp2f(mk - mn);
     }
-    s_den[g] = den;
+    s_red[threadIdx.x] = den;
+    __syncthreads();
+    if (threadIdx.x < G) {
+      float d_ = 0.f;
+      for (int i = threadIdx.x; i < kThreads; i += G) d_ += s_red[i];
+      s_den[threadIdx.x] = d_;
+    }
   }
-  __syncthreads();
-  for (int e = threadIdx.x; e < G * kHeadDim; e += kAttnWarps * 32) {
-    const int g = e / kHeadDim, ch = e % kHeadDim;
-    const float *pg_ = parts + g * kPartStride + ch;
-    float a_o = 0.f;
-    int k = 0;
-    for (; k + 8 <= n_chunks; k += 8) {
-      float v[8];
+  float a_o[G];                                                   // this thread's outputs: e = tid + j * kThreads
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = __ldcg(pg_ + (size_t)(k + j) * G * kPartStride);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) a_o = fmaf(v[j], s_scale[(k + j) * G + g], a_o);
+  for (int j = 0; j < G; ++j) a_o[j] = 0.f;
+  for (int k0 = 0; k0 < n_chunks; k0 += kMergeTile) {
+    const int kn = min(kMergeTile, n_chunks - k0);
+    __syncthreads();                                              // the previous tile's weights have been used
+    for (int e = threadIdx.x; e < kn * G; e += kThreads) {
+      const float mk = __ldcg(parts + ((size_t)k0 * G + e) * kPartStride + kHeadDim);
+      s_scale[e] = mk == -INFINITY ? 0.f : exp2f(mk - s_mx[e % G]);
     }
-    for (; k < n_chunks; ++k) a_o = fmaf(__ldcg(pg_ + (size_t)k * G * kPartStride), s_scale[k * G + g], a_o);
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < G; ++j) {
+      const int e = threadIdx.x + j * kThreads, g = e / kHeadDim, ch = e % kHeadDim;
+      const float *pg_ = parts + ((size_t)k0 * G + g) * kPartStride + ch;
+      float acc = a_o[j];
+      int k = 0;
+      for (; k + 8 <= kn; k += 8) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = __ldcg(pg_ + (size_t)(k + i) * G * kPartStride);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc = fmaf(v[i], s_scale[(k + i) * G + g], acc);
+      }
+      for (; k < kn; ++k) acc = fmaf(__ldcg(pg_ + (size_t)k * G * kPartStride), s_scale[k * G + g], acc);
+      a_o[j] = acc;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < G; ++j) {
+    const int e = threadIdx.x + j * kThreads, g = e / kHeadDim, ch = e % kHeadDim;
     const float den = s_den[g];
-    out[((size_t)i_req * c.Hq + head * G + g) * kHeadDim + ch] = __float2bfloat16(den > 0.f ? a_o / den : 0.f);
+    out[((size_t)i_req * c.Hq + head * G + g) * kHeadDim + ch] = __float2bfloat16(den > 0.f ? a_o[j] / den : 0.f);
   }
 }
 
@@ -399,7 +428,7 @@ k_attn(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *_
 // Sets whose page list is empty get a zero output (no CTA of k_attn reaches them).
 __global__ void k_attn_zero_empty(DevCtx c, __nv_bfloat16 *__restrict__ out, int n_sets) {
   const int b = blockIdx.x;
-  if (b >= n_sets || c.n_pages[b] != 0) return;
+  if (b >= n_sets || c.n_pages[b] > 0) return;
   const int i_req = b / c.Hkv, head = b % c.Hkv;
   for (int e = threadIdx.x; e < c.G * kHeadDim; e += blockDim.x)
     out[((size_t)i_req * c.Hq + head * c.G) * kHeadDim + e] = __float2bfloat16(0.f);
@@ -408,7 +437,8 @@ __global__ void k_attn_zero_empty(DevCtx c, __nv_bfloat16 *__restrict__ out, int
 template <int G>
 void launch_attn_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, __nv_bfloat16 *out, dim3 grid,
                    cudaStream_t st) {
-  static bool configured = false;
+  static bool configured_dev[kMaxDevices] = {};
+  bool &configured = configured_dev[current_device_slot()];
   constexpr int smem = kChunkPages * kPageBytes;
   if (!configured) {
     cudaFuncSetAttribute(k_attn<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -453,7 +483,6 @@ namespace spin {
 namespace {
 constexpr size_t kStaticPartialFloats = (size_t)2 << 20;                  // 8 MiB of fp32
 __device__ __align__(256) static float g_static_partials[kStaticPartialFloats];
-constexpr int kMaxDevices = 64;
 float *g_static_partials_addr[kMaxDevices] = {};                          // per device, set up once
 }  // namespace
 }  // namespace spin

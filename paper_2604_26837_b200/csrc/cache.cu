@@ -108,7 +108,8 @@ k_fetch(DevCtx c) {
 size_t cache_smem_bytes(const DevCtx &c) { return cache_stage_smem_bytes(c.max_parts, c.max_pages, c.max_slots); }
 
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
-  static size_t configured = 0;
+  static size_t configured_dev[kMaxDevices] = {};
+  size_t &configured = configured_dev[current_device_slot()];
   int tbl_cap = 0;
   size_t smem = 0;
   // one CTA per set: the snapshot of the partition tables may take what shared memory is left
@@ -120,6 +121,19 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof) {
   }
   launch_pdl(k_cache, dim3(b.n_req * c.Hkv), dim3(kCacheThreads), smem, st, 1, c, b, fast, tbl_cap);
   prof_mark(prof, st, kProfCache);
+  return 1;
+}
+
+// One warp waits, with the given poll limit, for a value that no kernel ever publishes (a
+// negative call number) in the first set's `scored` word: the wait runs out, the timeout bit is
+// set and the kernel returns.  This is how the bounded-wait path is exercised without any
+// other kernel misbehaving.
+__global__ void k_wait_probe(DevCtx c, int max_polls) {
+  if (threadIdx.x == 0) flag_wait(c, c.scored, -1, max_polls);
+}
+
+int launch_wait_probe(const DevCtx &c, int max_polls, cudaStream_t st) {
+  k_wait_probe<<<1, 32, 0, st>>>(c, max_polls);
   return 1;
 }
 

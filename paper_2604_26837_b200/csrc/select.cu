@@ -107,7 +107,8 @@ struct ScoreGrid {
 template <int G, bool MINMAX>
 __device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, const __nv_bfloat16 *__restrict__ q,
                                            const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
-                                           int fuse, int keys_cap, int tbl_cap, int b, int x, uint8_t *dyn_smem) {
+                                           int fuse, int keys_cap, int tbl_cap, int b, int x, uint8_t *dyn_smem,
+                                           unsigned long long *s_bar, uint32_t &phase_bits, const int *s_dead_in, int *s_dead) {
   const int i_req = b / c.Hkv, head = b % c.Hkv;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
   if (x < 0) {
@@ -139,16 +140,18 @@ __device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, con
   constexpr int kPerGroup = kPerHalfWarp / 4;            // entries per half-warp and quarter
   // The segment (or what the set has of it) comes in as four bulk copies (TMA), 16 KiB each, one
   // mbarrier per copy, issued by one thread; the warps score a quarter as soon as its barrier
-  // completes, so a CTA keeps its whole 64 KiB in flight with four instructions.  Waits on the
-  // barriers are bounded (a copy that never lands is reported, not waited for).
-  __shared__ __align__(8) unsigned long long s_bar[4];
+  // completes, so a CTA keeps its whole 64 KiB in flight with four instructions.  The four
+  // barriers are initialised once per CTA (by the kernel); a CTA that works on several items
+  // carries one phase bit per barrier from item to item (phase_bits, uniform over the CTA).
+  // Waits on the barriers are bounded: a copy that never lands is reported (the quarter is then
+  // scored from whatever the staging area holds: the error bit says that this step's results are
+  // void), and from its next item on the CTA scores nothing (its barriers' phases are no longer
+  // known, and the copy may still be writing the staging area): it only counts its arrivals.
+  // That decision is uniform over the CTA, so the rows' shuffles never lose a lane.
   constexpr int kGroupEntries = 16 * kPerGroup;
   const uint8_t *gseg = c.summaries + ((size_t)seg << c.sum_shift) * kEntry;
-  if (threadIdx.x == 0) {
-#pragma unroll
-    for (int gI = 0; gI < 4; ++gI)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"((uint32_t)__cvta_generic_to_shared(&s_bar[gI])));
-    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  const bool dead = *s_dead_in != 0;
+  if (threadIdx.x == 0 && !dead) {
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // earlier generic accesses to the staging area
 #pragma unroll
     for (int gI = 0; gI < 4; ++gI) {
@@ -178,21 +181,21 @@ __device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, con
     for (int j = 0; j < 4; ++j)
       qsel[g][j] = (qf[g][2 * j] >= 0.f ? 0x0000ffffu : 0u) | (qf[g][2 * j + 1] >= 0.f ? 0xffff0000u : 0u);
   }
-  __syncthreads();                                       // the initialised mbarriers are visible to all
   uint8_t *stage = dyn_smem + lane16 * 16;
 #pragma unroll
   for (int gI = 0; gI < 4; ++gI) {
-    if (gI * kGroupEntries < n_here) {
-      const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&s_bar[gI]);
+    if (gI * kGroupEntries < n_here && !dead) {
+      const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&s_bar[gI]), parity = (phase_bits >> gI) & 1u;
       uint32_t done = 0;
       for (int spin = 0; spin < (1 << 22) && !done; ++spin)
-        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(done) : "r"(bar) : "memory");
-      if (!done) { if (lane16 == 0) dev_error(c, kErrTimeout); }
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+      if (!done) { *s_dead = 1; if (lane16 == 0) dev_error(c, kErrTimeout); }
+      phase_bits ^= 1u << gI;
     }
 #pragma unroll
     for (int j = 0; j < kPerGroup; ++j) {
       const int slot = gI * kPerGroup + j, e = grp + 16 * slot;
-      if (e < n_here) {
+      if (e < n_here && !dead) {
         const uint4 a0 = *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry);
         const uint4 m0 = MINMAX ? *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry + kRowBytes)
                                 : make_uint4(0, 0, 0, 0);
@@ -245,13 +248,21 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
   pdl_launch_next();
   pdl_wait_prev();
   __shared__ int s_item[2];
+  __shared__ __align__(8) unsigned long long s_bar[4];     // one per quarter of the staged segment
+  __shared__ int s_dead[2];                                // [0] read at an item's start, [1] set by a wait that ran out
+  uint32_t phase_bits = 0;
   const bool pers = sg.persistent != 0;
-  if (pers) {
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int gI = 0; gI < 4; ++gI)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"((uint32_t)__cvta_generic_to_shared(&s_bar[gI])));
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    s_dead[0] = s_dead[1] = 0;
     // the first item is the CTA's own number (no storm on the counter at the start); the queue
     // hands out the items from gridDim.x on
-    if (threadIdx.x == 0) s_item[0] = (int)blockIdx.x;
-    __syncthreads();
+    s_item[0] = (int)blockIdx.x;
   }
+  __syncthreads();                                         // the initialised mbarriers are visible to all
   for (int it = 0;; ++it) {
     const int item = pers ? s_item[it & 1] : (int)blockIdx.x;
     if (item >= sg.n_items) break;
@@ -270,9 +281,9 @@ k_score(DevCtx c, Batch bt, const __nv_bfloat16 *__restrict__ q, const __nv_bflo
       b = lo * c.Hkv + off / segs_r;
       x = off % segs_r;
     }
-    score_item<G, MINMAX>(c, bt, q, k_new, v_new, fuse, keys_cap, tbl_cap, b, x, dyn_smem);
+    score_item<G, MINMAX>(c, bt, q, k_new, v_new, fuse, keys_cap, tbl_cap, b, x, dyn_smem, s_bar, phase_bits, &s_dead[0], &s_dead[1]);
     if (!pers) return;
-    if (threadIdx.x == 0) s_item[(it + 1) & 1] = next;
+    if (threadIdx.x == 0) { s_item[(it + 1) & 1] = next; if (s_dead[1]) s_dead[0] = 1; }
     __syncthreads();
   }
   // the last CTA out leaves the queue ready for the next step (every other CTA has drawn its
@@ -340,7 +351,8 @@ k_topk(DevCtx c, Batch bt, int keys_cap, int manage, int tbl_cap, int wait_flags
 
 
 int sm_count_of_device() {
-  static int sms = 0;
+  static int sms_dev[kMaxDevices] = {};
+  int &sms = sms_dev[current_device_slot()];
   if (!sms) {
     int dev = 0;
     cudaGetDevice(&dev);
@@ -354,7 +366,8 @@ template <int G>
 void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, const __nv_bfloat16 *k_new,
                     const __nv_bfloat16 *v_new, dim3 grid, size_t smem, int fuse, int keys_cap, int tbl_cap,
                     const ScoreGrid &sg, cudaStream_t st) {
-  static size_t configured = 0;
+  static size_t configured_dev[kMaxDevices] = {};
+  size_t &configured = configured_dev[current_device_slot()];
   if (smem > configured) {
     cudaFuncSetAttribute(k_score<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     cudaFuncSetAttribute(k_score<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -363,8 +376,10 @@ void launch_score_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, con
   if (sg.persistent) {
     // the resident grid: what fits on the GPU at this shared-memory size, less one CTA on 32
     // SMs (attention CTAs take that room from the start)
-    static size_t occ_smem = ~(size_t)0;
-    static int occ[2] = {1, 1};
+    static size_t occ_smem_dev[kMaxDevices] = {};
+    static int occ_dev[kMaxDevices][2] = {};
+    size_t &occ_smem = occ_smem_dev[current_device_slot()];
+    int (&occ)[2] = occ_dev[current_device_slot()];
     if (smem != occ_smem) {
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ[1], k_score<G, true>, kScoreThreads, smem);
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ[0], k_score<G, false>, kScoreThreads, smem);
@@ -449,7 +464,8 @@ int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_
     while (C < 8 && (max_cand + C - 1) / C > 8192) C *= 2;
     int kc = (max_cand + C - 1) / C;
     if (kc > 16384) kc = 0;                              // too many for shared memory: re-read from L2
-    static int smem_set = 0;
+    static int smem_set_dev[kMaxDevices] = {};
+    int &smem_set = smem_set_dev[current_device_slot()];
     int ksmem = kc * 4;
     // the cache manager runs in the same kernel when it can work on shared-memory copies
     if (manage) ksmem = ((ksmem + 15) & ~15) + (int)mgr_smem;    // the manager's tables sit behind the keys

@@ -144,6 +144,7 @@ __host__ __device__ inline int set_index(const DevCtx &c, int req, int layer, in
 // Records the error bits and, for the first error only, where it was raised (source file id *
 // 100000 + line), so that a sticky bit can be traced to its check.
 __device__ __forceinline__ void dev_error_site(const DevCtx &c, unsigned bits, unsigned site) {
+  if (!c.counters) return;                       // a caller without a context has no status words
   atomicOr(&c.counters->error_bits, bits);
   atomicCAS(&c.counters->first_site, 0u, site);
 }
@@ -217,12 +218,14 @@ __device__ __forceinline__ void flag_publish(int32_t *flag, int32_t value) {
   // before the call: the other threads' writes too) is visible to whoever acquires the flag
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
-__device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, int32_t value) {
+constexpr int kFlagWaitPolls = 1 << 19;          // ~0.1 s of polls at the capped back-off
+__device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, int32_t value,
+                                          int max_polls = kFlagWaitPolls) {
   // polls back off from 32 ns to 256 ns: hundreds of waiting CTAs should not keep the L2
   // lines of the flags busy, and a raised flag should still be seen within a fraction of a
   // microsecond
   unsigned pause = 32;
-  for (int spin = 0; spin < (1 << 19); ++spin) {
+  for (int spin = 0; spin < max_polls; ++spin) {
     int32_t v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (v == value) return true;
@@ -237,6 +240,16 @@ __device__ __forceinline__ const uint8_t *page_ptr(const DevCtx &c, int src) {
   return src >= 0 ? c.gpu_pages + (size_t)src * kPageBytes : c.host_pages + (size_t)(~src) * kPageBytes;
 }
 #endif
+
+// Function attributes (opt-in shared memory), occupancy and SM counts are properties of a device:
+// what a launcher remembers about them is kept per device ordinal (the current device, which a
+// launcher's caller has made the stream's device).
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+  return dev % kMaxDevices;
+}
 
 // Optional per-kernel timing: an event after every launch; durations are read afterwards.
 enum : int { kProfAppend = 0, kProfScore, kProfTopk, kProfCache, kProfFetch, kProfAttnSplit,
@@ -300,6 +313,7 @@ int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_
 int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
 int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
 int launch_shrink(const DevCtx &c, int req, int old_S, int new_S, cudaStream_t st);
+int launch_wait_probe(const DevCtx &c, int max_polls, cudaStream_t st);
 int launch_assign(const DevCtx &c, int req, int layer, int n_clusters, int n_tokens, int32_t *assign, cudaStream_t st);
 int launch_move_rows(const DevCtx &c, int req, int layer, const int64_t *dest, int n_tokens, cudaStream_t st);
 int launch_reindex_apply(const DevCtx &c, int req, int layer, int n_clusters, int n_folded_pages, int tail_first,

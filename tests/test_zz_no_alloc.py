@@ -5,7 +5,10 @@ component's fixed memory budget, or on a path where the allocator must not be to
 they cannot build a context.  For them the library carries its split-K scratch as a built-in
 array.  This test drives the entry point through the C ABI with page lists taken from a
 normal decode step and checks, on two calls in a row (the second reuses the array with the
-first call's leftovers in it), that the output matches spin_decode_step's.
+first call's leftovers in it), that the output matches spin_decode_step's; further cases
+(full and empty lists, one page, chunk boundaries, groups of 1 and 8, hundreds of chunks)
+compare it with the CPU oracle's fp64 attention over the same rows.  Only well-formed inputs
+are used.
 """
 import numpy as np
 import pytest
@@ -94,3 +97,73 @@ def test_static_attention_matches_decode_step_twice_in_a_row():
                                        q_sets, torch.cuda.current_stream())
     assert rc == 1
     run.close()
+
+
+def _static_case(group, counts, stride, seed, n_pool_pages=None, sm_scale=0.0):
+    """Random pool, lists and masks -> (library output, fp64 reference) for one call."""
+    import paper_2604_26837_b200 as P
+    from oracle import spin_oracle as O
+    dev, T, d = "cuda:0", 16, 128
+    n_sets = len(counts)
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    n_pool = n_pool_pages or (sum(counts) + 3)
+    pool = torch.randn(n_pool, 2, T, d, generator=g).to(torch.bfloat16)
+    q = torch.randn(n_sets, group, d, generator=g).to(torch.bfloat16)
+    rng = np.random.default_rng(seed)
+    ids = np.full((n_sets, stride), -1, dtype=np.int32)              # unused entries are never read
+    masks = np.zeros((n_sets, stride), dtype=np.uint32)
+    perm = rng.permutation(n_pool)
+    at = 0
+    for s, n in enumerate(counts):
+        ids[s, :n] = perm[at:at + n]
+        at += n
+        masks[s, :n] = rng.integers(0, 1 << 16, size=n, dtype=np.uint32)
+        if n > 2:
+            masks[s, 1] = 0                                          # a listed page with no token attended
+            masks[s, 0] = 0xFFFF
+    scale = sm_scale if sm_scale else 1.0 / np.sqrt(d)
+    ref = np.zeros((n_sets, group, d))
+    pool_bits = W.to_bits(pool)
+    for s, n in enumerate(counts):
+        rows_k, rows_v = [], []
+        for i in range(n):
+            keep = [r for r in range(T) if (int(masks[s, i]) >> r) & 1]
+            rows_k.append(pool_bits[ids[s, i], 0, keep])
+            rows_v.append(pool_bits[ids[s, i], 1, keep])
+        K = O.bf16_to_f32(np.concatenate(rows_k)) if rows_k else np.zeros((0, d), np.float32)
+        V = O.bf16_to_f32(np.concatenate(rows_v)) if rows_v else np.zeros((0, d), np.float32)
+        ref[s] = O.attention_fp64(O.bf16_to_f32(W.to_bits(q[s])), K, V, scale)
+    args = [x.to(dev) for x in (q, pool, torch.from_numpy(ids), torch.from_numpy(masks),
+                                torch.from_numpy(np.asarray(counts, dtype=np.int32)))]
+    outs = []
+    for call in range(2):
+        got = torch.full((n_sets, group, d), float("nan"), dtype=torch.bfloat16, device=dev)
+        rc = P.spin_paged_attention_static(args[0], args[1], args[2], args[3], args[4], n_sets, stride, group,
+                                           sm_scale, got, torch.cuda.current_stream())
+        assert rc == 0
+        torch.cuda.synchronize()
+        outs.append(got.float().cpu().numpy().astype(np.float64))
+    return outs, ref
+
+
+@pytest.mark.parametrize("group", [1, 8])
+def test_static_attention_boundary_lists_against_the_fp64_reference(group):
+    # a full list (n_pages == list_stride, three chunks of 8, 8 and 3 pages), an empty set, one
+    # page, exactly one chunk, one page more than a chunk; query groups of 1 and of 8
+    outs, ref = _static_case(group, [19, 0, 1, 8, 9], 19, seed=40 + group, sm_scale=1.0)
+    for call, got in enumerate(outs):
+        assert np.isfinite(got).all(), call
+        err = np.abs(got - ref)
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (call, err.max(), err.mean())
+        assert np.array_equal(got[1], np.zeros_like(got[1]))         # the empty set: zero output
+        rel = np.sqrt((err ** 2).sum() / (ref ** 2).sum())
+        assert rel < 2e-2, rel
+
+
+def test_static_attention_many_chunks_merge_in_tiles():
+    # 4800 pages in one set (600 chunks: the merge works through them in tiles), query group 8
+    outs, ref = _static_case(8, [4800], 4800, seed=7)
+    for got in outs:
+        err = np.abs(got - ref)
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (err.max(), err.mean())
+        assert np.sqrt((err ** 2).sum() / (ref ** 2).sum()) < 2e-2
