@@ -116,7 +116,9 @@ typedef struct spin_config {
                                    resident all at once and draws items from a queue when a step
                                    has more than 12 items per SM, so that attention can start
                                    fetching from the first sets), 1 = always the resident
-                                   form, -1 = never */
+                                   form, -1 = never, 2 = the streaming form: one scoring CTA per
+                                   SM fed by a ring of TMA stages, sets scored in order, one
+                                   selection CTA per set behind it (query groups of up to 4) */
   int32_t reserved0;
   int64_t offload_stage_bytes;  /* 0: appended pages are written through to pinned host memory on
                                    the caller's stream (Offload, Section 4.1).  > 0: asynchronous

@@ -229,6 +229,7 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
   d.evict_trace = cfg.trace ? a.take<int32_t>((size_t)g.n_sets * g.max_slots * 2) : nullptr;
   const size_t B = (size_t)g.max_batch_sets, PL = (size_t)(g.max_pages + g.tail_cap);
   d.scores = a.take<float>(B * g.max_cand);
+  d.score_xfer = a.take<float>(B * g.max_cand);
   d.sel_ids = a.take<int32_t>(B * g.max_sel);
   d.n_sel = a.take<int32_t>(B);
   d.parts = a.take<int32_t>(B * g.max_parts);
@@ -776,7 +777,7 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   d.n_host_pages = (int32_t)cfg->host_pages;
   d.fetch_mode = cfg->fetch_mode ? 1 : 0;
   d.evict_exact = cfg->evict_exact ? 1 : 0;
-  d.resident_scoring = cfg->resident_scoring > 0 ? 1 : cfg->resident_scoring < 0 ? -1 : 0;
+  d.resident_scoring = cfg->resident_scoring == 2 ? 2 : cfg->resident_scoring > 0 ? 1 : cfg->resident_scoring < 0 ? -1 : 0;
   d.sm_scale = cfg->sm_scale != 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)kHeadDim);
 
   // directories start unmapped (-1); states, counters and the miss queue start at zero
@@ -790,6 +791,7 @@ int spin_create(const spin_config *cfg, spin_ctx **out) {
   // tokens are masked out of the softmax but still enter the P*V tiles with weight 0)
   fill(d.gpu_pages, 0, (size_t)g.n_gpu_pages_total * kPageBytes);
   memset(ctx->host_base, 0, ctx->host_bytes);
+  fill(d.score_xfer, 0xff, (size_t)g.max_batch_sets * g.max_cand * 4);       // every word "not written"
   fill(d.att_count, 0, (size_t)g.max_batch_sets * 4);
   fill(d.sel_count, 0, (size_t)g.max_batch_sets * 4);
   fill(d.score_queue, 0, 4);

@@ -5,6 +5,10 @@
 
 namespace spin {
 
+// The append body is run by 256 threads that may be part of a larger CTA (the streaming scoring
+// kernel has a producer warp besides them): they meet at a named barrier of their own.
+__device__ __forceinline__ void sync_256() { asm volatile("bar.sync 1, 256;\n" ::: "memory"); }
+
 // 256 threads; thread t moves the 16-byte piece (t & 15) of row (t >> 4).
 __device__ __forceinline__ uint4 ld16(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
 __device__ __forceinline__ void st16(void *p, uint4 v) { *reinterpret_cast<uint4 *>(p) = v; }
@@ -76,7 +80,7 @@ __device__ __forceinline__ void append_edge_body(const DevCtx &c, int set, int i
   const int tid = threadIdx.x;
   const int r = tid >> 4, piece = tid & 15;
   SetState st = c.state[set];
-  __syncthreads();       // every thread has read the state before thread 0 rewrites it at the end
+  sync_256();            // every thread has read the state before thread 0 rewrites it at the end
   // the host has counted every append; its count is the one used, and a device word that
   // disagrees is reported (it is rewritten below)
   if (threadIdx.x == 0 && st.n_tokens != n0_host) {
@@ -142,9 +146,9 @@ __device__ __forceinline__ void append_edge_body(const DevCtx &c, int set, int i
       } else if (piece == 0) dev_error(c, 1u);
     }
     st16(reinterpret_cast<uint8_t *>(krows[r]) + piece * 16, kk);
-    __syncthreads();
+    sync_256();
     index_page(c, set, j0, krows, tid);
-    __syncthreads();                                        // tail rows are read before rewritten
+    sync_256();                                             // tail rows are read before rewritten
   }
   {
     const int lo = max(n0, j_end * kPageTokens) - j_end * kPageTokens;   // first new row

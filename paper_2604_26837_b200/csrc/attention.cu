@@ -442,6 +442,7 @@ void launch_attn_g(const DevCtx &c, const Batch &b, const __nv_bfloat16 *q, __nv
   constexpr int smem = kChunkPages * kPageBytes;
   if (!configured) {
     cudaFuncSetAttribute(k_attn<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(k_attn<G>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     configured = true;
   }
   launch_pdl(k_attn<G>, grid, dim3(kAttnWarps * 32), (size_t)smem, st, 1, c, b, q, out);

@@ -82,6 +82,9 @@ struct DevCtx {
   int32_t max_slots;
   // per-step scratch, indexed by batch set b = i_req * Hkv + head
   float *scores;                // [b][max_cand]
+  float *score_xfer;            // [b][max_cand] hand-over buffer of the streaming scoring kernel: all words hold the
+                                //   "not written" pattern between steps; the set's selection takes a score out
+                                //   (into `scores`) and puts the pattern back
   int32_t *sel_ids;             // [b][max_sel]   chosen candidates, ascending
   int32_t *n_sel;               // [b]
   int32_t *parts;               // [b][max_parts] partitions for the cache manager
@@ -234,6 +237,23 @@ __device__ __forceinline__ bool flag_wait(const DevCtx &c, const int32_t *flag, 
   }
   dev_error(c, kErrTimeout);
   return false;
+}
+
+// Scores handed from the streaming scoring kernel to a set's selection without a fence: a score
+// is one naturally aligned 4-byte store, so the word itself says whether it has arrived.  The
+// buffer holds kScoreUnset (a NaN pattern no finite computation produces) in every word between
+// steps; the reader polls a word until it differs (bounded), copies it and restores the pattern.
+constexpr uint32_t kScoreUnset = 0xffffffffu;
+__device__ __forceinline__ float take_score(const DevCtx &c, float *xfer) {
+  uint32_t v = kScoreUnset;
+  for (int spin = 0; spin < (1 << 20); ++spin) {
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(xfer) : "memory");
+    if (v != kScoreUnset) break;
+    __nanosleep(64);
+  }
+  if (v == kScoreUnset) { dev_error(c, kErrTimeout); v = 0u; }
+  *reinterpret_cast<uint32_t *>(xfer) = kScoreUnset;
+  return __uint_as_float(v);
 }
 
 __device__ __forceinline__ const uint8_t *page_ptr(const DevCtx &c, int src) {

@@ -105,8 +105,10 @@ __device__ __forceinline__ bool resolve_in_manager(const DevCtx &c) { return c.f
 #ifdef SPIN_TIMING
 __device__ unsigned long long g_dbg_ts[256][32];
 __device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; } }
+__device__ __forceinline__ void dbg_ts_any(int b, int slot) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; }
 #else
 __device__ __forceinline__ void dbg_ts(int, int) {}
+__device__ __forceinline__ void dbg_ts_any(int, int) {}
 #endif
 
 struct TopkShared {
@@ -129,9 +131,10 @@ template <bool CLUSTER> __device__ __forceinline__ void stage_sync() {
 // flag) and every CTA of a cluster executes the same number of them.  Without CLUSTER the
 // calling CTA owns the whole set.  On return (all threads of rank 0) the partitions handed to
 // the cache manager are in c.parts / c.n_parts; other ranks return false and must exit.
+// xfer: the scores come from the streaming kernel's hand-over buffer (taken out into c.scores on the way)
 template <int T, bool CLUSTER>
 __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partitions, uint32_t *s_keys,
-                                           int keys_cap, TopkShared &sh) {
+                                           int keys_cap, TopkShared &sh, bool xfer = false) {
   int C = 1, rank = 0;
   if constexpr (CLUSTER) {
     cg::cluster_group cluster = cg::this_cluster();
@@ -141,7 +144,8 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
   const int tid = threadIdx.x;
   const int n = c.kind == kKindToken ? n_partitions * kPageTokens : n_partitions;
   const int k = min(c.topk, n);
-  const float *scores = c.scores + (size_t)b * c.max_cand;
+  float *scores = c.scores + (size_t)b * c.max_cand;
+  float *xfer_in = c.score_xfer + (size_t)b * c.max_cand;
   int32_t *sel = c.sel_ids + (size_t)b * c.max_sel;
   const int per = (n + C - 1) / C;
   const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
@@ -157,7 +161,10 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
   {
     uint32_t k_or = 0, k_and = 0xffffffffu;
     for (int i = tid; i < m; i += T) {
-      const uint32_t key = order_key(__ldcg(scores + lo + i));
+      float sc;
+      if (xfer) { sc = take_score(c, xfer_in + lo + i); scores[lo + i] = sc; }
+      else sc = __ldcg(scores + lo + i);
+      const uint32_t key = order_key(sc);
       if (cached) s_keys[i] = key;
       k_or |= key; k_and &= key;
     }
@@ -839,9 +846,13 @@ template <int T>
 __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
                                            const FastLayout &L, int np_sel, FastShared &sh);
 
+// prefetched: the caller has already issued fast_prefetch_dirs, waited for it behind a barrier,
+// and issued fast_prefetch_gpt / fast_prefetch_tables (a CTA that waits for its set to be
+// scored brings the tables in while it waits)
 template <int T>
 __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, int b, int i_req, int set,
-                                            uint8_t *dyn, int keys_cap, int tbl_cap, FastShared &sh) {
+                                            uint8_t *dyn, int keys_cap, int tbl_cap, FastShared &sh,
+                                            bool prefetched = false, bool xfer = false) {
   const int tid = threadIdx.x;
   const bool token = c.kind == kKindToken;
   const int n = token ? bt.n_partitions[i_req] * kPageTokens : bt.n_partitions[i_req];
@@ -858,17 +869,31 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
 
   dbg_ts(b, 1);
   // ---- directories on their way (consumed after the keys are loaded) ------------------------
-  fast_prefetch_dirs<T>(c, L, set, S);
+  if (!prefetched) fast_prefetch_dirs<T>(c, L, set, S);
 
-  const float *scores = c.scores + (size_t)b * c.max_cand;
+  float *scores = c.scores + (size_t)b * c.max_cand;
+  float *xfer_in = c.score_xfer + (size_t)b * c.max_cand;
   auto key_at = [&](int i) { return cached ? s_keys[i] : order_key(__ldcg(scores + i)); };
   // keys -> shared memory, with the OR and AND of all keys taken on the way (see the select)
   uint32_t k_or = 0, k_and = 0xffffffffu;
+  if (xfer) {
+    // scores come through the hand-over buffer: taken out (pattern restored) and kept in c.scores
+#pragma unroll 4
+    for (int i = tid; i < n; i += T) {
+      const float sc = take_score(c, xfer_in + i);
+      scores[i] = sc;
+      const uint32_t key = order_key(sc);
+      if (cached) s_keys[i] = key;
+      k_or |= key; k_and &= key;
+    }
+    if (!cached) { __threadfence_block(); __syncthreads(); }       // key_at re-reads c.scores written by other threads
+  } else {
 #pragma unroll 8
-  for (int i = tid; i < n; i += T) {
-    const uint32_t key = order_key(__ldcg(scores + i));
-    if (cached) s_keys[i] = key;
-    k_or |= key; k_and &= key;
+    for (int i = tid; i < n; i += T) {
+      const uint32_t key = order_key(__ldcg(scores + i));
+      if (cached) s_keys[i] = key;
+      k_or |= key; k_and &= key;
+    }
   }
   k_or = __reduce_or_sync(0xffffffffu, k_or);
   k_and = __reduce_and_sync(0xffffffffu, k_and);
@@ -885,8 +910,10 @@ __device__ __forceinline__ void select_fast(const DevCtx &c, const Batch &bt, in
 
   dbg_ts(b, 2);
   // ---- the GPU page table on its way (consumed after top-k) ---------------------------------
-  fast_prefetch_gpt<T>(c, L, S);
-  fast_prefetch_tables<T>(c, L, bt.n_partitions[i_req]);
+  if (!prefetched) {
+    fast_prefetch_gpt<T>(c, L, S);
+    fast_prefetch_tables<T>(c, L, bt.n_partitions[i_req]);
+  }
 
   // ---- top-k: wide-digit radix select, one-scan ordered compaction ---------------------------
   int32_t *g_sel = c.sel_ids + (size_t)b * c.max_sel;

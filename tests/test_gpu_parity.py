@@ -358,6 +358,33 @@ def test_resident_scoring_grid(kind):
     assert r["stats"]["miss_pages"] > 0
 
 
+@pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_CLUSTER_CENTROID, W.PART_TOKEN_DOT, W.PART_PAGE_MEAN])
+def test_streaming_scoring_kernel(kind):
+    # the streaming form of scoring (ring of TMA stages, a selection CTA per set, scores handed
+    # over word by word): mixed lengths with an empty request, ragged last stages, steps that
+    # complete a page, query groups of 4, 2 and 1; scores must stay bit-exact
+    if kind == W.PART_CLUSTER_CENTROID:
+        w = _wl(kind, kv_recipe="mixture", num_clusters=37, topk=5, slots_per_set=30,
+                context=16 * 50 + 3, steps=24, max_partition_pages=8, lru_buckets=8)
+    else:
+        w = _wl(kind, batch=5, num_layers=1, context=16 * 300, ctx_range=(0, 16 * 300),
+                drift_choices=(0.01, 0.1, 0.5), topk=10 if kind != W.PART_TOKEN_DOT else 100, steps=36, lru_buckets=8)
+    r = run_parity(w, one_call=True, resident_scoring=2, check_bytes=kind == W.PART_PAGE_MINMAX)
+    assert r["stats"]["miss_pages"] > 0
+    for hq in (4, 2):
+        run_parity(_wl(kind if kind != W.PART_CLUSTER_CENTROID else W.PART_PAGE_MINMAX, num_q_heads=hq, num_kv_heads=2,
+                       steps=12, context=16 * 70 + 9), one_call=True, resident_scoring=2, check_bytes=False)
+
+
+def test_streaming_scoring_kernel_with_the_cluster_top_k_and_ties():
+    # > 16384 candidate keys per set: streaming scoring, then the thread-block cluster per set that
+    # takes the scores out of the hand-over buffer; tied scores across the slices
+    w = _wl(W.PART_TOKEN_DOT, context=16 * 1300 + 5, topk=300, slots_per_set=120, steps=10, batch=2,
+            num_layers=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8, drift=0.3, kv_recipe="tied", tie_period=1000)
+    r = run_parity(w, check_bytes=False, one_call=True, resident_scoring=2)
+    assert r["tied_at_k"] == 2 * 2 * 10
+
+
 def test_cluster_tail_is_folded_into_the_clusters_during_decode():
     # Index during decode: every 20 steps the full tail pages join the clusters of their best
     # centroids (new cluster pages, stale residency dropped, layout rewritten, tail rotated);
