@@ -120,7 +120,7 @@ def measure_pcie_gbs(torch, device, stream) -> float:
     return best
 
 
-def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests: int = 1):
+def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests: int = 1, first_request: int = 0):
     """Time the CPU oracle, as it stands, on `sample_requests` requests of the workload."""
     import numpy as np
     import workloads as W
@@ -133,7 +133,8 @@ def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests:
     orc = O.SpinOracle(O.OracleConfig(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                       w.page_tokens, w.partition_kind, w.topk, w.lru_buckets))
     reqs = []
-    for r in range(sample_requests):
+    ids = list(range(first_request, first_request + sample_requests))       # requests of the workload that are run
+    for r in ids:
         req = orc.request_open(w.slots_per_set if w.slots_per_set else min(w.topk * 2, 512))
         reqs.append(req)
         for l in range(w.num_layers):
@@ -144,20 +145,20 @@ def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests:
                               W.to_bits(W.centroids(w, r, l)))
             else:
                 orc.append_kv(req, l, W.to_bits(k), W.to_bits(v))
-    qs = {(r, l): W.QueryStream(w, r, l) for r in range(sample_requests) for l in range(w.num_layers)}
+    qs = {(r, l): W.QueryStream(w, r, l) for r in ids for l in range(w.num_layers)}
     times = []
     step = 0
     t_start = time.perf_counter()
     while True:
         ins = []
         for l in range(w.num_layers):
-            kv = [W.kv_tokens(w, r, l, w.request_context(r) + step, 1) for r in range(sample_requests)]
-            q = np.stack([W.to_bits(qs[(r, l)].next()) for r in range(sample_requests)])
+            kv = [W.kv_tokens(w, r, l, w.request_context(r) + step, 1) for r in ids]
+            q = np.stack([W.to_bits(qs[(r, l)].next()) for r in ids])
             ins.append((l, [(W.to_bits(k), W.to_bits(v)) for k, v in kv], q))
         t0 = time.perf_counter()
         for l, kv, q in ins:
-            for r, (kb, vb) in enumerate(kv):
-                orc.append_kv(reqs[r], l, kb, vb)
+            for i_, (kb, vb) in enumerate(kv):
+                orc.append_kv(reqs[i_], l, kb, vb)
             orc.decode_step(l, reqs, q)
         dt = time.perf_counter() - t0
         if step >= warmup:
@@ -196,6 +197,255 @@ def aggregate_value(units_per_rank: int, world: int, max_elapsed_ms: float) -> f
     return units_per_rank * world / (max_elapsed_ms * 1e-3)
 
 
+def workload_bytes(w, d):
+    """Algorithmic bytes of the counted set-steps `d` (differences of spin_stats): HBM = summaries
+    scanned + selected KV read once + the tail pages + missed pages written into their slots;
+    host link = missed pages.  Token-granular selection reads the selected token ROWS (512 B of
+    K and V each) of the selected pages, not whole pages."""
+    summ = d["candidates_scored"] * (512 if w.partition_kind == 0 else 256)
+    admit = (d["miss_pages"] - d["bypass_pages"]) * PAGE_BYTES
+    if w.partition_kind == 1:
+        cand_per_set = (w.context // w.page_tokens) * w.page_tokens
+        kv = d["set_steps"] * min(w.topk, cand_per_set) * 512 + d["tail_pages"] * PAGE_BYTES
+    else:
+        kv = (d["selected_pages"] + d["tail_pages"]) * PAGE_BYTES
+    return dict(hbm=summ + kv + admit, pcie=d["miss_pages"] * PAGE_BYTES, summaries=summ, kv=kv, admit=admit)
+
+
+def measure(base, args, K, Wm, rank, world, device, do_e2e, pcie_gbs, peaks, cache_pages_per_layer):
+    """Prefill, prime the cache to its steady state, warm up, time K steps of one workload.
+    Returns the record of this rank (times in ms; stats differences over the timed window)."""
+    import torch
+    import workloads as W
+    from paper_2604_26837_b200.driver import SpinRun
+    prime_cap = args.prime_cap
+    prof_steps = min(K, 32)
+    e2e_steps = K if do_e2e else 0
+    total_steps = prime_cap + Wm + K + K + prof_steps + (Wm + e2e_steps)
+    w = rank_workload(base, rank, total_steps)
+    run = SpinRun(w, device, fetch_mode=args.fetch_mode, cache_pages_per_layer=cache_pages_per_layer,
+                  resident_scoring=args.resident_scoring)
+    stream = torch.cuda.Stream(device)
+    B, L = w.batch, w.num_layers
+    t_setup = time.perf_counter()
+    with torch.cuda.stream(stream):
+        for r in range(B):
+            for l in range(L):
+                k, v, tp, cen = run.gen_prefill(r, l)
+                run.prefill(r, l, k, v, tp, cen, stream)
+                del k, v
+        qstreams = {(r, l): W.QueryStream(w, r, l, device) for r in range(B) for l in range(L)}
+        out = torch.zeros(B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=device)
+        flush = torch.empty(64 << 20, dtype=torch.int32, device=device)        # 256 MiB
+    torch.cuda.synchronize(device)
+    cur = [0]
+
+    def gen_inputs(n):
+        """Inputs of the next n decode steps, resident in HBM before any timed region."""
+        q_ = torch.empty(n, L, B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=device)
+        k_ = torch.empty(n, L, B, w.num_kv_heads, w.head_dim, dtype=torch.bfloat16, device=device)
+        v_ = torch.empty_like(k_)
+        with torch.cuda.stream(stream):
+            for i in range(n):
+                for l in range(L):
+                    k_[i, l], v_[i, l] = run.gen_step_tokens(l, cur[0] + i)
+                    for r in range(B):
+                        q_[i, l, r] = qstreams[(r, l)].next()
+        torch.cuda.synchronize(device)
+        return q_, k_, v_
+
+    def flush_l2_fn():
+        # write 256 MiB (> 126 MB L2), then read it back so that the L2 is left full of CLEAN
+        # lines, as it is after the weights of a model's other layers have streamed through;
+        # a write-only flush would leave dirty lines whose write-back taxes the timed kernels
+        flush.zero_()
+        flush.max()
+
+    def timed_steps(n, flush_l2=True):
+        q_, k_, v_ = gen_inputs(n)
+        evs = []
+        with torch.cuda.stream(stream):
+            for i in range(n):
+                if flush_l2:
+                    flush_l2_fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for l in range(L):
+                    run.step(l, k_[i, l], v_[i, l], q_[i, l], out, stream)
+                e1.record(stream)
+                evs.append((e0, e1))
+        torch.cuda.synchronize(device)
+        cur[0] += n
+        return [a.elapsed_time(b) for a, b in evs]
+
+    # cold start, then priming until the cache is in its steady state: the slots are full and
+    # every step evicts (Section 5.3 step 3 has work to do), or the cap is reached
+    cold_steps = timed_steps(8)
+    primed, evicting_chunks = 8, 0
+    while primed < prime_cap and evicting_chunks < 2:
+        s0 = run.spin.stats()
+        timed_steps(8, flush_l2=False)
+        s1 = run.spin.stats()
+        primed += 8
+        evicting_chunks = evicting_chunks + 1 if s1["evicted_pages"] > s0["evicted_pages"] else 0
+    timed_steps(Wm)
+    st0 = run.spin.stats()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.synchronize(device)
+        dist.barrier()
+    t_begin = datetime.datetime.now()
+    per_step = timed_steps(K)
+    if world > 1:
+        torch.cuda.synchronize(device)
+        dist.barrier()
+    t_end = datetime.datetime.now()
+    st1 = run.spin.stats()
+    # back-to-back variant without the L2 flush (one pair of events around all K steps)
+    q_, k_, v_ = gen_inputs(K)
+    with torch.cuda.stream(stream):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(K):
+            for l in range(L):
+                run.step(l, k_[i, l], v_[i, l], q_[i, l], out, stream)
+        e1.record(stream)
+    torch.cuda.synchronize(device)
+    cur[0] += K
+    noflush_ms = e0.elapsed_time(e1) / K
+    # per-kernel durations, measured live with CUDA events recorded between the launches
+    stp0 = run.spin.stats()
+    run.spin.profile(True)
+    timed_steps(prof_steps)
+    prof = run.spin.profile_read()
+    run.spin.profile(False)
+    stp1 = run.spin.stats()
+    rec = dict(w=w, per_step=per_step, noflush_ms=noflush_ms, cold_steps=cold_steps, primed=primed,
+               t_begin=t_begin, t_end=t_end, prof=prof, B=B, L=L)
+    skip = ("error_bits", "debug_words", "status")
+    rec["d"] = {k: st1[k] - st0[k] for k in st0 if k not in skip}
+    rec["dp"] = {k: stp1[k] - stp0[k] for k in stp0 if k not in skip}
+    # end to end: host buffers in, host buffer out, every step
+    if e2e_steps:
+        q_, k_, v_ = gen_inputs(Wm + e2e_steps)
+        qh, kh, vh = q_.cpu().pin_memory(), k_.cpu().pin_memory(), v_.cpu().pin_memory()
+        oh = torch.zeros(B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16).pin_memory()
+        e2e_times = []
+        oh_bits = oh.view(torch.int16).numpy()           # the pinned output buffer as the host reads it
+        checksum = 0
+        # the step's host buffers as the caller would hold them (views made outside the timed region)
+        host_in = [[(kh[i, l], vh[i, l], qh[i, l]) for l in range(L)] for i in range(Wm + e2e_steps)]
+        with torch.cuda.stream(stream):
+            for i in range(Wm + e2e_steps):
+                flush_l2_fn()
+                stream.synchronize()
+                t0 = time.perf_counter()
+                for l in range(L):
+                    kk, vv, qq = host_in[i][l]
+                    run.step(l, kk, vv, qq, oh, stream)
+                stream.synchronize()                       # the result is read on the host
+                checksum += int(oh_bits[0, 0, 0]) + int(oh_bits[-1, -1, -1])
+                if i >= Wm:
+                    e2e_times.append(time.perf_counter() - t0)
+        rec["e2e_ms"] = 1e3 * sum(e2e_times)
+        rec["h2d"] = L * (qh[0, 0].numel() + kh[0, 0].numel() + vh[0, 0].numel()) * 2
+        rec["d2h"] = L * oh.numel() * 2
+    rec["final"] = run.spin.stats()
+    rec["setup_s"] = time.perf_counter() - t_setup
+    run.close()
+    del run
+    torch.cuda.empty_cache()
+    return rec
+
+
+def summarise(rec, args, K, world, elapsed_ms, pcie_gbs, peaks, fused, full_size):
+    """The figures of one workload: throughput, step roofline, per-kernel table, dominant kernel."""
+    w, d, dp, prof, B = rec["w"], rec["d"], rec["dp"], rec["prof"], rec["B"]
+    per_step = rec["per_step"]
+    by = workload_bytes(w, d)
+    hbm_step, pcie_step = by["hbm"] / K, by["pcie"] / K
+    t_hbm = hbm_step / (peaks["hbm_gbs"] * 1e9)
+    t_pcie = pcie_step / (pcie_gbs * 1e9)
+    t_step = elapsed_ms * 1e-3 / K
+    byp = workload_bytes(w, dp)
+    miss_b, admit_b = byp["pcie"], byp["admit"]
+    # algorithmic bytes per kernel over the profiled steps: (HBM bytes, host-link bytes)
+    bytes_of = dict(score=(byp["summaries"], 0), fetch=(admit_b, admit_b),
+                    attn_split=((byp["kv"] - miss_b + admit_b, miss_b) if fused else (byp["kv"] - (miss_b - admit_b), miss_b - admit_b)))
+    kern = {}
+    tot_ms = sum(ms for _, ms in prof.values()) or 1.0
+    for name, (n, ms) in prof.items():
+        if not n:
+            continue
+        kern[name] = dict(launches=n, avg_us=1e3 * ms / n, share=ms / tot_ms)
+        if name in bytes_of:
+            hb, pb = bytes_of[name]
+            t_h, t_p = hb / (peaks["hbm_gbs"] * 1e9), pb / (pcie_gbs * 1e9)
+            kern[name].update(hbm_gbs=hb / (ms * 1e-3) / 1e9, pcie_gbs=pb / (ms * 1e-3) / 1e9,
+                              bound="pcie" if t_p > t_h else "hbm", roof_frac=max(t_h, t_p) / (ms * 1e-3))
+    top = max((k_ for k_ in ("fetch", "score", "attn_split") if k_ in kern), key=lambda k_: kern[k_]["share"])
+    bound = kern[top]["bound"]
+    peak = pcie_gbs if bound == "pcie" else peaks["hbm_gbs"]
+    achieved = kern[top]["pcie_gbs"] if bound == "pcie" else kern[top]["hbm_gbs"]
+    traffic = (NCU_TRAFFIC.get(w.name) or {}).get(top) if full_size else None
+    names = dict(fetch="k_fetch", score="k_score", attn_split="k_attn (attention + page fetch)" if fused else "k_attn")
+    roofline = dict(kernel=names[top], bound=bound, achieved=achieved, peak=peak, unit="GB/s",
+                    frac=kern[top]["roof_frac"], traffic=traffic,
+                    peak_source=("pinned H2D copy measured in this run" if bound == "pcie" else peaks["source"]),
+                    avg_launch_us=kern[top]["avg_us"],
+                    hbm_bytes_per_launch=bytes_of[top][0] / kern[top]["launches"],
+                    pcie_bytes_per_launch=bytes_of[top][1] / kern[top]["launches"])
+    step_roofline = dict(hbm_bytes_per_step=hbm_step, pcie_bytes_per_step=pcie_step,
+                         hbm_gbs_peak=peaks["hbm_gbs"], hbm_peak_source=peaks["source"], pcie_gbs_peak=pcie_gbs,
+                         t_hbm_us=1e6 * t_hbm, t_pcie_us=1e6 * t_pcie, t_step_us=1e6 * t_step,
+                         bound="pcie" if t_pcie > t_hbm else "hbm", frac=max(t_hbm, t_pcie) / t_step,
+                         frac_vs_nominal_8tbs=max(hbm_step / 8e12, t_pcie) / t_step,
+                         miss_ratio=d["miss_pages"] / max(d["selected_pages"], 1))
+    sets = d["set_steps"] / K
+    return dict(value=aggregate_value(B * K, world, elapsed_ms), ms_per_step=elapsed_ms / K,
+                p50_tpot_ms=statistics.median(per_step), ms_per_step_noflush=rec["noflush_ms"],
+                step_roofline=step_roofline, roofline=roofline, kernels=kern,
+                miss_ratio=step_roofline["miss_ratio"], evicted_pages_per_step=d["evicted_pages"] / K,
+                missed_pages_per_step=d["miss_pages"] / K, sets_per_step=sets, primed_steps=rec["primed"],
+                gpu_launches=int(d["kernel_launches"]), error_bits=rec["final"]["error_bits"],
+                setup_s=round(rec["setup_s"], 1))
+
+
+def workload_desc(base, world):
+    return dict(workload=f"{base.name}: batch {base.batch} x {base.num_layers} layer(s), "
+                         f"{base.num_q_heads}q/{base.num_kv_heads}kv heads, context {base.context}, "
+                         f"kind {base.partition_kind}, top-k {base.topk}, "
+                         f"{base.slots_per_set if base.slots_per_set else 'dynamic'} slots/set, "
+                         f"{base.lru_buckets} buckets, drift {base.drift}",
+                global_batch=base.batch * world, context=base.context, parallelism=f"replicas x{world}")
+
+
+def _oracle_worker(args):
+    name, kw, budget_s, steps_cap, r = args
+    import workloads as W
+    base = W.scaled(W.CONFIGS[name], **kw)
+    return oracle_run(base, budget_s, steps_cap, 1, sample_requests=1, first_request=r)
+
+
+def oracle_all_cores(base_name, kw, budget_s, steps_cap):
+    """The oracle on every host core at once: one process per request (requests are independent),
+    each a single numpy thread; throughput = requests x steps over the slowest process's time."""
+    import multiprocessing as mp
+    import workloads as W
+    base = W.scaled(W.CONFIGS[base_name], **kw)
+    n = min(os.cpu_count() or 1, base.batch)
+    ctx = mp.get_context("spawn")
+    t0 = time.perf_counter()
+    with ctx.Pool(n) as pool:
+        res = pool.map(_oracle_worker, [(base_name, kw, budget_s, steps_cap, r) for r in range(n)])
+    wall = time.perf_counter() - t0
+    steps = min(r["steps"] for r in res)
+    slowest = max(r["ms_per_step"] for r in res)
+    return dict(value=n / (slowest * 1e-3), unit="tokens/s", cores=n, nproc=os.cpu_count(), kind="oracle",
+                sample=f"{n} of {base.batch} requests in {n} processes (one numpy thread each) x {steps} decode steps; "
+                       f"rate = requests over the slowest process's mean step time", wall_s=round(wall, 1))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -203,10 +453,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--impl", default="spin", choices=["spin", "reference"])
-    ap.add_argument("--prime", type=int, default=24, help="untimed decode steps that warm the KV cache (setup)")
+    ap.add_argument("--prime-cap", type=int, default=160,
+                    help="at most this many untimed decode steps to bring the KV cache to its steady state (setup)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--resident-scoring", type=int, default=0, help="spin_config.resident_scoring: 0 automatic, 1 always, -1 never")
+    ap.add_argument("--no-per-config", action="store_true", help="only the headline workload, not the other configurations")
+    ap.add_argument("--per-config-steps", type=int, default=32)
+    ap.add_argument("--resident-scoring", type=int, default=0,
+                    help="spin_config.resident_scoring: 0 automatic, 1 queue-fed resident grid, -1 one CTA per item, 2 streaming")
     ap.add_argument("--context", type=int, default=0, help="override the context length (smaller captures)")
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (scaled runs of the 32-layer config)")
@@ -219,25 +473,21 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    base = W.CONFIGS[args.workload]
+    overrides = {}
     if args.context:
-        base = W.scaled(base, context=args.context)
+        overrides["context"] = args.context
     if args.batch:
-        base = W.scaled(base, batch=args.batch)
+        overrides["batch"] = args.batch
     if args.layers:
-        base = W.scaled(base, num_layers=args.layers)
-    # a workload without a fixed budget states a total: 60 GB of KV over its 32 layers and 64
-    # requests; a scaled run keeps the per-layer, per-request share
-    cache_pages_per_layer = None
-    if base.slots_per_set == 0:
-        cache_pages_per_layer = int(60e9 / 32 / PAGE_BYTES * base.batch / 64)
+        overrides["num_layers"] = args.layers
+    base = W.scaled(W.CONFIGS[args.workload], **overrides)
+
+    def cache_budget(b):
+        # a workload without a fixed budget states a total: 60 GB of KV over its 32 layers and 64
+        # requests; a scaled run keeps the per-layer, per-request share
+        return int(60e9 / 32 / PAGE_BYTES * b.batch / 64) if b.slots_per_set == 0 else None
     metric, unit = "decode_tokens_per_s", "tokens/s"
-    cfg_desc = dict(workload=f"{base.name}: batch {base.batch} x {base.num_layers} layer(s), "
-                             f"{base.num_q_heads}q/{base.num_kv_heads}kv heads, context {base.context}, "
-                             f"kind {base.partition_kind}, top-k {base.topk}, "
-                             f"{base.slots_per_set if base.slots_per_set else 'dynamic'} slots/set, "
-                             f"{base.lru_buckets} buckets, drift {base.drift}",
-                    global_batch=base.batch * world, context=base.context, parallelism=f"replicas x{world}")
+    cfg_desc = workload_desc(base, world)
 
     if args.impl == "reference":
         if rank != 0:
@@ -259,212 +509,84 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist.barrier()
-    from paper_2604_26837_b200.driver import SpinRun
 
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
-    K, Wm, P = args.steps, args.warmup, args.prime
-    prof_steps = min(K, 64)
-    e2e_steps = 0 if args.no_e2e else K
-    total_steps = P + Wm + K + K + prof_steps + (Wm + e2e_steps)
-    w = rank_workload(base, rank, total_steps)
-    run = SpinRun(w, device, fetch_mode=args.fetch_mode, cache_pages_per_layer=cache_pages_per_layer,
-                  resident_scoring=args.resident_scoring)
-    stream = torch.cuda.Stream(device)
-    B, L = w.batch, w.num_layers
-
-    def barrier():
-        torch.cuda.synchronize(device)
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize(device)
-
-    with torch.cuda.stream(stream):
-        for r in range(B):
-            for l in range(L):
-                k, v, tp, cen = run.gen_prefill(r, l)
-                run.prefill(r, l, k, v, tp, cen, stream)
-                del k, v
-        # inputs of every decode step, resident in HBM before any timed region
-        qstreams = {(r, l): W.QueryStream(w, r, l, device) for r in range(B) for l in range(L)}
-        q_all = torch.empty(total_steps, L, B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=device)
-        k_all = torch.empty(total_steps, L, B, w.num_kv_heads, w.head_dim, dtype=torch.bfloat16, device=device)
-        v_all = torch.empty_like(k_all)
-        for s in range(total_steps):
-            for l in range(L):
-                k_all[s, l], v_all[s, l] = run.gen_step_tokens(l, s)
-                for r in range(B):
-                    q_all[s, l, r] = qstreams[(r, l)].next()
-        out = torch.zeros(B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=device)
-        flush = torch.empty(64 << 20, dtype=torch.int32, device=device)        # 256 MiB
-    torch.cuda.synchronize(device)
-    pcie_gbs = measure_pcie_gbs(torch, device, stream)
-    cur = [0]
-
-    def flush_l2_fn():
-        # write 256 MiB (> 126 MB L2), then read it back so that the L2 is left full of CLEAN
-        # lines, as it is after the weights of a model's other layers have streamed through;
-        # a write-only flush would leave dirty lines whose write-back taxes the timed kernels
-        flush.zero_()
-        flush.max()
-
-    def one_step(s):
-        for l in range(L):
-            run.step(l, k_all[s, l], v_all[s, l], q_all[s, l], out, stream)
-
-    def timed_steps(n, flush_l2=True):
-        evs = []
-        with torch.cuda.stream(stream):
-            for _ in range(n):
-                if flush_l2:
-                    flush_l2_fn()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
-                one_step(cur[0])
-                e1.record(stream)
-                cur[0] += 1
-                evs.append((e0, e1))
-        torch.cuda.synchronize(device)
-        return [a.elapsed_time(b) for a, b in evs]
-
+    K, Wm = args.steps, args.warmup
+    peaks = load_peaks()
+    pcie_gbs = measure_pcie_gbs(torch, device, torch.cuda.Stream(device))
     props = torch.cuda.get_device_properties(device)
-    sampler = ClockSampler(f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank))
-    cold_steps = timed_steps(P + Wm)                       # cache priming + warm-up: reported apart (cold start)
-    st0 = run.spin.stats()
-    barrier()
-    t_begin = datetime.datetime.now()
-    per_step = timed_steps(K)
-    barrier()
-    t_end = datetime.datetime.now()
-    st1 = run.spin.stats()
-    elapsed_ms = sum(per_step)
-    # back-to-back variant without the L2 flush (one pair of events around all K steps)
-    with torch.cuda.stream(stream):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(K):
-            one_step(cur[0])
-            cur[0] += 1
-        e1.record(stream)
-    torch.cuda.synchronize(device)
-    noflush_ms = e0.elapsed_time(e1) / K
-    clocks = sampler.stop(t_begin, t_end)
-    link = pcie_link(f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank))
+    gpu_id = f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank)
+    fused = args.fetch_mode == 0
+    full_size = not overrides
 
-    # per-kernel durations, measured live with CUDA events recorded between the launches
-    stp0 = run.spin.stats()
-    run.spin.profile(True)
-    timed_steps(prof_steps)
-    prof = run.spin.profile_read()
-    run.spin.profile(False)
-    stp1 = run.spin.stats()
-
-    # end to end: host buffers in, host buffer out, every step
-    e2e = None
-    if e2e_steps:
-        qh = q_all[cur[0]:cur[0] + Wm + e2e_steps].cpu().pin_memory()
-        kh = k_all[cur[0]:cur[0] + Wm + e2e_steps].cpu().pin_memory()
-        vh = v_all[cur[0]:cur[0] + Wm + e2e_steps].cpu().pin_memory()
-        oh = torch.zeros(B, w.num_q_heads, w.head_dim, dtype=torch.bfloat16).pin_memory()
-        e2e_times = []
-        oh_bits = oh.view(torch.int16).numpy()           # the pinned output buffer as the host reads it
-        checksum = 0
-        # the step's host buffers as the caller would hold them (views made outside the timed region)
-        host_in = [[(kh[i, l], vh[i, l], qh[i, l]) for l in range(L)] for i in range(Wm + e2e_steps)]
-        with torch.cuda.stream(stream):
-            for i in range(Wm + e2e_steps):
-                flush_l2_fn()
-                stream.synchronize()
-                t0 = time.perf_counter()
-                for l in range(L):
-                    kk, vv, qq = host_in[i][l]
-                    run.step(l, kk, vv, qq, oh, stream)
-                stream.synchronize()                       # the result is read on the host
-                checksum += int(oh_bits[0, 0, 0]) + int(oh_bits[-1, -1, -1])
-                if i >= Wm:
-                    e2e_times.append(time.perf_counter() - t0)
-        e2e_ms = 1e3 * sum(e2e_times)
-        h2d = L * (qh[0, 0].numel() + kh[0, 0].numel() + vh[0, 0].numel()) * 2
-        d2h = L * oh.numel() * 2
-    final = run.spin.stats()
-
+    sampler = ClockSampler(gpu_id)
+    rec = measure(base, args, K, Wm, rank, world, device, not args.no_e2e, pcie_gbs, peaks, cache_budget(base))
+    clocks = sampler.stop(rec["t_begin"], rec["t_end"])
+    link = pcie_link(gpu_id)
+    elapsed_ms = sum(rec["per_step"])
+    e2e_ms = rec.get("e2e_ms", 0.0)
+    noflush_ms = rec["noflush_ms"]
     if world > 1:
-        elapsed_ms, e2e_max, noflush_ms = allreduce_max([elapsed_ms, e2e_ms if e2e_steps else 0.0, noflush_ms], device)
-        if e2e_steps:
-            e2e_ms = e2e_max
+        elapsed_ms, e2e_ms, noflush_ms = allreduce_max([elapsed_ms, e2e_ms, noflush_ms], device)
+        rec["noflush_ms"] = noflush_ms
     if rank != 0:
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
         return
 
-    peaks = load_peaks()
-    value = aggregate_value(B * K, world, elapsed_ms)
-    d = {k: st1[k] - st0[k] for k in st0 if k not in ("error_bits", "debug_words")}
-    hbm_step = d["hbm_bytes"] / K
-    pcie_step = d["pcie_bytes"] / K
-    t_hbm = hbm_step / (peaks["hbm_gbs"] * 1e9)
-    t_pcie = pcie_step / (pcie_gbs * 1e9)
-    t_step = elapsed_ms * 1e-3 / K
-    dp = {k: stp1[k] - stp0[k] for k in stp0 if k not in ("error_bits", "debug_words")}
-    kern = {}
-    miss_b = dp["miss_pages"] * PAGE_BYTES
-    admit_b = (dp["miss_pages"] - dp["bypass_pages"]) * PAGE_BYTES
-    kv_b = (dp["selected_pages"] + dp["tail_pages"]) * PAGE_BYTES
-    fused = args.fetch_mode == 0
-    # algorithmic bytes per kernel over the profiled steps: (HBM bytes, host-link bytes)
-    bytes_of = dict(score=(dp["candidates_scored"] * (512 if w.partition_kind == 0 else 256), 0),
-                    fetch=(admit_b, admit_b),
-                    attn_split=((kv_b - miss_b + admit_b, miss_b) if fused else (kv_b - (miss_b - admit_b), miss_b - admit_b)))
-    tot_ms = sum(ms for _, ms in prof.values()) or 1.0
-    for name, (n, ms) in prof.items():
-        if not n:
-            continue
-        kern[name] = dict(launches=n, avg_us=1e3 * ms / n, share=ms / tot_ms)
-        if name in bytes_of:
-            hb, pb = bytes_of[name]
-            t_h, t_p = hb / (peaks["hbm_gbs"] * 1e9), pb / (pcie_gbs * 1e9)
-            kern[name].update(hbm_gbs=hb / (ms * 1e-3) / 1e9, pcie_gbs=pb / (ms * 1e-3) / 1e9,
-                              bound="pcie" if t_p > t_h else "hbm", roof_frac=max(t_h, t_p) / (ms * 1e-3))
-    top = max((k_ for k_ in ("fetch", "score", "attn_split") if k_ in kern), key=lambda k_: kern[k_]["share"])
-    bound = kern[top]["bound"]
-    peak = pcie_gbs if bound == "pcie" else peaks["hbm_gbs"]
-    achieved = kern[top]["pcie_gbs"] if bound == "pcie" else kern[top]["hbm_gbs"]
-    traffic = (NCU_TRAFFIC.get(args.workload) or {}).get(top) if not (args.context or args.batch or args.layers) else None
-    names = dict(fetch="k_fetch", score="k_score", attn_split="k_attn (attention + page fetch)" if fused else "k_attn")
-    roofline = dict(kernel=names[top], bound=bound, achieved=achieved, peak=peak, unit="GB/s",
-                    frac=kern[top]["roof_frac"], traffic=traffic,
-                    peak_source=("pinned H2D copy measured in this run" if bound == "pcie" else peaks["source"]),
-                    avg_launch_us=kern[top]["avg_us"],
-                    hbm_bytes_per_launch=bytes_of[top][0] / kern[top]["launches"],
-                    pcie_bytes_per_launch=bytes_of[top][1] / kern[top]["launches"])
+    head = summarise(rec, args, K, world, elapsed_ms, pcie_gbs, peaks, fused, full_size)
+    head["step_roofline"]["pcie_link"] = link
     line = dict(
-        metric=metric, value=value, unit=unit, n_gpus=world, steps=K, warmup=Wm, ms_per_step=elapsed_ms / K,
+        metric=metric, value=head["value"], unit=unit, n_gpus=world, steps=K, warmup=Wm, ms_per_step=head["ms_per_step"],
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16 in, f32 accumulate", data="synthetic",
-        config=dict(cfg_desc, primed_steps=P, l2="flushed between timed steps (256 MiB written then read back, untimed)",
+        config=dict(cfg_desc, primed_steps=head["primed_steps"],
+                    prime="untimed decode steps until the slots are full and every step evicts (cap --prime-cap)",
+                    l2="flushed between timed steps (256 MiB written then read back, untimed)",
                     note="single-layer config: tokens/s is per-layer-step throughput"),
-        p50_tpot_ms=statistics.median(per_step), ms_per_step_noflush=noflush_ms,
-        gpu_launches=int(d["kernel_launches"]), clocks=clocks,
-        step_roofline=dict(hbm_bytes_per_step=hbm_step, pcie_bytes_per_step=pcie_step,
-                           hbm_gbs_peak=peaks["hbm_gbs"], hbm_peak_source=peaks["source"], pcie_gbs_peak=pcie_gbs,
-                           t_hbm_us=1e6 * t_hbm, t_pcie_us=1e6 * t_pcie, t_step_us=1e6 * t_step,
-                           bound="pcie" if t_pcie > t_hbm else "hbm", frac=max(t_hbm, t_pcie) / t_step,
-                           frac_vs_nominal_8tbs=max(hbm_step / 8e12, t_pcie) / t_step, pcie_link=link,
-                           miss_ratio=d["miss_pages"] / max(d["selected_pages"], 1)),
-        roofline=roofline, kernels=kern, error_bits=final["error_bits"])
+        p50_tpot_ms=head["p50_tpot_ms"], ms_per_step_noflush=head["ms_per_step_noflush"],
+        gpu_launches=head["gpu_launches"], clocks=clocks, step_roofline=head["step_roofline"],
+        roofline=head["roofline"], kernels=head["kernels"], miss_ratio=head["miss_ratio"],
+        evicted_pages_per_step=head["evicted_pages_per_step"], missed_pages_per_step=head["missed_pages_per_step"],
+        error_bits=head["error_bits"])
+    cold_steps = rec["cold_steps"]
     n_cold = min(8, len(cold_steps))
     if n_cold:
         # the first steps after prefill start from an empty GPU cache (every selected page misses)
         line["cold_start"] = dict(steps=n_cold, first_step_ms=cold_steps[0],
                                   mean_ms_per_step=sum(cold_steps[:n_cold]) / n_cold)
-    if e2e_steps:
-        line["e2e"] = dict(value=B * e2e_steps * world / (e2e_ms * 1e-3), unit=unit, h2d_bytes_per_step=h2d,
-                           d2h_bytes_per_step=d2h, ms_per_step=e2e_ms / e2e_steps)
-    run.close()
-    del run
+    if "e2e_ms" in rec:
+        line["e2e"] = dict(value=rec["B"] * K * world / (e2e_ms * 1e-3), unit=unit, h2d_bytes_per_step=rec["h2d"],
+                           d2h_bytes_per_step=rec["d2h"], ms_per_step=e2e_ms / K)
+
+    # the other benchmark configurations, each at its full size (the mixed-length one scaled to
+    # this box and labelled), fewer timed steps: which of them meet the roofline target
+    if world == 1 and not args.no_per_config and full_size and args.workload == "c2":
+        per = {}
+        others = [("c1", {}, "as worded"), ("c3", {}, "as worded"), ("c4", {}, "as worded"),
+                  ("c5_scaled", dict(batch=16, num_layers=1),
+                   "SCALED to this box: 16 of the 64 requests, 1 of the 32 layers, the same per-request and "
+                   "per-layer share of the 60 GB budget (the configuration as worded needs ~1.1 TB of pinned host memory)")]
+        Kp = args.per_config_steps
+        for name, kw, label in others:
+            b2 = W.scaled(W.CONFIGS[name.split("_")[0]], **kw)
+            smp = ClockSampler(gpu_id)
+            r2 = measure(b2, args, Kp, Wm, 0, 1, device, False, pcie_gbs, peaks, cache_budget(b2))
+            ck = smp.stop(r2["t_begin"], r2["t_end"])
+            s2 = summarise(r2, args, Kp, 1, sum(r2["per_step"]), pcie_gbs, peaks, fused, not kw)
+            s2.update(config=workload_desc(b2, 1)["workload"], size=label, steps=Kp, clocks=ck,
+                      meets_0p60=bool(s2["step_roofline"]["frac"] >= 0.60))
+            s2.pop("kernels")
+            per[name] = s2
+        line["per_config"] = per
+        line["target"] = dict(step_roofline_frac=0.60,
+                              met={**{"c2": bool(head["step_roofline"]["frac"] >= 0.60)},
+                                   **{k_: v_["meets_0p60"] for k_, v_ in per.items()}})
     if world == 1 and not args.no_cpu_baseline:
-        r = oracle_run(base, budget_s=20.0, steps_cap=64, warmup=1)
+        r = oracle_run(base, budget_s=15.0, steps_cap=64, warmup=1)
         line["cpu_baseline"] = dict(value=r["value"], unit=unit, cores=r["cores"], kind="oracle", sample=r["sample"])
+        line["cpu_baseline_all_cores"] = oracle_all_cores(args.workload, overrides, 15.0, 64)
     print(json.dumps(line))
     if world > 1:
         dist.barrier()

@@ -41,68 +41,87 @@ __device__ __forceinline__ float fma_bf16(uint16_t a, uint16_t b, float c) {
   return d;
 }
 
-// Score of one entry for this lane's 8 channels, all G heads; the 16 lanes of the row are
-// combined by the caller-visible butterfly.  For min/max summaries max(q*min, q*max) equals
+// Scores of E candidates at once for this lane's 8 channels and all G heads; the 16 lanes of a
+// row are combined by a butterfly.  For min/max summaries max(q*min, q*max) equals
 // q * (q >= 0 ? max : min) exactly (min <= max and the products are exact), so the operand is
 // picked with one bitwise blend per channel pair on the packed bf16 words (masks precomputed
 // per head) instead of two multiplies and a max per channel.
-template <int G, bool MINMAX>
-__device__ __forceinline__ float score_entry(const uint4 lo, const uint4 hi, const uint32_t (&qw)[G][4],
-                                             const uint32_t (&qsel)[G][4], uint32_t row_mask) {
-  const uint32_t a[4] = {lo.x, lo.y, lo.z, lo.w}, m[4] = {hi.x, hi.y, hi.z, hi.w};
-  float v[G];
+// The E x G block sums of a lane go up the balanced tree together (lanes l and l^1, then l^2,
+// l^4, l^8: both partners form the same sum, addition being commutative).  While more than one
+// value is left in a lane, a level also halves that number: the partners keep one half of the
+// values each and trade the other, so a level costs n/2 shuffles instead of n, and the
+// shuffles of a level are independent of one another (their latency is paid once per level,
+// not once per candidate).  After log2(E x G) levels a lane holds one (candidate, head) total;
+// the heads of a candidate are then added in ascending order.
+// Returns the lane's candidate total; *which = the candidate (0..E-1) it belongs to, *writer =
+// this lane is the one that stores it.
+template <int G, bool MINMAX, int E>
+__device__ __forceinline__ float score_group(const uint4 (&lo)[E], const uint4 (&hi)[E], const uint32_t (&qw)[G][4],
+                                             const uint32_t (&qsel)[G][4], uint32_t row_mask, int *which, bool *writer) {
+  constexpr int N = E * G;
+  static_assert(N <= 16 && (N & (N - 1)) == 0, "one value per lane of the row at most");
+  constexpr int K = N == 16 ? 4 : N == 8 ? 3 : N == 4 ? 2 : N == 2 ? 1 : 0;      // trading levels
+  constexpr int KG = G == 8 ? 3 : G == 4 ? 2 : G == 2 ? 1 : 0, KE = K - KG;
+  float v[N];
 #pragma unroll
-  for (int g = 0; g < G; ++g) v[g] = -0.0f;                     // -0.0 + p = p for every p: the first term is the bare product
+  for (int i = 0; i < N; ++i) v[i] = -0.0f;                    // -0.0 + p = p for every p: the first term is the bare product
   // channels left to right, one rounding per add (the mixed-precision fma takes the bf16 halves
-  // as they are: exact product, fp32 sum); the G heads' chains advance together
+  // as they are: exact product, fp32 sum); the E x G chains advance together
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    uint16_t xl[G], xh[G], ql[G], qh[G];
+    uint16_t xl[N], xh[N], ql[G], qh[G];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const uint32_t w = MINMAX ? ((m[j] & qsel[g][j]) | (a[j] & ~qsel[g][j])) : a[j];
-      asm("mov.b32 {%0, %1}, %2;" : "=h"(xl[g]), "=h"(xh[g]) : "r"(w));
-      asm("mov.b32 {%0, %1}, %2;" : "=h"(ql[g]), "=h"(qh[g]) : "r"(qw[g][j]));
+    for (int g = 0; g < G; ++g) asm("mov.b32 {%0, %1}, %2;" : "=h"(ql[g]), "=h"(qh[g]) : "r"(qw[g][j]));
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const uint32_t a = j == 0 ? lo[e].x : j == 1 ? lo[e].y : j == 2 ? lo[e].z : lo[e].w;
+      const uint32_t m = j == 0 ? hi[e].x : j == 1 ? hi[e].y : j == 2 ? hi[e].z : hi[e].w;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const uint32_t w = MINMAX ? ((m & qsel[g][j]) | (a & ~qsel[g][j])) : a;
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(xl[e * G + g]), "=h"(xh[e * G + g]) : "r"(w));
+      }
     }
 #pragma unroll
-    for (int g = 0; g < G; ++g) v[g] = fma_bf16(ql[g], xl[g], v[g]);
+    for (int i = 0; i < N; ++i) v[i] = fma_bf16(ql[i % G], xl[i], v[i]);
 #pragma unroll
-    for (int g = 0; g < G; ++g) v[g] = fma_bf16(qh[g], xh[g], v[g]);
+    for (int i = 0; i < N; ++i) v[i] = fma_bf16(qh[i % G], xh[i], v[i]);
   }
-  // The 16 block sums of every head go up the balanced tree (lanes l and l^1, then l^2, l^4,
-  // l^8: both partners form the same sum, addition being commutative).  While more than one
-  // head is left in a lane, a level also halves that number: the partners keep one half of
-  // the heads each and trade the other, so a level costs n/2 shuffles instead of n.  Lane l
-  // of a row ends up with the total of the head whose index is l's low bits reversed.
   const int lane = threadIdx.x & 15;
-  int n = G;
 #pragma unroll
   for (int level = 0; level < 4; ++level) {
-    if (n > 1) {
+    if (level < K) {
       const bool up = (lane >> level) & 1;
-      const int half = n / 2;
+      const int half = N >> (level + 1);
 #pragma unroll
-      for (int i = 0; i < G / 2; ++i)
+      for (int i = 0; i < N / 2; ++i)
         if (i < half) {
           const float send = up ? v[i] : v[i + half], keep = up ? v[i + half] : v[i];
           v[i] = keep + __shfl_xor_sync(row_mask, send, 1 << level);
         }
-      n = half;
     } else {
       v[0] = v[0] + __shfl_xor_sync(row_mask, v[0], 1 << level);
     }
   }
-  // heads in ascending order, into the row's first lane
-  float tot = v[0];
+  // lane bit `level` chose index bit K-1-level: candidate = the top KE index bits, head = the low KG
+  int e_idx = 0;
 #pragma unroll
-  for (int h = 1; h < G; ++h) {
-    constexpr int kBits = G == 8 ? 3 : G == 4 ? 2 : 1;
-    int src = 0;
+  for (int level = 0; level < KE; ++level) e_idx |= ((lane >> level) & 1) << (KE - 1 - level);
+  int head_lanes = 0;                                            // the lane bits that say which head the lane holds
 #pragma unroll
-    for (int bit = 0; bit < kBits; ++bit) src |= ((h >> bit) & 1) << (kBits - 1 - bit);
-    tot = tot + __shfl_sync(row_mask, v[0], src, 16);
+  for (int t = 0; t < KG; ++t) head_lanes |= 1 << (K - 1 - t);
+  float tot = 0.f;
+#pragma unroll
+  for (int h = 0; h < G; ++h) {                                  // heads in ascending order
+    int src = lane & ~head_lanes;
+#pragma unroll
+    for (int t = 0; t < KG; ++t) src |= ((h >> t) & 1) << (K - 1 - t);
+    const float sh = G > 1 ? __shfl_sync(row_mask, v[0], src, 16) : v[0];
+    tot = h == 0 ? sh : tot + sh;
   }
-  return tot + 0.0f;                              // -0.0 -> +0.0
+  *which = e_idx;
+  *writer = (lane & head_lanes) == 0 && (lane >> K) == 0;
+  return tot + 0.0f;                                             // -0.0 -> +0.0
 }
 
 // How the scoring kernel cuts a step into work items.  Items run in this order: the sets' tail
@@ -205,16 +224,31 @@ __device__ __forceinline__ void score_item(const DevCtx &c, const Batch &bt, con
       if (!done) { *s_dead = 1; if (lane16 == 0) dev_error(c, kErrTimeout); }
       phase_bits ^= 1u << gI;
     }
+    // the quarter's candidates of this half-warp, kE at a time (as many as give every lane of
+    // the row one value to carry up the tree)
+    constexpr int kE = kPerGroup * G <= 16 ? kPerGroup : 16 / G;
 #pragma unroll
-    for (int j = 0; j < kPerGroup; ++j) {
-      const int slot = gI * kPerGroup + j, e = grp + 16 * slot;
-      if (e < n_here && !dead) {
-        const uint4 a0 = *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry);
-        const uint4 m0 = MINMAX ? *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry + kRowBytes)
-                                : make_uint4(0, 0, 0, 0);
-
-        const float s0 = score_entry<G, MINMAX>(a0, m0, qw, qsel, row_mask);
-        if (lane16 == 0) out[e] = s0;
+    for (int j0 = 0; j0 < kPerGroup; j0 += kE) {
+      uint4 a0[kE], m0[kE];
+      bool any = false;
+#pragma unroll
+      for (int u = 0; u < kE; ++u) {
+        const int e = grp + 16 * (gI * kPerGroup + j0 + u);
+        if (e < n_here && !dead) {
+          a0[u] = *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry);
+          m0[u] = MINMAX ? *reinterpret_cast<const uint4 *>(stage + (size_t)e * kEntry + kRowBytes) : make_uint4(0, 0, 0, 0);
+          any = true;
+        } else {
+          a0[u] = make_uint4(0, 0, 0, 0);
+          m0[u] = make_uint4(0, 0, 0, 0);
+        }
+      }
+      if (any) {                                                   // uniform over the row: a candidate exists for all its lanes or for none
+        int which;
+        bool writer;
+        const float s0 = score_group<G, MINMAX, kE>(a0, m0, qw, qsel, row_mask, &which, &writer);
+        const int e = grp + 16 * (gI * kPerGroup + j0 + which);
+        if (writer && e < n_here) out[e] = s0;
       }
     }
   }
