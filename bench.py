@@ -103,21 +103,41 @@ def pcie_link(gpu_id: str):
         return None
 
 
-def measure_pcie_gbs(torch, device, stream) -> float:
-    """Peak of the host link as one large pinned host->device copy (best of 5)."""
+def measure_pcie_gbs(torch, device, stream) -> dict:
+    """Peak of the host link, host to device: the better of a large pinned copy-engine transfer
+    (best of 10) and of SM-issued reads of pinned memory by a grid that fills the GPU (the
+    library's link probe, best of 6).  The host is shared with other jobs, so single
+    measurements wander by 10-20%; the best one is the link's peak."""
+    import paper_2604_26837_b200 as P
     n = 256 << 20
     src = torch.empty(n, dtype=torch.uint8).pin_memory()
     dst = torch.empty(n, dtype=torch.uint8, device=device)
-    best = 0.0
+    dma = 0.0
     with torch.cuda.stream(stream):
-        for _ in range(6):
+        for _ in range(10):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             dst.copy_(src, non_blocking=True)
             e1.record(stream)
             e1.synchronize()
-            best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
-    return best
+            dma = max(dma, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del src, dst
+    # a small context just for its pinned host tier (256 MiB of pages)
+    cfg = P.make_config(device=device.index or 0, num_layers=1, num_q_heads=4, num_kv_heads=1, max_requests=1,
+                        max_context_tokens=4096, partition_kind=0, topk=16, gpu_cache_pages=64, host_pages=32768)
+    ctx = P.Spin(cfg, device)
+    sm = 0.0
+    with torch.cuda.stream(stream):
+        for _ in range(7):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            ctx.debug_link_probe(32768, stream)
+            e1.record(stream)
+            e1.synchronize()
+            sm = max(sm, 32768 * 8192 / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    ctx.close()
+    return dict(gbs=max(dma, sm), copy_engine_gbs=dma, sm_read_gbs=sm,
+                source="best of a 256 MiB pinned copy-engine transfer and of SM-issued reads of pinned memory, measured in this run")
 
 
 def oracle_run(w, budget_s: float, steps_cap: int, warmup: int, sample_requests: int = 1, first_request: int = 0):
@@ -391,7 +411,7 @@ def summarise(rec, args, K, world, elapsed_ms, pcie_gbs, peaks, fused, full_size
     names = dict(fetch="k_fetch", score="k_score", attn_split="k_attn (attention + page fetch)" if fused else "k_attn")
     roofline = dict(kernel=names[top], bound=bound, achieved=achieved, peak=peak, unit="GB/s",
                     frac=kern[top]["roof_frac"], traffic=traffic,
-                    peak_source=("pinned H2D copy measured in this run" if bound == "pcie" else peaks["source"]),
+                    peak_source=("host link peak measured in this run (see step_roofline.pcie_peak)" if bound == "pcie" else peaks["source"]),
                     avg_launch_us=kern[top]["avg_us"],
                     hbm_bytes_per_launch=bytes_of[top][0] / kern[top]["launches"],
                     pcie_bytes_per_launch=bytes_of[top][1] / kern[top]["launches"])
@@ -514,7 +534,8 @@ def main():
     torch.cuda.set_device(device)
     K, Wm = args.steps, args.warmup
     peaks = load_peaks()
-    pcie_gbs = measure_pcie_gbs(torch, device, torch.cuda.Stream(device))
+    link_peak = measure_pcie_gbs(torch, device, torch.cuda.Stream(device))
+    pcie_gbs = link_peak["gbs"]
     props = torch.cuda.get_device_properties(device)
     gpu_id = f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank)
     fused = args.fetch_mode == 0
@@ -538,6 +559,7 @@ def main():
 
     head = summarise(rec, args, K, world, elapsed_ms, pcie_gbs, peaks, fused, full_size)
     head["step_roofline"]["pcie_link"] = link
+    head["step_roofline"]["pcie_peak"] = link_peak
     line = dict(
         metric=metric, value=head["value"], unit=unit, n_gpus=world, steps=K, warmup=Wm, ms_per_step=head["ms_per_step"],
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16 in, f32 accumulate", data="synthetic",

@@ -272,6 +272,13 @@ SPIN_API int spin_decode_step_append(spin_ctx *ctx, int32_t layer, const int32_t
  * accesses that were skipped and leave the status at SPIN_OK). */
 SPIN_API int spin_stats(spin_ctx *ctx, spin_stats_t *out);
 
+/* Measures what the host link gives a kernel (Section 5.5 aims to saturate it; Eq. 3's BW_PCIe):
+ * reads `n_pages` pages of 8 KiB of the context's pinned host tier (wrapping around it) with a
+ * grid that fills the GPU, a warp per page as the page fetch does, and discards them.  The
+ * caller times it with events on cuda_stream: n_pages x 8192 bytes over the elapsed time is the
+ * rate of SM-issued reads over the link.  Asynchronous; no state is changed. */
+SPIN_API int spin_debug_link_probe(spin_ctx *ctx, int64_t n_pages, void *cuda_stream);
+
 /* Exercises the bounded-wait path (Section 5.3 keeps all control on the GPU, so kernels of a
  * step wait on one another's flags; every such wait has a poll limit): one warp polls, at most
  * `max_polls` times (1..4096, well under a millisecond), a flag word for a value that is never

@@ -1363,6 +1363,14 @@ int spin_stats(spin_ctx *ctx, spin_stats_t *out) {
   return SPIN_OK;
 }
 
+int spin_debug_link_probe(spin_ctx *ctx, int64_t n_pages, void *cuda_stream) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  if (n_pages < 1 || n_pages > (1ll << 22)) return fail(ctx, SPIN_ERR_INVALID, "n_pages must be 1..4194304");
+  ctx->launches += launch_link_probe(ctx->d, (int)n_pages, reinterpret_cast<cudaStream_t>(cuda_stream), ctx->sm_count);
+  CK(cudaGetLastError());
+  return SPIN_OK;
+}
+
 int spin_debug_wait_probe(spin_ctx *ctx, int32_t max_polls, void *cuda_stream) {
   if (!ctx) return SPIN_ERR_INVALID;
   if (max_polls < 1 || max_polls > 4096) return fail(ctx, SPIN_ERR_INVALID, "max_polls must be 1..4096");

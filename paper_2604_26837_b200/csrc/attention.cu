@@ -344,6 +344,7 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
   // the stride being a multiple of the group), then the outputs are accumulated over tiles of
   // kMergeTile chunks whose weights exp2(m_k - m) sit in shared memory.
   constexpr int kThreads = kAttnWarps * 32, kMergeTile = 512;
+  static_assert(kThreads == kHeadDim, "thread t of the merge owns channel t of every head");
   const float *parts = c.att_part + (size_t)b * c.max_chunks * G * kPartStride;
   float *s_red = reinterpret_cast<float *>(smem_pages);           // [kThreads]
   float *s_mx = s_red + kThreads;                                 // [G] the set's max per head
@@ -387,22 +388,25 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
       s_scale[e] = mk == -INFINITY ? 0.f : exp2f(mk - s_mx[e % G]);
     }
     __syncthreads();
+    // a thread's G outputs are channel `threadIdx.x` of every head: the loads of a batch of chunks
+    // for all G heads are issued together (their L2 latency is paid once per batch, not once per head)
+    const float *pt = parts + (size_t)k0 * G * kPartStride + threadIdx.x;
+    constexpr int kB = G >= 8 ? 4 : 8;                            // chunks per batch: 32 loads in flight per thread
+    int k = 0;
+    for (; k + kB <= kn; k += kB) {
+      float v[G][kB];
 #pragma unroll
-    for (int j = 0; j < G; ++j) {
-      const int e = threadIdx.x + j * kThreads, g = e / kHeadDim, ch = e % kHeadDim;
-      const float *pg_ = parts + ((size_t)k0 * G + g) * kPartStride + ch;
-      float acc = a_o[j];
-      int k = 0;
-      for (; k + 8 <= kn; k += 8) {
-        float v[8];
+      for (int j = 0; j < G; ++j)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = __ldcg(pg_ + (size_t)(k + i) * G * kPartStride);
+        for (int i = 0; i < kB; ++i) v[j][i] = __ldcg(pt + ((size_t)(k + i) * G + j) * kPartStride);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc = fmaf(v[i], s_scale[(k + i) * G + g], acc);
-      }
-      for (; k < kn; ++k) acc = fmaf(__ldcg(pg_ + (size_t)k * G * kPartStride), s_scale[k * G + g], acc);
-      a_o[j] = acc;
+      for (int j = 0; j < G; ++j)
+#pragma unroll
+        for (int i = 0; i < kB; ++i) a_o[j] = fmaf(v[j][i], s_scale[(k + i) * G + j], a_o[j]);
     }
+    for (; k < kn; ++k)
+#pragma unroll
+      for (int j = 0; j < G; ++j) a_o[j] = fmaf(__ldcg(pt + ((size_t)k * G + j) * kPartStride), s_scale[k * G + j], a_o[j]);
   }
 #pragma unroll
   for (int j = 0; j < G; ++j) {
@@ -410,6 +414,7 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
     const float den = s_den[g];
     out[((size_t)i_req * c.Hq + head * G + g) * kHeadDim + ch] = __float2bfloat16(den > 0.f ? a_o[j] / den : 0.f);
   }
+  dbg_ta(b, 15);
 }
 
 // The kernel: the CTA's work; one CTA then waits for the kernel before this one.  CTAs that

@@ -1022,8 +1022,8 @@ int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_
     }
   }
   // resident form (grid sized in launch_score_g) when scoring is many waves long
-  sg.persistent = (!stream && fuse == 2 && c.ready && c.resident_scoring >= 0 &&
-                   (c.resident_scoring == 1 || sg.n_items > 12 * sm_count_of_device())) ? 1 : 0;
+  sg.persistent = (!stream && (fuse == 2 || fuse == 3) && c.ready && c.resident_scoring >= 0 &&
+                   (c.resident_scoring == 1 || (fuse == 2 && sg.n_items > 12 * sm_count_of_device()))) ? 1 : 0;
   dim3 grid(sg.n_items);
   if (!stream) b.attn_set_major = sg.persistent;
   if (!stream) {

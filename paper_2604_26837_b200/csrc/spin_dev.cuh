@@ -334,6 +334,7 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
 int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
 int launch_shrink(const DevCtx &c, int req, int old_S, int new_S, cudaStream_t st);
 int launch_wait_probe(const DevCtx &c, int max_polls, cudaStream_t st);
+int launch_link_probe(const DevCtx &c, int n_pages, cudaStream_t st, int sm_count);
 int launch_assign(const DevCtx &c, int req, int layer, int n_clusters, int n_tokens, int32_t *assign, cudaStream_t st);
 int launch_move_rows(const DevCtx &c, int req, int layer, const int64_t *dest, int n_tokens, cudaStream_t st);
 int launch_reindex_apply(const DevCtx &c, int req, int layer, int n_clusters, int n_folded_pages, int tail_first,

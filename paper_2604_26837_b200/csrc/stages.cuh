@@ -160,6 +160,7 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
   // keys -> shared memory, with the OR and AND of the slice taken on the way
   {
     uint32_t k_or = 0, k_and = 0xffffffffu;
+#pragma unroll 8
     for (int i = tid; i < m; i += T) {
       float sc;
       if (xfer) { sc = take_score(c, xfer_in + lo + i); scores[lo + i] = sc; }
