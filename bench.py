@@ -370,6 +370,18 @@ def measure(base, args, K, Wm, rank, world, device, do_e2e, pcie_gbs, peaks, cac
         rec["e2e_ms"] = 1e3 * sum(e2e_times)
         rec["h2d"] = L * (qh[0, 0].numel() + kh[0, 0].numel() + vh[0, 0].numel()) * 2
         rec["d2h"] = L * oh.numel() * 2
+    # the design's latency floor: two chained launches and one flag hand-over, timed like a step
+    floor = []
+    with torch.cuda.stream(stream):
+        for _ in range(24):
+            flush_l2_fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            run.spin.debug_launch_floor(stream)
+            e1.record(stream)
+            floor.append((e0, e1))
+    torch.cuda.synchronize(device)
+    rec["floor_us"] = 1e3 * statistics.median(a.elapsed_time(b) for a, b in floor[4:])
     rec["final"] = run.spin.stats()
     rec["setup_s"] = time.perf_counter() - t_setup
     run.close()
@@ -428,7 +440,10 @@ def summarise(rec, args, K, world, elapsed_ms, pcie_gbs, peaks, fused, full_size
                 miss_ratio=step_roofline["miss_ratio"], evicted_pages_per_step=d["evicted_pages"] / K,
                 missed_pages_per_step=d["miss_pages"] / K, sets_per_step=sets, primed_steps=rec["primed"],
                 gpu_launches=int(d["kernel_launches"]), error_bits=rec["final"]["error_bits"],
-                setup_s=round(rec["setup_s"], 1))
+                setup_s=round(rec["setup_s"], 1),
+                latency_floor=dict(us=rec["floor_us"], step_over_floor=(elapsed_ms / K * 1e3) / max(rec["floor_us"], 1e-9),
+                                   what="two empty kernels chained by programmatic dependent launch with one flag "
+                                        "hand-over, same stream, CUDA events, L2 flushed: what a step costs before it touches KV"))
 
 
 def workload_desc(base, world):
@@ -571,7 +586,7 @@ def main():
         gpu_launches=head["gpu_launches"], clocks=clocks, step_roofline=head["step_roofline"],
         roofline=head["roofline"], kernels=head["kernels"], miss_ratio=head["miss_ratio"],
         evicted_pages_per_step=head["evicted_pages_per_step"], missed_pages_per_step=head["missed_pages_per_step"],
-        error_bits=head["error_bits"])
+        latency_floor=head["latency_floor"], error_bits=head["error_bits"])
     cold_steps = rec["cold_steps"]
     n_cold = min(8, len(cold_steps))
     if n_cold:

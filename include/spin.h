@@ -128,8 +128,10 @@ typedef struct spin_config {
                                    host memory on a stream of the library's own; the caller's
                                    stream goes on at once (it waits only when the ring is full),
                                    and a later decode step waits for the pages it may fetch.
-                                   Page / token / page-mean granularity; at least 4 pages of
-                                   every kv head must fit (4 x 8 KiB x num_kv_heads x 4 bytes) */
+                                   Cluster granularity: the prefill's rows are packed into their
+                                   clusters' pages in the ring, range by range of the sets'
+                                   pages, and drain the same way.  At least 4 pages of every kv
+                                   head must fit (4 x 8 KiB x num_kv_heads x 4 bytes) */
   int64_t gpu_cache_pages;      /* HBM pages (8 KiB each) shared by all sets' cache slots */
   int64_t host_pages;           /* pinned host pages (8 KiB each) for the complete KV */
   void *hbm_pool;               /* device pointer, 256-byte aligned, caller-owned */
@@ -278,6 +280,14 @@ SPIN_API int spin_stats(spin_ctx *ctx, spin_stats_t *out);
  * caller times it with events on cuda_stream: n_pages x 8192 bytes over the elapsed time is the
  * rate of SM-issued reads over the link.  Asynchronous; no state is changed. */
 SPIN_API int spin_debug_link_probe(spin_ctx *ctx, int64_t n_pages, void *cuda_stream);
+
+/* The latency floor of a decode step in this design (Section 5.3 keeps control on the GPU: a step
+ * is two kernels chained by programmatic dependent launch that hand work over through flags):
+ * enqueues two one-warp kernels launched the same way, the second of which waits for a flag the
+ * first raises, and nothing else.  Timed by the caller with events on cuda_stream, it is what a
+ * step costs before it has touched a byte of KV; a single-set step is a small multiple of it.
+ * Asynchronous. */
+SPIN_API int spin_debug_launch_floor(spin_ctx *ctx, void *cuda_stream);
 
 /* Exercises the bounded-wait path (Section 5.3 keeps all control on the GPU, so kernels of a
  * step wait on one another's flags; every such wait has a poll limit): one warp polls, at most

@@ -24,7 +24,7 @@ PAGE_BYTES = 8192
 EXPORTS = ["spin_required_bytes", "spin_create", "spin_destroy", "spin_request_open", "spin_reindex",
            "spin_request_close", "spin_set_budget", "spin_append_kv", "spin_append_kv_batch", "spin_decode_step",
            "spin_decode_step_append", "spin_stats", "spin_profile", "spin_profile_read", "spin_debug_dump",
-           "spin_debug_read_page", "spin_debug_wait_probe", "spin_debug_link_probe", "spin_paged_attention_static", "spin_last_error",
+           "spin_debug_read_page", "spin_debug_wait_probe", "spin_debug_link_probe", "spin_debug_launch_floor", "spin_paged_attention_static", "spin_last_error",
            "spin_version"]
 KERNEL_NAMES = ["append", "score", "topk", "cache", "fetch", "attn_split", "unused"]
 
@@ -117,6 +117,7 @@ def load() -> C.CDLL:
     lib.spin_debug_read_page.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
     lib.spin_debug_wait_probe.argtypes = [vp, i32, vp]
     lib.spin_debug_link_probe.argtypes = [vp, C.c_int64, vp]
+    lib.spin_debug_launch_floor.argtypes = [vp, vp]
     lib.spin_paged_attention_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
     lib.spin_last_error.argtypes = [vp]
     lib.spin_last_error.restype = C.c_char_p
@@ -270,6 +271,9 @@ class Spin:
         out["debug_words"] = list(s.debug_words)
         out["status"] = rc
         return out
+
+    def debug_launch_floor(self, stream=None):
+        self._ck(self.lib.spin_debug_launch_floor(self.h, _stream_ptr(stream)))
 
     def debug_link_probe(self, n_pages: int, stream=None):
         self._ck(self.lib.spin_debug_link_probe(self.h, n_pages, _stream_ptr(stream)))

@@ -176,6 +176,7 @@ struct spin_ctx {
   size_t dir_bytes_in_use = 0;
   Prof prof;
   int32_t epoch = 0;                 // decode calls so far (value of the per-set ready flags)
+  uint32_t floor_calls = 0;          // spin_debug_launch_floor calls (their flag values)
   // asynchronous offload: a ring of kOffloadSlots staging slots in HBM, drained by copy-engine
   // transfers on offload_stream; slot i is free again once ev_done[i] has happened
   static constexpr int kOffloadSlots = 4;
@@ -628,8 +629,55 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
     cen = reinterpret_cast<const __nv_bfloat16 *>(cen_tmp);
   }
   ctx->launches += launch_copy_centroids(d, req, layer, cen, C, st);
-  // rows -> host pages, in chunks through the staging buffers
   const bool dev_kv = is_device_ptr(k);
+  if (dev_kv && ctx->offload_slot_units > 0) {
+    // Asynchronous offload (Section 4.1): the rows are packed into pages in HBM staging slots on
+    // the caller's stream, at HBM speed, range by range of the sets' logical pages; each slot
+    // then moves to host memory by copy-engine transfers (one per run of consecutive host
+    // pages) on the library's stream, behind this call.
+    std::vector<int32_t> lrow((size_t)n * H);
+    std::fill(filled.begin(), filled.end(), 0);
+    for (int64_t t = 0; t < n; ++t)
+      for (int h = 0; h < H; ++h) {
+        const int32_t c = tp[(size_t)t * H + h];
+        const int32_t r = filled[(size_t)h * C + c]++;
+        lrow[(size_t)t * H + h] = (first_row_page[(size_t)h * C + c] + r / kPageTokens) * kPageTokens + r % kPageTokens;
+      }
+    int32_t *d_lrow = nullptr;
+    CK(cudaMalloc(reinterpret_cast<void **>(&d_lrow), lrow.size() * 4));
+    CK(cudaMemcpyAsync(d_lrow, lrow.data(), lrow.size() * 4, cudaMemcpyHostToDevice, st));
+    const int64_t per = ctx->offload_slot_units / H;
+    for (int64_t p0 = 0; p0 < total_pages_max; p0 += per) {
+      const int m = (int)std::min<int64_t>(per, total_pages_max - p0), slot = ctx->offload_next;
+      ctx->offload_next = (slot + 1) % spin_ctx::kOffloadSlots;
+      if (ctx->slot_used[slot]) CK(cudaStreamWaitEvent(st, ctx->ev_done[slot], 0));     // ring full: wait for the drain
+      uint8_t *stage = ctx->offload_stage + (size_t)slot * ctx->offload_slot_units * kPageBytes;
+      CK(cudaMemsetAsync(stage, 0, (size_t)H * m * kPageBytes, st));                   // rows past a cluster's last token stay zero
+      ctx->launches += launch_cluster_scatter_staged(d, reinterpret_cast<const __nv_bfloat16 *>(k),
+                                                     reinterpret_cast<const __nv_bfloat16 *>(v), d_lrow, (int)n, (int)p0, m, stage, st);
+      CK(cudaEventRecord(ctx->ev_staged[slot], st));
+      CK(cudaStreamWaitEvent(ctx->offload_stream, ctx->ev_staged[slot], 0));
+      for (int h = 0; h < H; ++h) {
+        const std::vector<int32_t> &hpv = set_of(ctx, req, layer, h).host_pages;
+        for (int i = 0; i < m;) {
+          const int32_t hp0 = hpv[(size_t)(p0 + i)];
+          if (hp0 < 0) { ++i; continue; }                                               // this head has fewer pages
+          int len = 1;
+          while (i + len < m && hpv[(size_t)(p0 + i + len)] == hp0 + len) ++len;
+          CK(cudaMemcpyAsync(ctx->h_pages + (size_t)hp0 * kPageBytes, stage + ((size_t)h * m + i) * kPageBytes,
+                             (size_t)len * kPageBytes, cudaMemcpyDeviceToHost, ctx->offload_stream));
+          i += len;
+        }
+      }
+      CK(cudaEventRecord(ctx->ev_done[slot], ctx->offload_stream));
+      ctx->slot_used[slot] = true;
+      ctx->offload_last = slot;
+      ++ctx->offload_gen;
+    }
+    CK(cudaStreamSynchronize(st));          // the host-side sources of this call's copies end here; the drain goes on
+    CK(cudaFree(d_lrow));
+  } else {
+  // rows -> host pages, in chunks through the staging buffers
   const int64_t chunk = g.stage_tokens;
   for (int64_t t0 = 0; t0 < n; t0 += chunk) {
     const int64_t m = std::min(chunk, n - t0);
@@ -645,6 +693,7 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
     CK(cudaMemcpyAsync(ctx->stage_dest, dest.data() + (size_t)t0 * H, rows * 8, cudaMemcpyHostToDevice, st));
     ctx->launches += launch_cluster_scatter(d, req, layer, kk, vv, ctx->stage_dest, (int)m, st);
     CK(cudaStreamSynchronize(st));
+  }
   }
   if (cen_tmp) CK(cudaFree(cen_tmp));
   CK(cudaGetLastError());
@@ -912,6 +961,7 @@ int spin_reindex(spin_ctx *ctx, int32_t req, int32_t layer, void *cuda_stream) {
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   LayerHost &L = ctx->reqs[(size_t)req].layers[(size_t)layer];
   if (!L.clustered) return fail(ctx, SPIN_ERR_STATE, "request %d has no cluster prefill yet", req);
+  if (int rc2 = wait_for_offload(ctx, st)) return rc2;     // prefill pages still on their way must not land on the moved rows
   const Geometry &g = ctx->g;
   const DevCtx &d = ctx->d;
   const int H = ctx->cfg.num_kv_heads, C = ctx->cfg.num_clusters;
@@ -1367,6 +1417,13 @@ int spin_debug_link_probe(spin_ctx *ctx, int64_t n_pages, void *cuda_stream) {
   if (!ctx) return SPIN_ERR_INVALID;
   if (n_pages < 1 || n_pages > (1ll << 22)) return fail(ctx, SPIN_ERR_INVALID, "n_pages must be 1..4194304");
   ctx->launches += launch_link_probe(ctx->d, (int)n_pages, reinterpret_cast<cudaStream_t>(cuda_stream), ctx->sm_count);
+  CK(cudaGetLastError());
+  return SPIN_OK;
+}
+
+int spin_debug_launch_floor(spin_ctx *ctx, void *cuda_stream) {
+  if (!ctx) return SPIN_ERR_INVALID;
+  ctx->launches += launch_floor(ctx->d, -(int)(++ctx->floor_calls & 0xffffff) - 1, reinterpret_cast<cudaStream_t>(cuda_stream));
   CK(cudaGetLastError());
   return SPIN_OK;
 }

@@ -71,6 +71,27 @@ k_cluster_scatter(DevCtx c, const __nv_bfloat16 *__restrict__ k, const __nv_bflo
   }
 }
 
+// The same through a staging slot in HBM (asynchronous offload): lrow[token][head] = the row's
+// place in its set's logical page order (CPU-page-table index * 16 + row); the rows whose page
+// lies in [p0, p0 + m) go to the slot, laid out head-major ([head][page - p0], the order in
+// which copy-engine transfers then move the pages to host memory), the others are left for
+// another pass.
+__global__ void __launch_bounds__(256)
+k_cluster_scatter_staged(DevCtx c, const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__restrict__ v,
+                         const int32_t *__restrict__ lrow, int n_tokens, int p0, int m, uint8_t *__restrict__ stage) {
+  const int piece = threadIdx.x & 15;
+  const size_t rows = (size_t)n_tokens * c.Hkv;
+  for (size_t row = (size_t)blockIdx.x * 16 + (threadIdx.x >> 4); row < rows; row += (size_t)gridDim.x * 16) {
+    const int32_t d = lrow[row];
+    const int lp = d >> 4;
+    if (lp < p0 || lp >= p0 + m) continue;
+    const int head = (int)(row % c.Hkv);
+    uint8_t *dst = stage + ((size_t)head * m + (lp - p0)) * kPageBytes + (size_t)(d & 15) * kRowBytes + piece * 16;
+    st16(dst, ld16(reinterpret_cast<const uint8_t *>(k) + row * kRowBytes + piece * 16));
+    st16(dst + kHalfPageBytes, ld16(reinterpret_cast<const uint8_t *>(v) + row * kRowBytes + piece * 16));
+  }
+}
+
 // Centroids [C][Hkv][d] -> the summary rows of each head's set.
 __global__ void __launch_bounds__(256)
 k_copy_centroids(DevCtx c, int req, int layer, const __nv_bfloat16 *__restrict__ cen, int n_clusters) {
@@ -135,6 +156,15 @@ int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloa
   int grid = (int)((rows + 15) / 16 < 148 * 16 ? (rows + 15) / 16 : 148 * 16);
   if (grid < 1) grid = 1;
   k_cluster_scatter<<<grid, 256, 0, st>>>(c, k, v, dest_row, n_tokens);
+  return 1;
+}
+
+int launch_cluster_scatter_staged(const DevCtx &c, const __nv_bfloat16 *k, const __nv_bfloat16 *v, const int32_t *lrow,
+                                  int n_tokens, int p0, int m, uint8_t *stage, cudaStream_t st) {
+  size_t rows = (size_t)n_tokens * c.Hkv;
+  int grid = (int)((rows + 15) / 16 < 148 * 16 ? (rows + 15) / 16 : 148 * 16);
+  if (grid < 1) grid = 1;
+  k_cluster_scatter_staged<<<grid, 256, 0, st>>>(c, k, v, lrow, n_tokens, p0, m, stage);
   return 1;
 }
 

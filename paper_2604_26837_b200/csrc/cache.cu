@@ -156,6 +156,29 @@ int launch_link_probe(const DevCtx &c, int n_pages, cudaStream_t st, int sm_coun
   return 1;
 }
 
+// The least a decode step of this design can take: its two launches, chained by programmatic
+// stream serialization like the step's kernels, with one flag handed from the first to the
+// second and nothing else to do.
+__global__ void k_floor_first(DevCtx c, int token) {
+  pdl_launch_next();
+  pdl_wait_prev();
+  if (threadIdx.x == 0) flag_publish(c.score_done, token);
+}
+__global__ void k_floor_second(DevCtx c, int token) {
+  pdl_launch_next();
+  if (threadIdx.x == 0) {
+    flag_wait(c, c.score_done, token);
+    pdl_wait_prev();                                // not to complete ahead of the kernel before it
+    *c.score_done = 0;                              // as the scoring kernel expects to find it
+  }
+}
+
+int launch_floor(const DevCtx &c, int token, cudaStream_t st) {
+  launch_pdl(k_floor_first, dim3(1), dim3(32), 0, st, 1, c, token);
+  launch_pdl(k_floor_second, dim3(1), dim3(32), 0, st, 1, c, token);
+  return 2;
+}
+
 int launch_wait_probe(const DevCtx &c, int max_polls, cudaStream_t st) {
   k_wait_probe<<<1, 32, 0, st>>>(c, max_polls);
   return 1;

@@ -324,6 +324,8 @@ int launch_append_edge(const DevCtx &c, const AppendEdgeArgs &a, const __nv_bflo
 int launch_cluster_scatter(const DevCtx &c, int req, int layer, const __nv_bfloat16 *k,
                            const __nv_bfloat16 *v, const int64_t *dest_row, int n_tokens,
                            cudaStream_t st);
+int launch_cluster_scatter_staged(const DevCtx &c, const __nv_bfloat16 *k, const __nv_bfloat16 *v, const int32_t *lrow,
+                                  int n_tokens, int p0, int m, uint8_t *stage, cudaStream_t st);
 int launch_stage_in(void *dq, const void *sq, size_t q_bytes, void *dk, const void *sk, void *dv, const void *sv,
                     size_t kv_bytes, cudaStream_t st);
 int launch_copy_centroids(const DevCtx &c, int req, int layer, const __nv_bfloat16 *cen,
@@ -334,6 +336,7 @@ int launch_cache(const DevCtx &c, const Batch &b, cudaStream_t st, Prof *prof);
 int launch_fetch(const DevCtx &c, cudaStream_t st, int sm_count, Prof *prof);
 int launch_shrink(const DevCtx &c, int req, int old_S, int new_S, cudaStream_t st);
 int launch_wait_probe(const DevCtx &c, int max_polls, cudaStream_t st);
+int launch_floor(const DevCtx &c, int token, cudaStream_t st);
 int launch_link_probe(const DevCtx &c, int n_pages, cudaStream_t st, int sm_count);
 int launch_assign(const DevCtx &c, int req, int layer, int n_clusters, int n_tokens, int32_t *assign, cudaStream_t st);
 int launch_move_rows(const DevCtx &c, int req, int layer, const int64_t *dest, int n_tokens, cudaStream_t st);

@@ -37,12 +37,6 @@ def request_budgets(w: W.Workload, cache_pages_per_layer: int) -> List[int]:
     return out
 
 
-def make_spin(w: W.Workload, device="cuda:0", trace: bool = False, sm_scale: float = 0.0,
-              slots_per_set: Optional[int] = None, segment_entries: int = 0,
-              fetch_mode: int = 0, host_tables_only: int = 0) -> "SpinRun":
-    return SpinRun(w, device, trace, sm_scale, slots_per_set, segment_entries, fetch_mode, host_tables_only)
-
-
 class SpinRun:
     """A library context sized for one workload, plus the per-step call sequence."""
 

@@ -17,6 +17,14 @@ def test_c2_llama_shaped_full_size_sampled_request():
     assert r["stats"]["miss_pages"] > 0 and r["stats"]["evicted_pages"] == 0   # 512 slots: still filling
 
 
+def test_c2_llama_shaped_full_size_softmax_scale_one():
+    # the same with sm_scale = 1: logits of the outlier-channel keys are tens of units apart, the
+    # softmax is sharp and outputs are of order one, so the tolerances discriminate
+    w = W.scaled(W.CONFIGS["c2"], steps=6)
+    r = run_parity(w, sm_scale=1.0, one_call=True, check_bytes=False, oracle_reqs=[5])
+    assert r["rel_l2"] < 2e-2 and r["stats"]["miss_pages"] > 0
+
+
 def test_c2_full_size_small_budget_evicts():
     w = W.scaled(W.CONFIGS["c2"], steps=24, slots_per_set=160, lru_buckets=8)
     r = run_parity(w, one_call=True, check_bytes=True, oracle_reqs=[0])
@@ -33,6 +41,12 @@ def test_c4_cluster_granular_full_size_sampled_request():
     w = W.scaled(W.CONFIGS["c4"], steps=8, batch=4)  # 4 of the 16 requests: 131072 tokens, 1024 clusters each
     r = run_parity(w, one_call=True, check_bytes=False, oracle_reqs=[2])
     assert r["stats"]["miss_pages"] > 0
+
+
+def test_c4_cluster_granular_full_size_softmax_scale_one():
+    w = W.scaled(W.CONFIGS["c4"], steps=4, batch=2)
+    r = run_parity(w, sm_scale=1.0, one_call=True, check_bytes=False, oracle_reqs=[1])
+    assert r["rel_l2"] < 2e-2 and r["stats"]["miss_pages"] > 0
 
 
 def test_c5_mixed_batch_scaled_sampled_requests():

@@ -206,10 +206,11 @@ def test_separate_fetch_kernel_mode():
                    steps=20), fetch_mode=1, one_call=True)
 
 
-def test_page_minmax_outlier_keys_gqa4_many_buckets():
+@pytest.mark.parametrize("sm_scale", [0.0, 1.0])
+def test_page_minmax_outlier_keys_gqa4_many_buckets(sm_scale):
     w = _wl(W.PART_PAGE_MINMAX, num_q_heads=8, num_kv_heads=2, kv_recipe="outlier", outlier_channels=4,
             lru_buckets=64, steps=80, topk=8, slots_per_set=24, drift=0.1, context=16 * 70 + 15)
-    run_parity(w, sm_scale=0.0)
+    run_parity(w, sm_scale=sm_scale)
 
 
 def test_page_minmax_step_counter_passes_bucket_count_and_segments_are_crossed():
@@ -341,6 +342,21 @@ def test_asynchronous_offload_of_prefill_pages(kind):
     w = _wl(kind, topk=6 if kind == W.PART_PAGE_MINMAX else 64, steps=12)
     r = run_parity(w, offload_stage_bytes=4 * 3 * 2 * 8192, check_bytes=True)
     assert r["stats"]["miss_pages"] > 0
+
+
+def test_asynchronous_offload_of_a_cluster_prefill():
+    # cluster granularity: the prefill's rows are packed into the clusters' pages in the staging
+    # ring (4 slots x 3 pages x 2 kv heads: ~90 pages per head wrap it many times), with heads
+    # that own different numbers of pages; host bytes, traces and outputs as written through
+    w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=37, topk=5, slots_per_set=30,
+            context=16 * 50 + 3, steps=16, max_partition_pages=8, lru_buckets=8)
+    r = run_parity(w, offload_stage_bytes=4 * 3 * 2 * 8192, check_bytes=True, one_call=True)
+    assert r["stats"]["miss_pages"] > 0
+    # and with Index during decode folding tail pages into clusters whose pages came through the ring
+    w = _wl(W.PART_CLUSTER_CENTROID, kv_recipe="mixture", num_clusters=23, topk=5, slots_per_set=40,
+            context=16 * 30 + 7, steps=44, max_partition_pages=12, lru_buckets=8, batch=2, num_layers=1)
+    r = run_parity(w, offload_stage_bytes=4 * 4 * 2 * 8192, reindex_every=20)
+    assert r["folded"] == 2 * 2 * 32
 
 
 @pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_CLUSTER_CENTROID, W.PART_TOKEN_DOT])
