@@ -182,6 +182,7 @@ struct spin_ctx {
   static constexpr int kOffloadSlots = 4;
   uint8_t *offload_stage = nullptr;
   int32_t *offload_hp = nullptr;     // per staged unit: its host page id (what the kernel records in the mirror)
+  int32_t *offload_lrow = nullptr;   // cluster prefill: row places of one prefill's tokens (see prefill_clustered)
   int64_t offload_slot_units = 0;    // (page, kv head) units of 8 KiB per slot; 0 = write-through
   cudaStream_t offload_stream = nullptr;
   cudaEvent_t ev_staged[kOffloadSlots] = {}, ev_done[kOffloadSlots] = {};
@@ -269,7 +270,10 @@ void carve(Arena &a, const spin_config &cfg, const Geometry &g, DevCtx &d, spin_
     const int64_t units = cfg.offload_stage_bytes / spin_ctx::kOffloadSlots / kPageBytes;
     uint8_t *os = a.take<uint8_t>((size_t)units * spin_ctx::kOffloadSlots * kPageBytes);
     int32_t *oh = a.take<int32_t>((size_t)units * spin_ctx::kOffloadSlots);
-    if (ctx) { ctx->offload_stage = os; ctx->offload_hp = oh; ctx->offload_slot_units = units; }
+    // cluster granularity: where every (token, head) row of a prefill goes in its set's page order
+    int32_t *ol = cfg.partition_kind == SPIN_PART_CLUSTER_CENTROID
+                      ? a.take<int32_t>((size_t)cfg.max_context_tokens * cfg.num_kv_heads) : nullptr;
+    if (ctx) { ctx->offload_stage = os; ctx->offload_hp = oh; ctx->offload_slot_units = units; ctx->offload_lrow = ol; }
   }
 }
 
@@ -643,8 +647,7 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
         const int32_t r = filled[(size_t)h * C + c]++;
         lrow[(size_t)t * H + h] = (first_row_page[(size_t)h * C + c] + r / kPageTokens) * kPageTokens + r % kPageTokens;
       }
-    int32_t *d_lrow = nullptr;
-    CK(cudaMalloc(reinterpret_cast<void **>(&d_lrow), lrow.size() * 4));
+    int32_t *d_lrow = ctx->offload_lrow;                    // this call ends with the stream idle: no earlier prefill still reads it
     CK(cudaMemcpyAsync(d_lrow, lrow.data(), lrow.size() * 4, cudaMemcpyHostToDevice, st));
     const int64_t per = ctx->offload_slot_units / H;
     for (int64_t p0 = 0; p0 < total_pages_max; p0 += per) {
@@ -675,7 +678,6 @@ int prefill_clustered(spin_ctx *ctx, int req, int layer, const void *k, const vo
       ++ctx->offload_gen;
     }
     CK(cudaStreamSynchronize(st));          // the host-side sources of this call's copies end here; the drain goes on
-    CK(cudaFree(d_lrow));
   } else {
   // rows -> host pages, in chunks through the staging buffers
   const int64_t chunk = g.stage_tokens;
