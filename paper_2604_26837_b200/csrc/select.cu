@@ -811,46 +811,51 @@ __device__ __forceinline__ void topk_cta(const DevCtx &c, const Batch &bt, int k
   const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const int b = blockIdx.x / C, i_req = b / c.Hkv, head = b % c.Hkv, tid = threadIdx.x;
   const int set = set_index(c, bt.req[i_req], bt.layer, head);
-  if (wait_flags) {
-    if (rank == 0 && tid == 0) {
-      // 1: the flag the last scoring CTA of the set raises; 2: the streaming kernel's arrival counter
-      const int n_cand = c.kind == kKindToken ? bt.n_partitions[i_req] * kPageTokens : bt.n_partitions[i_req];
-      // (the tail flag first: it says that this step's kernels have the GPU, which a count of zero
-      // stages -- a set without candidates -- does not)
-      s_ok = wait_flags == 2 ? (flag_wait(c, c.tail_ready + b, bt.epoch) && wait_scored(c, b, stream_stages_of(n_cand)))
-                             : flag_wait(c, c.scored + b, bt.epoch);
-    }
-    cluster.sync();
-    const int ok = *cluster.map_shared_rank(&s_ok, 0);
-    cluster.sync();                                   // the first CTA's word is not read after this
-    if (!ok) return;
-  } else {
-    pdl_wait_prev();
-  }
-  if (rank == 0) dbg_ts(b, 9);
-  // the first CTA is also the set's cache manager: its tables start towards shared memory now
-  // (behind the keys' slice) and arrive while the select runs
+  // the first CTA is also the set's cache manager: its tables go to shared memory (behind the
+  // keys' slice) before the set is scored -- they do not depend on this step's scores and are
+  // stable once this step's kernels have the GPU, which the set's tail flag says -- or, without
+  // flags, once the kernel before this one has completed
   const int S = bt.slots[i_req];
   const FastLayout L = fast_layout(c, dyn_smem + (((size_t)keys_cap * 4 + 15) & ~(size_t)15), 0, S, tbl_cap);
   const bool mgr = manage && rank == 0;
-  if (mgr) {
+  if (wait_flags) {
+    if (rank == 0) {
+      if (tid == 0) s_ok = flag_wait(c, c.tail_ready + b, bt.epoch);
+      __syncthreads();
+    }
+  } else {
+    pdl_wait_prev();
+  }
+  if (mgr && (!wait_flags || s_ok)) {
     fast_prefetch_dirs<kTopkThreads>(c, L, set, S);
     asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     __syncthreads();
     fast_prefetch_gpt<kTopkThreads>(c, L, S);
     fast_prefetch_tables<kTopkThreads>(c, L, bt.n_partitions[i_req]);
   }
+  if (wait_flags) {
+    if (rank == 0 && tid == 0 && s_ok) {
+      // 1: the flag the last scoring CTA of the set raises; 2: the streaming kernel's arrival counter
+      const int n_cand = c.kind == kKindToken ? bt.n_partitions[i_req] * kPageTokens : bt.n_partitions[i_req];
+      s_ok = wait_flags == 2 ? wait_scored(c, b, stream_stages_of(n_cand)) : flag_wait(c, c.scored + b, bt.epoch);
+    }
+    cluster.sync();
+    const int ok = *cluster.map_shared_rank(&s_ok, 0);
+    cluster.sync();                                   // the first CTA's word is not read after this
+    if (!ok) return;
+  }
+  if (rank == 0) dbg_ts(b, 9);
   const bool first = topk_stage<kTopkThreads, true>(c, b, bt.n_partitions[i_req], reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh, wait_flags == 2);
   if (!first || !manage) return;
-  const int np = c.n_parts[b];
+  const int np = __ldcg(c.n_parts + b);               // with the row-wise select, written by the cluster's other CTAs
   const int32_t *g_parts = c.parts + (size_t)b * c.max_parts;
-  for (int r = tid; r < np; r += kTopkThreads) L.s_parts[r] = g_parts[r];
+  for (int r = tid; r < np; r += kTopkThreads) L.s_parts[r] = __ldcg(g_parts + r);
   asm volatile("cp.async.wait_group 0;\n" ::: "memory");
   __syncthreads();
   cache_fast<kTopkThreads>(c, bt, b, i_req, set, L, np, shm.f);
 }
 
-__global__ void __launch_bounds__(kTopkThreads)
+__global__ void __launch_bounds__(kTopkThreads, 1)
 k_topk(DevCtx c, Batch bt, int keys_cap, int manage, int tbl_cap, int wait_flags) {
   extern __shared__ __align__(16) uint8_t dyn_smem[];
   pdl_launch_next();
@@ -1040,7 +1045,7 @@ int launch_select(const DevCtx &c, Batch &b, const __nv_bfloat16 *q, const __nv_
     // cluster size from the largest candidate count: slices of at most 8192 keys stay in smem
     int C = 1;
     while (C < 8 && (max_cand + C - 1) / C > 8192) C *= 2;
-    int kc = (max_cand + C - 1) / C;
+    int kc = (((max_cand + C - 1) / C) + 31) & ~31;     // a CTA's slice: whole rows of 32 keys
     if (kc > 16384) kc = 0;                              // too many for shared memory: re-read from L2
     static int smem_set_dev[kMaxDevices] = {};
     int &smem_set = smem_set_dev[current_device_slot()];
@@ -1065,5 +1070,9 @@ extern "C" __attribute__((visibility("default"))) int spin_debug_timestamps_stre
 extern "C" __attribute__((visibility("default"))) int spin_debug_timestamps(unsigned long long *out) {
   cudaDeviceSynchronize();
   return (int)cudaMemcpyFromSymbol(out, spin::g_dbg_ts, sizeof(unsigned long long) * 256 * 32);
+}
+extern "C" __attribute__((visibility("default"))) int spin_debug_cycles(unsigned long long *out) {
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpyFromSymbol(out, spin::g_dbg_ck, sizeof(unsigned long long) * 256 * 32);
 }
 #endif

@@ -10,6 +10,7 @@
 //                  metadata only; the page bytes move in the attention kernel (or k_fetch).
 #pragma once
 #include <cooperative_groups.h>
+#include <cstddef>
 
 #include "spin_dev.cuh"
 
@@ -106,10 +107,17 @@ __device__ __forceinline__ bool resolve_in_manager(const DevCtx &c) { return c.f
 __device__ unsigned long long g_dbg_ts[256][32];
 __device__ __forceinline__ void dbg_ts(int b, int slot) { if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; } }
 __device__ __forceinline__ void dbg_ts_any(int b, int slot) { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); g_dbg_ts[b & 255][slot] = t; }
+// cycle stamps of one CTA (differences within a CTA only)
+__device__ unsigned long long g_dbg_ck[256][32];
+__device__ __forceinline__ void dbg_ck(int b, int slot) { if (threadIdx.x == 0) g_dbg_ck[b & 255][slot] = (unsigned long long)clock64(); }
 #else
 __device__ __forceinline__ void dbg_ts(int, int) {}
 __device__ __forceinline__ void dbg_ts_any(int, int) {}
+__device__ __forceinline__ void dbg_ck(int, int) {}
 #endif
+
+constexpr int kWideBits = 11, kWideBins = 1 << kWideBits;   // digit of the row-wise cluster select
+constexpr int kGatherMax = 256;                             // a threshold bin this small is ranked directly
 
 struct TopkShared {
   uint32_t hist[256];          // this CTA's histogram (read remotely inside a cluster)
@@ -118,10 +126,293 @@ struct TopkShared {
   uint32_t cnt[2];             // this CTA's (above threshold, equal) counts
   uint32_t prefix, remaining;
   uint32_t orand[2];           // OR and AND of this CTA's keys (read remotely inside a cluster)
+  // row-wise select (topk_cluster_rows)
+  alignas(16) uint32_t whist[2][kWideBins];    // this CTA's wide-digit histograms, alternating between passes (read
+                                               //   remotely, four bins at a time: 16-byte aligned)
+  uint32_t cand[kGatherMax];       // this CTA's keys of the threshold bin (read remotely)
+  uint32_t gath[kGatherMax];       // the threshold bin's keys of all CTAs
+  uint32_t ncand, bin_count;
+  uint32_t result[2];              // threshold key and how many keys equal to it are taken
+  uint32_t wcnt[32], wpg[32];      // per-warp (above | equal << 16) counts and page counts
+  uint32_t rcnt[8], rpages[8];     // the same per CTA of the cluster (written by their owners)
 };
+
+static_assert(offsetof(TopkShared, whist) % 16 == 0 && sizeof(uint32_t[kWideBins]) % 16 == 0, "uint4 reads of the histograms");
 
 template <bool CLUSTER> __device__ __forceinline__ void stage_sync() {
   if constexpr (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
+}
+
+// Radix select of one set by a thread-block cluster.  A CTA owns a slice of `per` consecutive
+// candidates (a multiple of 32) whose keys it holds in shared memory; a warp owns R x 32
+// consecutive candidates of it as R rows of 32 (lane l: candidate 32 j + l of the warp's run).
+// Loads are coalesced, a row's ballot is the order of its 32 candidates (for token granularity
+// also the masks of the row's two pages), so that the ordered compaction needs no scan over
+// candidates and no second look at memory.
+// Every pass over the keys is a ROLLED loop over rows: this code runs once per launch with cold
+// instruction caches, where a straight-line instruction costs tens of cycles of fetch, so the
+// number of distinct instructions on the path matters more than the work per key.
+// Digits are the key's bits 31..21, 20..10 and 10..0.  A CTA's histogram is read by all CTAs of
+// the cluster through distributed shared memory (each finds the threshold bin itself: no
+// broadcast, one cluster barrier per pass, the histograms alternating between two buffers); a
+// threshold bin of at most 256 keys is gathered by every CTA from all CTAs and ranked directly.
+// Counts that other CTAs need are pushed into their shared memory before a barrier, so nothing
+// is read remotely after the last one.  Cluster barriers are hardware barriers and every CTA
+// executes the same sequence of them (every decision is taken on set-wide values).
+// Leaves the chosen candidates, ascending, in c.sel_ids and the partitions of the cache manager
+// in c.parts / c.part_mask / c.n_parts; the caller's closing cluster barrier publishes them.
+// Needs per <= 1024 T (a warp's rows are numbered by its lanes) and per keys of shared memory.
+template <int T>
+__device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n, int k, int per, uint32_t *s_keys,
+                                                  TopkShared &sh, bool xfer) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lt = (1u << lane) - 1u;
+  constexpr int W = T / 32;
+  float *scores = c.scores + (size_t)b * c.max_cand;
+  int32_t *sel = c.sel_ids + (size_t)b * c.max_sel;
+  int32_t *parts = c.parts + (size_t)b * c.max_parts;
+  const bool token = c.kind == kKindToken;
+  const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
+  const int R = (per / 32 + W - 1) / W;                                // rows of a warp (at most 32)
+  const int wbase = warp * R * 32;                                     // the warp's run starts here in the slice
+  const int nvr = max(0, min(R, (m - wbase - lane + 31) >> 5));        // rows j < nvr hold a candidate of this lane
+  uint32_t *mykeys = s_keys + wbase + lane;                            // row j: mykeys[32 j]
+  if (rank == 0) dbg_ck(b, 0);
+  if (xfer) {
+    float *xfer_in = c.score_xfer + (size_t)b * c.max_cand + lo + wbase + lane;
+#pragma unroll 1
+    for (int j = 0; j < nvr; ++j) {
+      const float sc = take_score(c, xfer_in + 32 * j);
+      scores[lo + wbase + lane + 32 * j] = sc;
+      mykeys[32 * j] = order_key(sc);
+    }
+  } else {
+    // asynchronous copies: all rows in flight at once from a two-instruction loop
+    const float *src = scores + lo + wbase + lane;
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(mykeys);
+#pragma unroll 1
+    for (int j = 0; j < nvr; ++j)
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(dst + 128u * j), "l"(src + 32 * j) : "memory");
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+  }
+#pragma unroll 1
+  for (int i = tid; i < 2 * kWideBins; i += T) (&sh.whist[0][0])[i] = 0;
+  if (tid == 0) {
+    sh.ncand = 0;
+    if (rank == 0) {
+      c.n_sel[b] = k;
+      atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
+    }
+  }
+  if (!xfer) {
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+#pragma unroll 1
+    for (int j = 0; j < nvr; ++j) mykeys[32 * j] = order_key(__uint_as_float(mykeys[32 * j]));   // a thread's own words
+  }
+  __syncthreads();
+  if (rank == 0) { dbg_ts(b, 10); dbg_ck(b, 1); }
+  uint32_t thr = 0, need_eq = (uint32_t)k;
+  {
+    uint32_t mask = 0, prefix = 0, remaining = (uint32_t)k;              // decided bits and their value
+    int buf = 0;
+    constexpr int kPer = kWideBins / T;                                // bins per thread
+    constexpr uint32_t dmask = kWideBins - 1;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;           // the last digit repeats bit 10 (decided: harmless)
+      uint32_t *hist = sh.whist[buf];
+      if (pass == 2) {
+        // this buffer served two passes ago; every CTA has read it since (the barrier of the pass between)
+#pragma unroll 1
+        for (int i = tid; i < kWideBins; i += T) hist[i] = 0;
+        __syncthreads();
+      }
+#pragma unroll 1
+      for (int j = 0; j < nvr; ++j) {
+        const uint32_t key = mykeys[32 * j];
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+      }
+      if (rank == 0) dbg_ck(b, 2 + 6 * pass);
+      cluster.sync();                                                  // every CTA's histogram of this pass is complete
+      if (rank == 0) { dbg_ts(b, 11 + pass); dbg_ck(b, 3 + 6 * pass); }
+      // this thread's kPer bins over the whole set, best first: one 16-byte read per CTA of the
+      // cluster, all of them issued before the first is used (a CTA beyond the cluster's size
+      // stands for the last one and counts for nothing)
+      uint32_t loc[kPer], sum = 0;
+      static_assert(kPer == 4, "a thread reads its bins of one CTA as one uint4");
+      {
+        uint4 part[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r)
+          part[r] = *reinterpret_cast<const uint4 *>(cluster.map_shared_rank(hist, min(r, C - 1)) + (kWideBins - kPer * (tid + 1)));
+        uint4 acc = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int r = 0; r < 8; ++r)
+          if (r < C) { acc.x += part[r].x; acc.y += part[r].y; acc.z += part[r].z; acc.w += part[r].w; }
+        loc[0] = acc.w; loc[1] = acc.z; loc[2] = acc.y; loc[3] = acc.x;          // bins in descending order
+        sum = acc.x + acc.y + acc.z + acc.w;
+      }
+      if (rank == 0) dbg_ck(b, 4 + 6 * pass);
+      uint32_t tot_all;
+      const uint32_t before = block_scan1<T>(sum, sh.wsum + (pass & 1) * 16, &tot_all);
+      if (rank == 0) dbg_ck(b, 5 + 6 * pass);
+      if (before < remaining && before + sum >= remaining) {
+        uint32_t cum = before;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+          if (cum < remaining && cum + loc[j] >= remaining) {
+            sh.prefix = (prefix & ~(dmask << shift)) | ((uint32_t)(kWideBins - 1 - kPer * tid - j) << shift);
+            sh.remaining = remaining - cum;
+            sh.bin_count = loc[j];
+          }
+          cum += loc[j];
+        }
+      }
+      __syncthreads();
+      prefix = sh.prefix;
+      remaining = sh.remaining;
+      const uint32_t bin_count = sh.bin_count;
+      mask |= dmask << shift;
+      __syncthreads();                                                 // sh.prefix etc. are rewritten by the next pass
+      if (rank == 0) dbg_ck(b, 6 + 6 * pass);
+      if (shift == 0) break;                                           // the key is decided to its last bit
+      if (bin_count <= (uint32_t)kGatherMax) {
+        // the bin's keys of this CTA, then those of all CTAs, ranked by one thread per key
+#pragma unroll 1
+        for (int j = 0; j < nvr; ++j) {
+          const uint32_t key = mykeys[32 * j];
+          if ((key & mask) == prefix) sh.cand[atomicAdd(&sh.ncand, 1u) & (kGatherMax - 1)] = key;
+        }
+        if (rank == 0) dbg_ck(b, 20);
+        cluster.sync();
+        if (rank == 0) dbg_ck(b, 21);
+        if (tid < kGatherMax) {
+          uint32_t cnt[8], val[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) cnt[r] = *cluster.map_shared_rank(&sh.ncand, min(r, C - 1));
+#pragma unroll
+          for (int r = 0; r < 8; ++r) {
+            val[r] = 0;
+            if (r < C && tid < (int)cnt[r]) val[r] = cluster.map_shared_rank(sh.cand, r)[tid];
+          }
+          uint32_t off = 0;
+#pragma unroll
+          for (int r = 0; r < 8; ++r)
+            if (r < C) {
+              if (tid < (int)cnt[r]) sh.gath[(off + tid) & (kGatherMax - 1)] = val[r];
+              off += cnt[r];
+            }
+        }
+        __syncthreads();
+        if (rank == 0) dbg_ck(b, 22);
+        if (tid < (int)bin_count) {
+          const uint32_t mine = sh.gath[tid];
+          uint32_t gt = 0, ge = 0;
+#pragma unroll 1
+          for (uint32_t j = 0; j < bin_count; ++j) { const uint32_t o = sh.gath[j]; gt += o > mine; ge += o >= mine; }
+          if (gt < remaining && ge >= remaining) { sh.result[0] = mine; sh.result[1] = remaining - gt; }
+        }
+        __syncthreads();
+        if (rank == 0) dbg_ck(b, 23);
+        prefix = sh.result[0];
+        remaining = sh.result[1];
+        break;
+      }
+      buf ^= 1;
+    }
+    thr = prefix;
+    need_eq = remaining;
+  }
+  if (rank == 0) dbg_ts(b, 15);
+  // ---- ordered compaction: everything above thr, plus the first need_eq keys equal to it ----
+  // counts of this warp (row ballots), of the warps before it, of the CTAs before this one
+  uint32_t wgt = 0, weq = 0;
+#pragma unroll 1
+  for (int j = 0; j < R; ++j) {
+    const uint32_t key = j < nvr ? mykeys[32 * j] : 0u;
+    wgt += __popc(__ballot_sync(0xffffffffu, j < nvr && key > thr));
+    weq += __popc(__ballot_sync(0xffffffffu, j < nvr && key == thr));
+  }
+  if (lane == 0) sh.wcnt[warp] = wgt | (weq << 16);                    // a slice holds fewer than 65536 candidates
+  __syncthreads();
+  uint32_t gt_base = 0, eq_base = 0;
+  {
+    uint32_t before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+      const uint32_t v = sh.wcnt[w];
+      before += w < warp ? v : 0u;
+      total += v;
+    }
+    if (tid < C) cluster.map_shared_rank(sh.rcnt, tid)[rank] = total;  // pushed: read locally after the barrier
+    if (rank == 0) dbg_ck(b, 24);
+    cluster.sync();
+    if (rank == 0) dbg_ck(b, 25);
+    gt_base = before & 0xffffu;
+    eq_base = before >> 16;
+    for (int r = 0; r < rank; ++r) { const uint32_t v = sh.rcnt[r]; gt_base += v & 0xffffu; eq_base += v >> 16; }
+  }
+  uint32_t row_taken = 0;                                              // lane l: which candidates of row l were chosen
+  int32_t *dst2 = token ? sel : parts;                                 // without tokens the partitions are the selection
+#pragma unroll 1
+  for (int j = 0; j < R; ++j) {
+    const uint32_t key = j < nvr ? mykeys[32 * j] : 0u;
+    const bool g = j < nvr && key > thr, e = j < nvr && key == thr;
+    const uint32_t bg = __ballot_sync(0xffffffffu, g), be = __ballot_sync(0xffffffffu, e);
+    const uint32_t eq_b = eq_base + __popc(be & lt);
+    const bool take = g || (e && eq_b < need_eq);
+    if (take) {
+      const uint32_t pos = gt_base + __popc(bg & lt) + min(eq_b, need_eq);
+      const int id = lo + wbase + 32 * j + lane;
+      sel[pos] = id;
+      dst2[pos] = id;
+    }
+    const uint32_t bt = __ballot_sync(0xffffffffu, take);
+    if (lane == j) row_taken = bt;
+    gt_base += __popc(bg);
+    eq_base += __popc(be);
+  }
+  if (rank == 0) dbg_ck(b, 26);
+  if (!token) {
+    if (rank == 0 && tid == 0) c.n_parts[b] = k;
+    return;
+  }
+  // ---- chosen tokens -> their pages (ascending, unique) and a 16-bit token mask per page.
+  // A row is two pages: lane l numbers the pages of row l.
+  uint32_t *pmask = c.part_mask + (size_t)b * c.max_parts;
+  const uint32_t m_lo = row_taken & 0xffffu, m_hi = row_taken >> 16;
+  const uint32_t mine = (m_lo != 0) + (m_hi != 0);
+  uint32_t inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) sh.wpg[warp] = inc;
+  __syncthreads();
+  uint32_t pg_base = 0, pg_total = 0;
+#pragma unroll
+  for (int w = 0; w < W; ++w) {
+    const uint32_t v = sh.wpg[w];
+    pg_base += w < warp ? v : 0u;
+    pg_total += v;
+  }
+  if (tid < C) cluster.map_shared_rank(sh.rpages, tid)[rank] = pg_total;
+  if (rank == 0) dbg_ck(b, 27);
+  cluster.sync();
+  if (rank == 0) dbg_ck(b, 28);
+  uint32_t cta_base = 0;
+  for (int r = 0; r < rank; ++r) cta_base += sh.rpages[r];
+  if (mine) {
+    uint32_t at = cta_base + pg_base + inc - mine;
+    const int page = (lo + wbase + 32 * lane) >> 4;
+    if (m_lo) { parts[at] = page; pmask[at] = m_lo; ++at; }
+    if (m_hi) { parts[at] = page + 1; pmask[at] = m_hi; }
+  }
+  if (rank == C - 1 && tid == 0) c.n_parts[b] = (int)(cta_base + pg_total);
+  if (rank == 0) dbg_ck(b, 29);
 }
 
 // Top-k of one set.  With CLUSTER the set's candidates are cut into one contiguous slice per
@@ -151,6 +442,17 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
   const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
   const bool cached = m <= keys_cap;
 
+  bool selected = false;
+  if constexpr (CLUSTER) {
+    // slices that fit in shared memory, at most 32 rows per warp: the row-wise select
+    const int per32 = (per + 31) & ~31;
+    if (k < n && per32 <= 32 * T && per32 <= keys_cap) {
+      if (rank == 0) dbg_ts(b, 25);
+      topk_cluster_rows<T>(c, b, n, k, per32, s_keys, sh, xfer);
+      selected = true;
+    }
+  }
+  if (!selected) {
   if (tid == 0 && rank == 0) {
     c.n_sel[b] = k;
     atomicAdd(&c.counters->candidates_scored, (unsigned long long)n);
@@ -160,14 +462,22 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
   // keys -> shared memory, with the OR and AND of the slice taken on the way
   {
     uint32_t k_or = 0, k_and = 0xffffffffu;
+    if (xfer) {
+#pragma unroll 4
+      for (int i = tid; i < m; i += T) {
+        const float sc = take_score(c, xfer_in + lo + i);
+        scores[lo + i] = sc;
+        const uint32_t key = order_key(sc);
+        if (cached) s_keys[i] = key;
+        k_or |= key; k_and &= key;
+      }
+    } else {
 #pragma unroll 8
-    for (int i = tid; i < m; i += T) {
-      float sc;
-      if (xfer) { sc = take_score(c, xfer_in + lo + i); scores[lo + i] = sc; }
-      else sc = __ldcg(scores + lo + i);
-      const uint32_t key = order_key(sc);
-      if (cached) s_keys[i] = key;
-      k_or |= key; k_and &= key;
+      for (int i = tid; i < m; i += T) {
+        const uint32_t key = order_key(__ldcg(scores + lo + i));
+        if (cached) s_keys[i] = key;
+        k_or |= key; k_and &= key;
+      }
     }
     k_or = __reduce_or_sync(0xffffffffu, k_or);
     k_and = __reduce_and_sync(0xffffffffu, k_and);
@@ -312,10 +622,12 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
       }
     }
   }
+  }
   if (rank == 0) dbg_ts(b, 27);
   stage_sync<CLUSTER>();     // selections of all slices are written; no remote smem is read after this
   if (rank != 0) return false;
   dbg_ts(b, 28);
+  if (selected) { dbg_ts(b, 29); return true; }      // the row-wise select wrote the partitions itself
 
   // ---- candidates -> partitions of the cache manager (first CTA of the cluster) ----------
   int32_t *parts = c.parts + (size_t)b * c.max_parts;
