@@ -804,7 +804,7 @@ k_select(DevCtx c, Batch bt, int keys_cap, int tbl_cap) {
 // cluster take the same path through the cluster barriers.
 __device__ __forceinline__ void topk_cta(const DevCtx &c, const Batch &bt, int keys_cap, int manage, int tbl_cap,
                                          int wait_flags, uint8_t *dyn_smem) {
-  __shared__ union { TopkShared t; FastShared f; } shm;
+  __shared__ union { TopkShared t; FastShared f; TopkRowsShared r; } shm;   // r instead of t when the row-wise select runs
   __shared__ int s_ok;
   TopkShared &tsh = shm.t;
   cg::cluster_group cluster = cg::this_cluster();
@@ -845,7 +845,7 @@ __device__ __forceinline__ void topk_cta(const DevCtx &c, const Batch &bt, int k
     if (!ok) return;
   }
   if (rank == 0) dbg_ts(b, 9);
-  const bool first = topk_stage<kTopkThreads, true>(c, b, bt.n_partitions[i_req], reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh, wait_flags == 2);
+  const bool first = topk_stage<kTopkThreads, true>(c, b, bt.n_partitions[i_req], reinterpret_cast<uint32_t *>(dyn_smem), keys_cap, tsh, wait_flags == 2, &shm.r);
   if (!first || !manage) return;
   const int np = __ldcg(c.n_parts + b);               // with the row-wise select, written by the cluster's other CTAs
   const int32_t *g_parts = c.parts + (size_t)b * c.max_parts;

@@ -126,7 +126,10 @@ struct TopkShared {
   uint32_t cnt[2];             // this CTA's (above threshold, equal) counts
   uint32_t prefix, remaining;
   uint32_t orand[2];           // OR and AND of this CTA's keys (read remotely inside a cluster)
-  // row-wise select (topk_cluster_rows)
+};
+
+// Shared memory of the row-wise cluster select (topk_cluster_rows); only the cluster kernel holds it.
+struct TopkRowsShared {
   alignas(16) uint32_t whist[2][kWideBins];    // this CTA's wide-digit histograms, alternating between passes (read
                                                //   remotely, four bins at a time: 16-byte aligned)
   uint32_t cand[kGatherMax];       // this CTA's keys of the threshold bin (read remotely)
@@ -135,9 +138,11 @@ struct TopkShared {
   uint32_t result[2];              // threshold key and how many keys equal to it are taken
   uint32_t wcnt[32], wpg[32];      // per-warp (above | equal << 16) counts and page counts
   uint32_t rcnt[8], rpages[8];     // the same per CTA of the cluster (written by their owners)
+  uint32_t wsum[33];
+  uint32_t prefix, remaining;
 };
 
-static_assert(offsetof(TopkShared, whist) % 16 == 0 && sizeof(uint32_t[kWideBins]) % 16 == 0, "uint4 reads of the histograms");
+static_assert(offsetof(TopkRowsShared, whist) % 16 == 0 && sizeof(uint32_t[kWideBins]) % 16 == 0, "uint4 reads of the histograms");
 
 template <bool CLUSTER> __device__ __forceinline__ void stage_sync() {
   if constexpr (CLUSTER) cg::this_cluster().sync(); else __syncthreads();
@@ -161,10 +166,10 @@ template <bool CLUSTER> __device__ __forceinline__ void stage_sync() {
 // executes the same sequence of them (every decision is taken on set-wide values).
 // Leaves the chosen candidates, ascending, in c.sel_ids and the partitions of the cache manager
 // in c.parts / c.part_mask / c.n_parts; the caller's closing cluster barrier publishes them.
-// Needs per <= 1024 T (a warp's rows are numbered by its lanes) and per keys of shared memory.
+// Needs per <= 2048 T (a warp's rows are numbered by its lanes, two rows each) and per keys of shared memory.
 template <int T>
 __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n, int k, int per, uint32_t *s_keys,
-                                                  TopkShared &sh, bool xfer) {
+                                                  TopkRowsShared &sh, bool xfer) {
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -175,7 +180,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
   int32_t *parts = c.parts + (size_t)b * c.max_parts;
   const bool token = c.kind == kKindToken;
   const int lo = min(n, rank * per), m = min(n, lo + per) - lo;
-  const int R = (per / 32 + W - 1) / W;                                // rows of a warp (at most 32)
+  const int R = (per / 32 + W - 1) / W;                                // rows of a warp (at most 64)
   const int wbase = warp * R * 32;                                     // the warp's run starts here in the slice
   const int nvr = max(0, min(R, (m - wbase - lane + 31) >> 5));        // rows j < nvr hold a candidate of this lane
   uint32_t *mykeys = s_keys + wbase + lane;                            // row j: mykeys[32 j]
@@ -237,22 +242,27 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
       if (rank == 0) dbg_ck(b, 2 + 6 * pass);
       cluster.sync();                                                  // every CTA's histogram of this pass is complete
       if (rank == 0) { dbg_ts(b, 11 + pass); dbg_ck(b, 3 + 6 * pass); }
-      // this thread's kPer bins over the whole set, best first: one 16-byte read per CTA of the
-      // cluster, all of them issued before the first is used (a CTA beyond the cluster's size
-      // stands for the last one and counts for nothing)
+      // this thread's kPer bins over the whole set, best first: 16-byte reads, one batch of the
+      // cluster's CTAs at a time, all reads of a batch issued before the first is used (a CTA
+      // beyond the cluster's size stands for the last one and counts for nothing)
       uint32_t loc[kPer], sum = 0;
-      static_assert(kPer == 4, "a thread reads its bins of one CTA as one uint4");
+      static_assert(kPer % 4 == 0 && kPer <= 8, "a thread reads its bins of one CTA as one or two uint4");
       {
-        uint4 part[8];
+        uint32_t bins[kPer];                                           // ascending
 #pragma unroll
-        for (int r = 0; r < 8; ++r)
-          part[r] = *reinterpret_cast<const uint4 *>(cluster.map_shared_rank(hist, min(r, C - 1)) + (kWideBins - kPer * (tid + 1)));
-        uint4 acc = make_uint4(0, 0, 0, 0);
+        for (int q = 0; q < kPer / 4; ++q) {
+          uint4 part[8];
 #pragma unroll
-        for (int r = 0; r < 8; ++r)
-          if (r < C) { acc.x += part[r].x; acc.y += part[r].y; acc.z += part[r].z; acc.w += part[r].w; }
-        loc[0] = acc.w; loc[1] = acc.z; loc[2] = acc.y; loc[3] = acc.x;          // bins in descending order
-        sum = acc.x + acc.y + acc.z + acc.w;
+          for (int r = 0; r < 8; ++r)
+            part[r] = *reinterpret_cast<const uint4 *>(cluster.map_shared_rank(hist, min(r, C - 1)) + (kWideBins - kPer * (tid + 1)) + 4 * q);
+          uint4 acc = make_uint4(0, 0, 0, 0);
+#pragma unroll
+          for (int r = 0; r < 8; ++r)
+            if (r < C) { acc.x += part[r].x; acc.y += part[r].y; acc.z += part[r].z; acc.w += part[r].w; }
+          bins[4 * q] = acc.x; bins[4 * q + 1] = acc.y; bins[4 * q + 2] = acc.z; bins[4 * q + 3] = acc.w;
+        }
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) { loc[j] = bins[kPer - 1 - j]; sum += loc[j]; }
       }
       if (rank == 0) dbg_ck(b, 4 + 6 * pass);
       uint32_t tot_all;
@@ -354,7 +364,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
     eq_base = before >> 16;
     for (int r = 0; r < rank; ++r) { const uint32_t v = sh.rcnt[r]; gt_base += v & 0xffffu; eq_base += v >> 16; }
   }
-  uint32_t row_taken = 0;                                              // lane l: which candidates of row l were chosen
+  uint32_t row_taken[2] = {0, 0};                                      // lane l: which candidates of rows l and 32 + l were chosen
   int32_t *dst2 = token ? sel : parts;                                 // without tokens the partitions are the selection
 #pragma unroll 1
   for (int j = 0; j < R; ++j) {
@@ -370,7 +380,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
       dst2[pos] = id;
     }
     const uint32_t bt = __ballot_sync(0xffffffffu, take);
-    if (lane == j) row_taken = bt;
+    if (lane == (j & 31)) { if (j < 32) row_taken[0] = bt; else row_taken[1] = bt; }
     gt_base += __popc(bg);
     eq_base += __popc(be);
   }
@@ -380,17 +390,21 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
     return;
   }
   // ---- chosen tokens -> their pages (ascending, unique) and a 16-bit token mask per page.
-  // A row is two pages: lane l numbers the pages of row l.
+  // A row is two pages: lane l numbers the pages of rows l and 32 + l.
   uint32_t *pmask = c.part_mask + (size_t)b * c.max_parts;
-  const uint32_t m_lo = row_taken & 0xffffu, m_hi = row_taken >> 16;
-  const uint32_t mine = (m_lo != 0) + (m_hi != 0);
-  uint32_t inc = mine;
+  uint32_t mine[2], inc[2], half_total[2];
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
+  for (int h = 0; h < 2; ++h) {
+    mine[h] = ((row_taken[h] & 0xffffu) != 0) + ((row_taken[h] >> 16) != 0);
+    inc[h] = mine[h];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, inc[h], o);
+      if (lane >= o) inc[h] += t;
+    }
+    half_total[h] = __shfl_sync(0xffffffffu, inc[h], 31);
   }
-  if (lane == 31) sh.wpg[warp] = inc;
+  if (lane == 0) sh.wpg[warp] = half_total[0] + half_total[1];
   __syncthreads();
   uint32_t pg_base = 0, pg_total = 0;
 #pragma unroll
@@ -405,12 +419,15 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
   if (rank == 0) dbg_ck(b, 28);
   uint32_t cta_base = 0;
   for (int r = 0; r < rank; ++r) cta_base += sh.rpages[r];
-  if (mine) {
-    uint32_t at = cta_base + pg_base + inc - mine;
-    const int page = (lo + wbase + 32 * lane) >> 4;
-    if (m_lo) { parts[at] = page; pmask[at] = m_lo; ++at; }
-    if (m_hi) { parts[at] = page + 1; pmask[at] = m_hi; }
-  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+    if (mine[h]) {
+      uint32_t at = cta_base + pg_base + (h ? half_total[0] : 0u) + inc[h] - mine[h];
+      const int page = (lo + wbase + 32 * (lane + 32 * h)) >> 4;
+      const uint32_t m_lo = row_taken[h] & 0xffffu, m_hi = row_taken[h] >> 16;
+      if (m_lo) { parts[at] = page; pmask[at] = m_lo; ++at; }
+      if (m_hi) { parts[at] = page + 1; pmask[at] = m_hi; }
+    }
   if (rank == C - 1 && tid == 0) c.n_parts[b] = (int)(cta_base + pg_total);
   if (rank == 0) dbg_ck(b, 29);
 }
@@ -425,7 +442,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
 // xfer: the scores come from the streaming kernel's hand-over buffer (taken out into c.scores on the way)
 template <int T, bool CLUSTER>
 __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partitions, uint32_t *s_keys,
-                                           int keys_cap, TopkShared &sh, bool xfer = false) {
+                                           int keys_cap, TopkShared &sh, bool xfer = false, TopkRowsShared *rows = nullptr) {
   int C = 1, rank = 0;
   if constexpr (CLUSTER) {
     cg::cluster_group cluster = cg::this_cluster();
@@ -444,11 +461,11 @@ __device__ __forceinline__ bool topk_stage(const DevCtx &c, int b, int n_partiti
 
   bool selected = false;
   if constexpr (CLUSTER) {
-    // slices that fit in shared memory, at most 32 rows per warp: the row-wise select
+    // slices that fit in shared memory, at most 64 rows per warp: the row-wise select
     const int per32 = (per + 31) & ~31;
-    if (k < n && per32 <= 32 * T && per32 <= keys_cap) {
+    if (rows != nullptr && k < n && per32 <= 64 * T && per32 <= keys_cap) {
       if (rank == 0) dbg_ts(b, 25);
-      topk_cluster_rows<T>(c, b, n, k, per32, s_keys, sh, xfer);
+      topk_cluster_rows<T>(c, b, n, k, per32, s_keys, *rows, xfer);
       selected = true;
     }
   }
