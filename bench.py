@@ -481,6 +481,37 @@ def oracle_all_cores(base_name, kw, budget_s, steps_cap):
                        f"rate = requests over the slowest process's mean step time", wall_s=round(wall, 1))
 
 
+def parse_cpulist(text):
+    """'0-3,8,10-11' -> [0, 1, 2, 3, 8, 10, 11]"""
+    cpus = []
+    for part in text.strip().split(","):
+        if not part:
+            continue
+        lo, _, hi = part.partition("-")
+        cpus.extend(range(int(lo), int(hi or lo) + 1))
+    return cpus
+
+
+def bind_near_gpu(props, sysfs="/sys/bus/pci/devices"):
+    """Pin this process to the CPUs local to its GPU (the PCI device's local_cpulist), so that the
+    pinned host tier it allocates next is first touched, and hence placed, on the GPU's NUMA node:
+    with several replicas each pulling tens of GB/s over its own link, host-memory placement
+    decides the scaling curve.  A no-op where the file is missing or lists every CPU (a
+    single-node host).  Returns what it did, for the JSON line."""
+    try:
+        bus = "%04x:%02x:%02x.0" % (props.pci_domain_id, props.pci_bus_id, props.pci_device_id)
+        with open(os.path.join(sysfs, bus, "local_cpulist")) as f:
+            local = set(parse_cpulist(f.read()))
+        allowed = os.sched_getaffinity(0)
+        target = local & allowed
+        if not target or target == allowed:
+            return dict(bound=False, local_cpus=len(local), why="single node or no locality information")
+        os.sched_setaffinity(0, target)
+        return dict(bound=True, local_cpus=len(target))
+    except (OSError, AttributeError, ValueError) as e:
+        return dict(bound=False, why=type(e).__name__)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -547,6 +578,7 @@ def main():
 
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
+    numa = bind_near_gpu(torch.cuda.get_device_properties(device))     # before any pinned allocation
     K, Wm = args.steps, args.warmup
     peaks = load_peaks()
     link_peak = measure_pcie_gbs(torch, device, torch.cuda.Stream(device))
@@ -583,7 +615,7 @@ def main():
                     l2="flushed between timed steps (256 MiB written then read back, untimed)",
                     note="single-layer config: tokens/s is per-layer-step throughput"),
         p50_tpot_ms=head["p50_tpot_ms"], ms_per_step_noflush=head["ms_per_step_noflush"],
-        gpu_launches=head["gpu_launches"], clocks=clocks, step_roofline=head["step_roofline"],
+        gpu_launches=head["gpu_launches"], clocks=clocks, numa=numa, step_roofline=head["step_roofline"],
         roofline=head["roofline"], kernels=head["kernels"], miss_ratio=head["miss_ratio"],
         evicted_pages_per_step=head["evicted_pages_per_step"], missed_pages_per_step=head["missed_pages_per_step"],
         latency_floor=head["latency_floor"], error_bits=head["error_bits"])

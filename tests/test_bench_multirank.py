@@ -43,3 +43,30 @@ def test_single_process_is_identity():
     import bench
     assert bench.allreduce_max([1.5, 2.5]) == [1.5, 2.5]
     assert bench.aggregate_value(100, 1, 1000.0) == 100.0
+
+
+def test_cpu_list_parsing_and_binding_is_a_no_op_without_locality(tmp_path):
+    """The NUMA helper: cpulist syntax; a device whose local CPUs are all of the allowed ones (a
+    single-node host) or whose sysfs entry is missing leaves the affinity alone."""
+    import os
+    import types
+    import bench
+    assert bench.parse_cpulist("0-3,8,10-11\n") == [0, 1, 2, 3, 8, 10, 11]
+    assert bench.parse_cpulist("5") == [5]
+    before = os.sched_getaffinity(0)
+    props = types.SimpleNamespace(pci_domain_id=0, pci_bus_id=0x1b, pci_device_id=0)
+    r = bench.bind_near_gpu(props, sysfs=str(tmp_path))                      # no such device
+    assert r["bound"] is False and os.sched_getaffinity(0) == before
+    d = tmp_path / "0000:1b:00.0"
+    d.mkdir()
+    (d / "local_cpulist").write_text(",".join(str(c) for c in sorted(before)) + "\n")
+    r = bench.bind_near_gpu(props, sysfs=str(tmp_path))                      # every allowed CPU is local
+    assert r["bound"] is False and os.sched_getaffinity(0) == before
+    if len(before) > 1:
+        keep = sorted(before)[:1]
+        (d / "local_cpulist").write_text(str(keep[0]) + "\n")
+        try:
+            r = bench.bind_near_gpu(props, sysfs=str(tmp_path))
+            assert r == {"bound": True, "local_cpus": 1} and os.sched_getaffinity(0) == set(keep)
+        finally:
+            os.sched_setaffinity(0, before)
