@@ -116,6 +116,10 @@ __device__ __forceinline__ void dbg_ts_any(int, int) {}
 __device__ __forceinline__ void dbg_ck(int, int) {}
 #endif
 
+// The row loops of the cluster select, unrolled just enough for the shared-memory reads of
+// consecutive rows to overlap (1 -> 4: 19.3 -> 16.6 us for 65552 keys; fully unrolled the
+// code's first-time instruction fetch costs more than the loops save).
+constexpr int kRowUnroll = 4;
 constexpr int kWideBits = 11, kWideBins = 1 << kWideBits;   // digit of the row-wise cluster select
 constexpr int kGatherMax = 256;                             // a threshold bin this small is ranked directly
 
@@ -213,7 +217,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
   }
   if (!xfer) {
     asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-#pragma unroll 1
+#pragma unroll kRowUnroll
     for (int j = 0; j < nvr; ++j) mykeys[32 * j] = order_key(__uint_as_float(mykeys[32 * j]));   // a thread's own words
   }
   __syncthreads();
@@ -234,7 +238,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
         for (int i = tid; i < kWideBins; i += T) hist[i] = 0;
         __syncthreads();
       }
-#pragma unroll 1
+#pragma unroll kRowUnroll
       for (int j = 0; j < nvr; ++j) {
         const uint32_t key = mykeys[32 * j];
         if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
@@ -290,7 +294,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
       if (shift == 0) break;                                           // the key is decided to its last bit
       if (bin_count <= (uint32_t)kGatherMax) {
         // the bin's keys of this CTA, then those of all CTAs, ranked by one thread per key
-#pragma unroll 1
+#pragma unroll kRowUnroll
         for (int j = 0; j < nvr; ++j) {
           const uint32_t key = mykeys[32 * j];
           if ((key & mask) == prefix) sh.cand[atomicAdd(&sh.ncand, 1u) & (kGatherMax - 1)] = key;
@@ -339,7 +343,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
   // ---- ordered compaction: everything above thr, plus the first need_eq keys equal to it ----
   // counts of this warp (row ballots), of the warps before it, of the CTAs before this one
   uint32_t wgt = 0, weq = 0;
-#pragma unroll 1
+#pragma unroll kRowUnroll
   for (int j = 0; j < R; ++j) {
     const uint32_t key = j < nvr ? mykeys[32 * j] : 0u;
     wgt += __popc(__ballot_sync(0xffffffffu, j < nvr && key > thr));
@@ -366,7 +370,7 @@ __device__ __forceinline__ void topk_cluster_rows(const DevCtx &c, int b, int n,
   }
   uint32_t row_taken[2] = {0, 0};                                      // lane l: which candidates of rows l and 32 + l were chosen
   int32_t *dst2 = token ? sel : parts;                                 // without tokens the partitions are the selection
-#pragma unroll 1
+#pragma unroll kRowUnroll
   for (int j = 0; j < R; ++j) {
     const uint32_t key = j < nvr ? mykeys[32 * j] : 0u;
     const bool g = j < nvr && key > thr, e = j < nvr && key == thr;
