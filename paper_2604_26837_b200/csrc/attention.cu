@@ -350,10 +350,26 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
   float *s_mx = s_red + kThreads;                                 // [G] the set's max per head
   float *s_den = s_mx + G;                                        // [G]
   float *s_scale = s_den + G;                                     // [kMergeTile][G]
+  float *s_sum = s_scale + kMergeTile * G;                        // [kMergeTile][G] (single-tile form only)
+  // A set of at most kMergeTile chunks (every decode step of the benchmark configurations) reads
+  // its (max, sum) pairs from memory once, all loads of a thread in flight together; larger
+  // sets take three passes over them, tile by tile.
+  const bool one_tile = n_chunks <= kMergeTile;
   {
     float mx = -INFINITY;
-    for (int e = threadIdx.x; e < n_chunks * G; e += kThreads)
-      mx = fmaxf(mx, __ldcg(parts + (size_t)e * kPartStride + kHeadDim));
+    if (one_tile) {
+#pragma unroll 4
+      for (int e = threadIdx.x; e < n_chunks * G; e += kThreads) {
+        const float *pp = parts + (size_t)e * kPartStride + kHeadDim;
+        const float mk = __ldcg(pp), lk = __ldcg(pp + 1);
+        s_scale[e] = mk;
+        s_sum[e] = lk;
+        mx = fmaxf(mx, mk);
+      }
+    } else {
+      for (int e = threadIdx.x; e < n_chunks * G; e += kThreads)
+        mx = fmaxf(mx, __ldcg(parts + (size_t)e * kPartStride + kHeadDim));
+    }
     s_red[threadIdx.x] = mx;
     __syncthreads();
     if (threadIdx.x < G) {
@@ -364,10 +380,19 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
     __syncthreads();
     const float mn = s_mx[threadIdx.x % G];
     float den = 0.f;
-    for (int e = threadIdx.x; e < n_chunks * G; e += kThreads) {
-      const float *pp = parts + (size_t)e * kPartStride;
-      const float mk = __ldcg(pp + kHeadDim);
-      den += mk == -INFINITY ? 0.f : __ldcg(pp + kHeadDim + 1) * exp2f(mk - mn);
+    if (one_tile) {
+      // a thread's own entries: the chunk's maximum gives way to its weight in place
+      for (int e = threadIdx.x; e < n_chunks * G; e += kThreads) {
+        const float mk = s_scale[e], w = mk == -INFINITY ? 0.f : exp2f(mk - mn);
+        s_scale[e] = w;
+        den += mk == -INFINITY ? 0.f : s_sum[e] * w;
+      }
+    } else {
+      for (int e = threadIdx.x; e < n_chunks * G; e += kThreads) {
+        const float *pp = parts + (size_t)e * kPartStride;
+        const float mk = __ldcg(pp + kHeadDim);
+        den += mk == -INFINITY ? 0.f : __ldcg(pp + kHeadDim + 1) * exp2f(mk - mn);
+      }
     }
     s_red[threadIdx.x] = den;
     __syncthreads();
@@ -382,12 +407,14 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
   for (int j = 0; j < G; ++j) a_o[j] = 0.f;
   for (int k0 = 0; k0 < n_chunks; k0 += kMergeTile) {
     const int kn = min(kMergeTile, n_chunks - k0);
-    __syncthreads();                                              // the previous tile's weights have been used
-    for (int e = threadIdx.x; e < kn * G; e += kThreads) {
-      const float mk = __ldcg(parts + ((size_t)k0 * G + e) * kPartStride + kHeadDim);
-      s_scale[e] = mk == -INFINITY ? 0.f : exp2f(mk - s_mx[e % G]);
+    __syncthreads();                                              // the previous tile's weights have been used (one tile: the weights are all written)
+    if (!one_tile) {
+      for (int e = threadIdx.x; e < kn * G; e += kThreads) {
+        const float mk = __ldcg(parts + ((size_t)k0 * G + e) * kPartStride + kHeadDim);
+        s_scale[e] = mk == -INFINITY ? 0.f : exp2f(mk - s_mx[e % G]);
+      }
+      __syncthreads();
     }
-    __syncthreads();
     // a thread's G outputs are channel `threadIdx.x` of every head: the loads of a batch of chunks
     // for all G heads are issued together (their L2 latency is paid once per batch, not once per head)
     const float *pt = parts + (size_t)k0 * G * kPartStride + threadIdx.x;
