@@ -359,6 +359,15 @@ def test_asynchronous_offload_of_a_cluster_prefill():
     assert r["folded"] == 2 * 2 * 32
 
 
+def test_page_minmax_more_pages_than_one_cta_holds():
+    # > 16384 candidate PAGES per set (a 264K-token context): the thread-block cluster selects
+    # whole partitions here (no token masks), its first CTA manages the cache
+    w = _wl(W.PART_PAGE_MINMAX, context=16 * 16500 + 3, topk=64, slots_per_set=100, steps=6, batch=1,
+            num_layers=1, num_q_heads=2, num_kv_heads=1, lru_buckets=8, drift=0.3)
+    r = run_parity(w, check_bytes=False, one_call=True)
+    assert r["stats"]["miss_pages"] > 0
+
+
 @pytest.mark.parametrize("kind", [W.PART_PAGE_MINMAX, W.PART_CLUSTER_CENTROID, W.PART_TOKEN_DOT])
 def test_resident_scoring_grid(kind):
     # the queue-fed form of the scoring kernel (automatic only for long scoring phases), forced

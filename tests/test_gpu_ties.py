@@ -77,6 +77,21 @@ def test_token_rows_repeat_across_the_slices_of_the_cluster_top_k():
               batch=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8)
     r = run_parity(w, check_bytes=False, one_call=True)
     assert r["tied_at_k"] == 2 * 6
+    # groups of 520 equal keys (period 40): larger than what the select ranks directly, so the
+    # threshold key is decided digit by digit to its last bit, and the k-th place falls inside a group
+    w = _tied(W.PART_TOKEN_DOT, context=16 * 1300 + 5, tie_period=40, topk=300, slots_per_set=60, steps=8,
+              batch=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8)
+    r = run_parity(w, check_bytes=False, one_call=True)
+    assert r["tied_at_k"] == 2 * 8
+
+
+def test_pages_repeat_across_the_slices_of_the_cluster_top_k():
+    # page granularity through the cluster kernel: 16500 candidate pages per set whose keys repeat
+    # with a period of 7 pages (2357 equal bounds per group, spread over all slices)
+    w = _tied(W.PART_PAGE_MINMAX, context=16 * 16500 + 3, tie_period=16 * 7, topk=64, slots_per_set=100, steps=6,
+              batch=1, num_layers=1, num_q_heads=2, num_kv_heads=1, lru_buckets=8)
+    r = run_parity(w, check_bytes=False, one_call=True)
+    assert r["tied_at_k"] == 6
 
 
 def test_clusters_with_equal_centroids():
