@@ -418,22 +418,24 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
     // a thread's G outputs are channel `threadIdx.x` of every head: the loads of a batch of chunks
     // for all G heads are issued together (their L2 latency is paid once per batch, not once per head)
     const float *pt = parts + (size_t)k0 * G * kPartStride + threadIdx.x;
-    constexpr int kB = G >= 8 ? 4 : 8;                            // chunks per batch: 32 loads in flight per thread
-    int k = 0;
-    for (; k + kB <= kn; k += kB) {
+    // 64 loads in flight per thread; the last batch is padded with its last chunk at weight zero
+    // (one loop, no chunk-by-chunk remainder whose loads would each wait for the one before)
+    constexpr int kB = G >= 8 ? 8 : G == 4 ? 16 : 32;
+#pragma unroll 1
+    for (int k = 0; k < kn; k += kB) {
       float v[G][kB];
 #pragma unroll
       for (int j = 0; j < G; ++j)
 #pragma unroll
-        for (int i = 0; i < kB; ++i) v[j][i] = __ldcg(pt + ((size_t)(k + i) * G + j) * kPartStride);
+        for (int i = 0; i < kB; ++i) v[j][i] = __ldcg(pt + ((size_t)min(k + i, kn - 1) * G + j) * kPartStride);
 #pragma unroll
       for (int j = 0; j < G; ++j)
 #pragma unroll
-        for (int i = 0; i < kB; ++i) a_o[j] = fmaf(v[j][i], s_scale[(k + i) * G + j], a_o[j]);
+        for (int i = 0; i < kB; ++i) {
+          const float w = k + i < kn ? s_scale[(k + i) * G + j] : 0.f;
+          a_o[j] = fmaf(v[j][i], w, a_o[j]);
+        }
     }
-    for (; k < kn; ++k)
-#pragma unroll
-      for (int j = 0; j < G; ++j) a_o[j] = fmaf(__ldcg(pt + ((size_t)k * G + j) * kPartStride), s_scale[k * G + j], a_o[j]);
   }
 #pragma unroll
   for (int j = 0; j < G; ++j) {
