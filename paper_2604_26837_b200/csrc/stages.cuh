@@ -1447,9 +1447,11 @@ __device__ __forceinline__ void cache_fast(const DevCtx &c, const Batch &bt, int
                    : oseg >= 0 ? (c.off_mirror ? c.off_mirror : c.off_pool)[((size_t)oseg << c.seg_shift) + (p & seg_mask)] : -1;
       }
     }
+    // two single-barrier scans on buffers of their own: each one's barrier also separates the
+    // other buffer's reads from its next writes
     uint32_t tot_a, tot_m;
-    const uint32_t ex_a = block_scan<T>(npg, sh.wsum, &tot_a);
-    const uint32_t ex_m = block_scan<T>(miss ? npg : 0, sh.wsum, &tot_m);
+    const uint32_t ex_a = block_scan1<T>(npg, sh.wsum, &tot_a);
+    const uint32_t ex_m = block_scan1<T>(miss ? npg : 0, sh.wsum + 16, &tot_m);
     if (r < np) {
       s_pageoff[r] = run_all + ex_a;
       s_missoff[r] = run_miss + ex_m;
