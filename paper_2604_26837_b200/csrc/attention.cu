@@ -179,45 +179,44 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
   // launch order: chunk 0 of every set first (the chunks that hold the missed pages), or set by set
   const int b = bt.attn_set_major ? blockIdx.y : blockIdx.x, chunk = bt.attn_set_major ? blockIdx.x : blockIdx.y;
   const int first = chunk * kChunkPages;
-  bool slots_known = true;                 // false: the chunk holds early descriptors only
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int np = 0, nm = 0;                      // pages in the set's list; how many of them are early descriptors
   if (c.ready) {
     // A set raises two flags.  The first says that its missed pages are listed (the leading
-    // n_miss descriptors, slot still open): a chunk made of those alone starts at once, so
-    // the pages cross the host link while the cache manager is still freeing slots for them.
-    // Every other chunk waits for the second flag (complete list) and for the tail page.
+    // n_miss descriptors, slot still open): a warp requests those of its pages at once, so the
+    // pages cross the host link while the cache manager is still freeing slots for them.  For
+    // its other pages a warp waits for the second flag (complete list) and for the tail page.
     __shared__ int sh_ok, sh_np, sh_nm;
     if (threadIdx.x == 0) {
-      int ok = flag_wait(c, c.ready1 + b, bt.epoch);
-      int np_ = 0, nm_ = 0;
-      if (ok) {
-        np_ = max(0, min(c.n_pages[b], c.max_pages + c.tail_cap)); nm_ = c.n_miss[b];
-        if (first < np_ && min(np_, first + kChunkPages) > nm_)
-          ok = flag_wait(c, c.ready + b, bt.epoch) && flag_wait(c, c.tail_ready + b, bt.epoch);
-      }
-      sh_ok = ok; sh_np = np_; sh_nm = nm_;
+      const int ok = flag_wait(c, c.ready1 + b, bt.epoch);
+      // a count beyond the list's stride can neither read past the set's row nor leave the merge
+      // waiting for chunks that no CTA of the grid owns
+      sh_np = ok ? max(0, min(c.n_pages[b], c.max_pages + c.tail_cap)) : 0;
+      sh_nm = ok ? c.n_miss[b] : 0;
+      sh_ok = ok;
     }
     __syncthreads();
     if (!sh_ok) return;
-    slots_known = first >= sh_np || min(sh_np, first + kChunkPages) > sh_nm;
+    np = sh_np; nm = sh_nm;
   } else {
     pdl_wait_prev();
+    np = max(0, min(c.n_pages[b], c.max_pages + c.tail_cap));
   }
   if (chunk == 0) dbg_ta(b, 10);
-  // a count beyond the list's stride can neither read past the set's row nor leave the merge
-  // waiting for chunks that no CTA of the grid owns
-  const int np = max(0, min(c.n_pages[b], c.max_pages + c.tail_cap));
   if (first >= np) return;
   const int last = min(np, first + kChunkPages);
   const int i_req = b / c.Hkv, head = b % c.Hkv;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t pl = (size_t)b * (c.max_pages + c.tail_cap);
 
-  // the warp's two pages; the one that has to cross the host link is waited for last
+  // the warp's two pages.  Early descriptors lead the list, so the first page is early whenever
+  // the second is.  Requests go out, and are waited for, in this order: early pages, then (after
+  // the second flag) the others, of which the one that has to cross the host link comes last.
   int pg[2] = {first + warp, first + warp + kAttnWarps};
   int n_mine = (pg[0] < last) + (pg[1] < last);
+  const int n_early = (n_mine >= 1 && pg[0] < nm) + (n_mine >= 2 && pg[1] < nm);
   int src[2] = {0, 0}, fill[2] = {-1, -1}, open_idx[2] = {-1, -1};
   uint32_t mask[2] = {0, 0};
-  for (int i = 0; i < n_mine; ++i) {
+  auto describe = [&](int i) {
     if (c.page_desc) {                      // work-ordered descriptors written by the cache manager
       const int4 dsc = c.page_desc[pl + pg[i]];
       src[i] = dsc.x; fill[i] = dsc.y; mask[i] = (uint32_t)dsc.z;
@@ -242,22 +241,40 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
     // a descriptor that points outside the pools is dropped (and reported), never followed
     const bool ok = (src[i] >= 0 ? src[i] < c.n_gpu_pages : ~src[i] < c.n_host_pages) && fill[i] < c.n_host_pages;
     if (!ok) { if (lane == 0) dev_error(c, kErrBounds); src[i] = 0; fill[i] = -1; mask[i] = 0; open_idx[i] = -1; }
-  }
-  if (n_mine == 2 && (fill[0] >= 0 || src[0] < 0) && !(fill[1] >= 0 || src[1] < 0)) {
-    int t = src[0]; src[0] = src[1]; src[1] = t;
-    t = fill[0]; fill[0] = fill[1]; fill[1] = t;
-    t = open_idx[0]; open_idx[0] = open_idx[1]; open_idx[1] = t;
-    uint32_t u = mask[0]; mask[0] = mask[1]; mask[1] = u;
-  }
-  if (chunk == 0) dbg_ta(b, 11);
+  };
   uint8_t *spage[2] = {smem_pages + (size_t)(2 * warp) * kPageBytes, smem_pages + (size_t)(2 * warp + 1) * kPageBytes};
-  for (int i = 0; i < 2; ++i) {
-    if (i < n_mine) {
-      const uint8_t *from = fill[i] >= 0 ? c.host_pages + (size_t)fill[i] * kPageBytes : page_ptr(c, src[i]);
-      request_page(smem_u32(spage[i]), from, lane);
+  auto request = [&](int i) {
+    const uint8_t *from = fill[i] >= 0 ? c.host_pages + (size_t)fill[i] * kPageBytes : page_ptr(c, src[i]);
+    request_page(smem_u32(spage[i]), from, lane);
+  };
+  // one cp.async group per page slot, in slot order (an empty group where the warp has no page)
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+    if (i < n_early) { describe(i); request(i); cp_async_commit(); }
+  if (n_early < n_mine) {
+    if (c.ready) {
+      int ok = 1;
+      if (lane == 0) ok = flag_wait(c, c.ready + b, bt.epoch) && flag_wait(c, c.tail_ready + b, bt.epoch);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) n_mine = n_early;            // reported by the wait: the warp attends what it has and the CTA still arrives
     }
-    cp_async_commit();
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      if (i >= n_early && i < n_mine) describe(i);
+    if (n_early == 0 && n_mine == 2 && (fill[0] >= 0 || src[0] < 0) && !(fill[1] >= 0 || src[1] < 0)) {
+      int t = src[0]; src[0] = src[1]; src[1] = t;
+      t = fill[0]; fill[0] = fill[1]; fill[1] = t;
+      t = open_idx[0]; open_idx[0] = open_idx[1]; open_idx[1] = t;
+      uint32_t u = mask[0]; mask[0] = mask[1]; mask[1] = u;
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      if (i >= n_early && i < n_mine) { request(i); cp_async_commit(); }
   }
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+    if (i >= n_mine) cp_async_commit();
+  if (chunk == 0) dbg_ta(b, 11);
 
   // Q as A-operand fragments: row = lane/4 (query head, zero beyond G), 8 k-steps of 16 channels
   uint32_t qa[8][2];
@@ -282,14 +299,14 @@ __device__ __forceinline__ void attn_cta(const DevCtx &c, const Batch &bt, const
   if (chunk == 0) dbg_ta(b, 12);
   if (n_mine >= 1) {
     attend_page(smem_u32(spage[0]), qa, mask[0], scale2, acc, lane);
-    if (fill[0] >= 0) fetched_page_to_slot(c, bt, b, pl, spage[0], src[0], open_idx[0], slots_known, lane);
+    if (fill[0] >= 0) fetched_page_to_slot(c, bt, b, pl, spage[0], src[0], open_idx[0], n_early < 1, lane);
   }
   cp_async_wait<0>();
   __syncwarp();
   if (chunk == 0) dbg_ta(b, 13);
   if (n_mine >= 2) {
     attend_page(smem_u32(spage[1]), qa, mask[1], scale2, acc, lane);
-    if (fill[1] >= 0) fetched_page_to_slot(c, bt, b, pl, spage[1], src[1], open_idx[1], slots_known, lane);
+    if (fill[1] >= 0) fetched_page_to_slot(c, bt, b, pl, spage[1], src[1], open_idx[1], n_early < 2, lane);
   }
 
   // row sums live in the 4 lanes of a quad
