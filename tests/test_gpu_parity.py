@@ -359,6 +359,15 @@ def test_asynchronous_offload_of_a_cluster_prefill():
     assert r["folded"] == 2 * 2 * 32
 
 
+def test_token_dot_more_keys_resident_scoring_grid():
+    # the queue-fed resident scoring grid in front of the cluster top-k: several items per CTA,
+    # ragged last segments, tail items
+    w = _wl(W.PART_TOKEN_DOT, context=16 * 1300 + 5, topk=300, slots_per_set=120, steps=20, batch=2,
+            num_layers=1, num_q_heads=4, num_kv_heads=2, lru_buckets=8, drift=0.3, kv_recipe="page_centre", centre_sd=0.5)
+    r = run_parity(w, check_bytes=False, one_call=True, resident_scoring=1)
+    assert r["stats"]["evicted_pages"] > 0
+
+
 def test_page_minmax_more_pages_than_one_cta_holds():
     # > 16384 candidate PAGES per set (a 264K-token context): the thread-block cluster selects
     # whole partitions here (no token masks), its first CTA manages the cache
